@@ -1,0 +1,263 @@
+/*
+ * tad - evaluation of element-wise defined tensor expressions and of the
+ * derivative expressions obtained by the element-wise derivation algorithm of
+ * "Automatic Differentiation for Tensor Algebras" (Urban & van der Smagt, 2017).
+ *
+ * Model (Sec. 5.1 and Sec. 5.2 of the paper).  An output tensor f is defined
+ * element by element,
+ *
+ *     f[alpha] = fbar( x^1[A^1 alpha_hat + o^1], ..., x^P[A^P alpha_hat + o^P] ),
+ *
+ * where alpha_hat = [alpha, k_1, ..., k_S] is the output multi-index extended by
+ * the indices of the sums that occur inside the scalar function fbar, every A is
+ * an integer matrix and every o an integer offset (the paper has o = 0; offsets
+ * are an extension: beta is replaced by beta - o in every formula).  Given
+ * df = dl/df the library evaluates, for every argument,
+ *
+ *     dx^p[beta] = delta(C (beta-o)) * sum_{z in Sigma(beta)} df[alpha] * d fbar / d x^p
+ *                  at alpha_hat = I (beta-o) + K z                    (final equation of Sec. 5.1)
+ *
+ * with I, K, C from the Smith normal form of A (Sec. 4.1) and the summation
+ * ranges Sigma from Fourier-Motzkin elimination (Sec. 4.2), as laid out in the
+ * element-wise derivation algorithm of Sec. 5.3.
+ *
+ * Conventions
+ *   - all tensors are float32, contiguous, row-major, zero-based (Sec. 6);
+ *   - tad_compile / tad_plan_* are host-only and touch no GPU;
+ *   - tad_forward / tad_backward take DEVICE pointers, enqueue work on the given
+ *     CUDA stream (a cudaStream_t passed as void*, NULL = default stream), do not
+ *     synchronise and allocate nothing;
+ *   - the caller owns every buffer; a plan is immutable and may be shared;
+ *   - every function returns a status; tad_last_error() gives a thread-local text.
+ */
+#ifndef TAD_INCLUDE_TAD_H
+#define TAD_INCLUDE_TAD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tad_plan tad_plan;   /* opaque, owned by the library, freed by tad_destroy */
+
+typedef enum {
+    TAD_OK = 0,
+    TAD_ERR_INVALID_ARG = 1,   /* NULL pointer, negative size, bad index */
+    TAD_ERR_BAD_EXPR = 2,      /* malformed node list (order, operands, sum indices) */
+    TAD_ERR_OUT_OF_RANGE = 3,  /* an index expression leaves its argument's shape */
+    TAD_ERR_OVERFLOW = 4,      /* exact integer arithmetic left int64 / a tensor has >= 2^31 elements */
+    TAD_ERR_UNSUPPORTED = 5,   /* valid but beyond the limits stated below */
+    TAD_ERR_WORKSPACE = 6,     /* workspace too small or misaligned */
+    TAD_ERR_CUDA = 7,          /* a CUDA runtime call failed; see tad_last_error() */
+    TAD_ERR_NOMEM = 8
+} tad_status;
+
+/* Elementary functions of the scalar expression fbar (Sec. 2: "addition, subtraction,
+ * multiplication, division, trigonometric function, the exponential function, the logarithm"). */
+typedef enum {
+    TAD_OP_CONST = 0,   /* imm */
+    TAD_OP_LOAD = 1,    /* element of an argument, through access[access] */
+    TAD_OP_NEG = 2,
+    TAD_OP_ADD = 3,
+    TAD_OP_SUB = 4,
+    TAD_OP_MUL = 5,
+    TAD_OP_DIV = 6,
+    TAD_OP_POWI = 7,    /* in0 ** ipow, literal integer exponent (the ** of Sec. 6) */
+    TAD_OP_EXP = 8,
+    TAD_OP_LOG = 9,
+    TAD_OP_SIN = 10,
+    TAD_OP_COS = 11,
+    TAD_OP_TANH = 12,
+    TAD_OP_SINH = 13,
+    TAD_OP_COSH = 14,
+    TAD_OP_SUM = 15     /* sum of in0 over alpha_hat[sum_idx] = sum_lo .. sum_hi (Sec. 5.2) */
+} tad_op;
+
+/* One index expression of one argument: x^arg[A alpha_hat + offset]  (Sec. 5.1). */
+typedef struct {
+    int32_t arg;             /* which tensor argument, 0 <= arg < n_args */
+    const int64_t *A;        /* arg_rank[arg] x n_idx, row-major; n_idx = n_out_dims + n_sum_idx */
+    const int64_t *offset;   /* arg_rank[arg] entries */
+} tad_access;
+
+typedef struct {
+    int32_t op;              /* tad_op */
+    int32_t in0, in1;        /* operand node ids (< own id), -1 if unused */
+    int32_t access;          /* TAD_OP_LOAD: index into tad_expr.access */
+    int32_t ipow;            /* TAD_OP_POWI */
+    int32_t sum_idx;         /* TAD_OP_SUM: position of the sum's index in alpha_hat, >= n_out_dims */
+    int64_t sum_lo, sum_hi;  /* TAD_OP_SUM: inclusive constant range (a convex integer set, Sec. 5.2) */
+    double imm;              /* TAD_OP_CONST */
+} tad_node;
+
+typedef struct {
+    int32_t n_out_dims;                 /* D_f */
+    const int64_t *out_shape;           /* N^f */
+    int32_t n_sum_idx;                  /* number of sum indices appended to alpha */
+    int32_t n_args;                     /* P */
+    const int32_t *arg_rank;            /* D_p */
+    const int64_t *const *arg_shape;    /* N^p */
+    int32_t n_access;
+    const tad_access *access;
+    int32_t n_nodes;
+    const tad_node *nodes;              /* topological order, root last */
+} tad_expr;
+
+typedef struct {
+    int32_t debug_bounds;   /* non-zero: kernels range-check every computed address, skip bad
+                               accesses and record the first one (tad_debug_status) */
+    int32_t reserved[7];    /* must be zero */
+} tad_options;
+
+/* Limits: n_idx <= 8, argument rank <= 4, kernel dimension kappa <= 4, every tensor
+ * < 2^31 elements, compiled program <= a few KB of bytecode (TAD_ERR_UNSUPPORTED beyond).
+ * Every sum index belongs to exactly one sum node; a non-constant node must have one
+ * set of enclosing sums on every path from the root. */
+#define TAD_MAX_IDX 8
+#define TAD_MAX_RANK 4
+#define TAD_MAX_KAPPA 4
+#define TAD_MAX_BOUND_ROWS 16
+
+/*
+ * tad_compile: the element-wise derivation algorithm of Sec. 5.3, once per expression.
+ * For every index expression: Smith normal form of A restricted to the output indices and
+ * the enclosing sum indices (Sec. 4.1; extended Euclid for the Bezout factors), cokernel /
+ * pseudo-inverse / kernel, Fourier-Motzkin elimination of the box constraints written in
+ * the kernel coordinates z (Sec. 4.2), scalar reverse-mode differentiation of fbar (Sec. 2)
+ * and emission of bytecode for the forward and the derivative expressions.
+ * opt may be NULL.  *out is written only on TAD_OK.  Host only.
+ */
+tad_status tad_compile(const tad_expr *expr, const tad_options *opt, tad_plan **out);
+
+/* Frees a plan (NULL is allowed).  The caller makes sure no launch still uses it. */
+void tad_destroy(tad_plan *plan);
+
+/* Bytes of device workspace tad_backward needs for this plan (may be 0).  The workspace
+ * must be 256-byte aligned.  It holds the partial sums of gradients whose summation is
+ * split over several thread blocks, and the debug word of a debug_bounds plan. */
+size_t tad_workspace_bytes(const tad_plan *plan);
+
+/*
+ * tad_forward: f[alpha] for every alpha of the output box (definition of an element-wise
+ * specified function, Sec. 5.1; inner sums per Sec. 5.2).
+ *   args  host array of n_args DEVICE pointers (read-only inputs), none NULL
+ *   f     DEVICE pointer, prod(out_shape) floats, fully overwritten
+ */
+tad_status tad_forward(const tad_plan *plan, const float *const *args, float *f, void *cuda_stream);
+
+/*
+ * tad_backward: dx^p[beta] for every element of every requested argument, by the final
+ * equation of Sec. 5.1 (gather form: one owner per output element, no atomics, fp32
+ * accumulation); the results of several index expressions of one argument are added
+ * (Sec. 5.3: dx <- 0, then accumulate over q).
+ *   args   host array of n_args DEVICE pointers
+ *   df     DEVICE pointer, prod(out_shape) floats
+ *   dargs  host array of n_args DEVICE pointers; NULL entry = gradient not wanted;
+ *          every requested tensor is fully overwritten (zeros where Gamma(beta) is empty)
+ *   workspace  DEVICE pointer of at least tad_workspace_bytes() bytes (may be NULL if 0)
+ */
+tad_status tad_backward(const tad_plan *plan, const float *const *args, const float *df,
+                        float *const *dargs, void *workspace, size_t workspace_bytes,
+                        void *cuda_stream);
+
+/*
+ * tad_step_host: one forward and one backward pass with HOST buffers (same meaning as
+ * tad_forward followed by tad_backward).  Inputs are copied to the device staging area,
+ * results copied back; all copies and launches are enqueued on the stream and the call
+ * returns after the stream has drained.  Host buffers should be pinned for the copies to
+ * be asynchronous.  staging is a DEVICE buffer of at least tad_staging_bytes() bytes,
+ * 256-byte aligned, that the caller allocated; the library allocates nothing.  h_f and
+ * entries of h_dargs may be NULL (not wanted).  (The paper has no counterpart; it is the
+ * end-to-end entry point.)
+ */
+size_t tad_staging_bytes(const tad_plan *plan);
+tad_status tad_step_host(const tad_plan *plan, const float *const *h_args, const float *h_df,
+                         float *h_f, float *const *h_dargs,
+                         void *staging, size_t staging_bytes, void *cuda_stream);
+
+/* Text of the last non-OK status on the calling thread ("" if none). */
+const char *tad_last_error(void);
+
+/* debug_bounds plans: reads back (and clears) the debug word in `workspace` after
+ * synchronising the stream.  TAD_ERR_OUT_OF_RANGE if a kernel skipped an out-of-range
+ * access since the last query, TAD_OK otherwise. */
+tad_status tad_debug_status(const tad_plan *plan, void *workspace, void *cuda_stream);
+
+/* ------------------------------------------------------------------------- */
+/* Introspection (host only).  These are what the bit-exact plan tests use.   */
+/* ------------------------------------------------------------------------- */
+
+typedef struct {
+    int32_t arg;                 /* argument this index expression reads */
+    int32_t rank;                /* D_p: rows of A */
+    int32_t n_idx;               /* columns of A-hat: output dims + enclosing sum indices */
+    int32_t idx_pos[TAD_MAX_IDX];/* position in alpha_hat of each column */
+    int32_t R;                   /* rank of A-hat (number of non-zero invariant factors) */
+    int32_t kappa;               /* kernel dimension n_idx - R */
+    int64_t A[TAD_MAX_RANK * TAD_MAX_IDX];      /* A-hat, rank x n_idx */
+    int64_t offset[TAD_MAX_RANK];
+    int64_t S[TAD_MAX_RANK];                    /* invariant factors alpha_1..alpha_R (Smith normal form) */
+    int64_t U[TAD_MAX_RANK * TAD_MAX_RANK];     /* rank x rank, S = U A V; rows R.. are the cokernel C */
+    int64_t V[TAD_MAX_IDX * TAD_MAX_IDX];       /* n_idx x n_idx; columns R.. are the kernel K in loop order */
+    int64_t box_lo[TAD_MAX_IDX], box_hi[TAD_MAX_IDX];   /* inclusive range of every column's index */
+    /* Bound rows of the kernel coordinates, loop 0 = outermost:
+     *   ceil(max_r lower[r]) <= z_l <= floor(min_r upper[r]),
+     *   row value = (c0 + sum_j cx[j]*x'_j + sum_{m<l} cz[m]*z_m) / den,  den > 0,
+     * with x' = diag(1/alpha) U_R (beta - o). */
+    int32_t n_lower[TAD_MAX_KAPPA], n_upper[TAD_MAX_KAPPA];
+    int32_t masked;              /* 1 if a cokernel row or an invariant factor > 1 exists */
+    int32_t lane_var;            /* which loop variable the kernel spreads over lanes */
+} tad_access_info;
+
+tad_status tad_plan_access_info(const tad_plan *plan, int32_t access, tad_access_info *out);
+
+/* One bound row of loop `loop` (0 = outermost kernel coordinate) of an index expression.
+ * upper = 0: lower-bound row, 1: upper-bound row.  coef_x has R entries, coef_z `loop` entries. */
+tad_status tad_plan_bound_row(const tad_plan *plan, int32_t access, int32_t loop, int32_t upper,
+                              int32_t row, int64_t *den, int64_t *c0, int64_t *coef_x, int64_t *coef_z);
+
+/*
+ * Enumerates Gamma-hat(beta) of one index expression on the host by walking the plan exactly
+ * as the kernel does (mask, index transform, bound rows, nested ranges).  Writes up to `cap`
+ * multi-indices alpha_hat (n_idx int64 each, in idx_pos order) and always the full count.
+ */
+tad_status tad_plan_enumerate(const tad_plan *plan, int32_t access, const int64_t *beta,
+                              int64_t *alpha_hat_out, size_t cap, size_t *n_terms);
+
+typedef struct {
+    int64_t outputs;        /* elements written */
+    int64_t terms;          /* sum over outputs of |Gamma-hat| (0 for the forward kernel) */
+    double alg_bytes;       /* distinct elements read once + outputs written once, in bytes */
+    double alg_flops;       /* each expression node once per distinct binding of the indices it depends on */
+    double alg_transcendentals;
+    int32_t bytecode_words; /* length of the program the interpreter runs */
+    int32_t n_launches;     /* kernel launches this part issues */
+} tad_kernel_stats;
+
+/* which = -1: forward kernel; which = q: backward kernel of index expression q. */
+tad_status tad_plan_kernel_stats(const tad_plan *plan, int32_t which, tad_kernel_stats *out);
+
+/* Human-readable listing of the compiled program (`which` as above); returns bytes needed. */
+size_t tad_plan_disassemble(const tad_plan *plan, int32_t which, char *buf, size_t cap);
+
+/* Host-only pieces of Sec. 4, exported for tests.  Matrices are row-major int64. */
+tad_status tad_extended_euclid(int64_t a, int64_t b, int64_t *gcd, int64_t *x, int64_t *y);
+tad_status tad_smith_normal_form(const int64_t *A, int32_t n_rows, int32_t n_cols,
+                                 int64_t *S, int64_t *U, int64_t *V, int32_t *rank);
+/* Fourier-Motzkin elimination of  A z >= b  (b symbolic) in the order z_1 (eliminated first,
+ * innermost loop) .. z_M (Algorithm of Sec. 4.2).  Per variable k the bounds are
+ *   z_k >= (L b + L-hat z) / den   and   z_k <= (H b + H-hat z) / den
+ * with integer rows and a positive denominator per row; F b <= 0 is the feasibility test.
+ * Row r of variable k is stored at index k * cap_rows + r. */
+tad_status tad_fourier_motzkin(const int64_t *A, int32_t n_rows, int32_t n_cols, int32_t cap_rows,
+                               int32_t *n_lower, int32_t *n_upper,
+                               int64_t *L_num, int64_t *Lhat_num, int64_t *L_den,
+                               int64_t *H_num, int64_t *Hhat_num, int64_t *H_den,
+                               int32_t *n_feas, int64_t *F_num);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TAD_INCLUDE_TAD_H */
