@@ -1,0 +1,5 @@
+"""B200-native evaluation of element-wise defined tensor expressions and of their derivative
+expressions (Urban & van der Smagt, 2017).  Everything runs in libtad.so; this package is the
+ctypes binding."""
+from .binding import (AccessInfo, KernelStats, Plan, TadError, extended_euclid,  # noqa: F401
+                      fourier_motzkin, smith_normal_form, lib, EXPORTS)

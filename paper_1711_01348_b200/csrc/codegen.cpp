@@ -1,0 +1,835 @@
+// Code generator (host only): scalar reverse-mode differentiation of the expression (Sec. 2),
+// sum liberation (Sec. 5.2), loop scheduling and emission of the interpreter's bytecode.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <tuple>
+
+#include "plan.h"
+
+namespace tad {
+
+namespace {
+
+// ---- derivative-graph instances -------------------------------------------------------
+enum IOp {
+    I_CONST, I_LOAD, I_NEG, I_EXP, I_LOG, I_SIN, I_COS, I_TANH, I_SINH, I_COSH,
+    I_SQR, I_POWI, I_ADD, I_SUB, I_MUL, I_DIV, I_MULC, I_ADDC, I_SUM
+};
+
+struct Inst {
+    int op = I_CONST, a = -1, b = -1;
+    int load = -1;          // I_LOAD
+    int ipow = 0;           // I_POWI
+    float imm = 0.f;        // I_CONST, I_MULC, I_ADDC
+    int var = -1;           // I_SUM: bound loop variable
+    int64_t lo = 0, hi = -1;// I_SUM
+    uint32_t deps = 0;      // kernel variables it depends on
+    uint32_t adeps = 0;     // alpha_hat positions (free) it depends on; bit 16+v for bound variable v
+    int uses = 0;
+    int temp = -1;
+    int home_sum = -1;      // innermost bound-sum instance whose variable it depends on (-1: none)
+    int zlevel = 0;         // 1 + deepest kernel-coordinate loop it depends on, 0 if none
+};
+
+struct VarInfo {
+    int kind;               // 0 outer, 1 kernel coordinate, 2 bound sum
+    int64_t ext;            // extent (exact for outer and bound sums, estimate for kernel coordinates)
+    int sum_inst;           // kind 2
+};
+
+struct Gen {
+    tad_plan &p;
+    int q;                               // index expression being differentiated, -1 for forward
+    int n_outer = 0, kappa = 0;
+    std::vector<VarInfo> vars;
+    // affine map of every alpha_hat position over (outer, kernel-coordinate) variables
+    std::vector<int64_t> a_c0;
+    std::vector<std::vector<int64_t>> a_coef;
+    std::vector<bool> a_free_ok;
+    std::vector<Inst> inst;
+    std::map<std::tuple<int, int, int, int, int, int32_t, int>, int> cse;
+    std::vector<TadpLoad> loads;
+    std::map<std::pair<int, uint32_t>, int> val_memo;        // (node, free set) -> inst
+    std::map<std::pair<int, uint32_t>, int> bound_var;       // (sum slot, free set) -> var
+    std::vector<int> zorder;                                  // loop l -> kernel column
+    std::vector<int> zpos;                                    // kernel column -> loop position
+    int lane_var = -1;
+
+    Gen(tad_plan &pl, int acc) : p(pl), q(acc) {}
+
+    int n_idx() const { return p.n_out + p.n_sum; }
+
+    // -- instance construction with common-subexpression elimination
+    int intern(Inst in)
+    {
+        int32_t immbits; std::memcpy(&immbits, &in.imm, 4);
+        auto key = std::make_tuple(in.op, in.a, in.b, in.load, in.ipow, immbits, in.var);
+        auto it = cse.find(key);
+        if (it != cse.end()) return it->second;
+        if (in.op != I_CONST && in.op != I_LOAD && in.op != I_SUM) {
+            in.deps = inst[in.a].deps | (in.b >= 0 ? inst[in.b].deps : 0);
+            in.adeps = inst[in.a].adeps | (in.b >= 0 ? inst[in.b].adeps : 0);
+        }
+        inst.push_back(in);
+        cse[key] = (int)inst.size() - 1;
+        return (int)inst.size() - 1;
+    }
+    int konst(float v) { Inst i; i.op = I_CONST; i.imm = v; return intern(i); }
+    int un(int op, int a) { Inst i; i.op = op; i.a = a; return intern(i); }
+    int neg(int a) { if (inst[a].op == I_NEG) return inst[a].a; return un(I_NEG, a); }
+    int mulc(int a, float c)
+    {
+        if (c == 1.f) return a;
+        if (inst[a].op == I_CONST) return konst(inst[a].imm * c);
+        Inst i; i.op = I_MULC; i.a = a; i.imm = c; return intern(i);
+    }
+    int addc(int a, float c)
+    {
+        if (c == 0.f) return a;
+        if (inst[a].op == I_CONST) return konst(inst[a].imm + c);
+        Inst i; i.op = I_ADDC; i.a = a; i.imm = c; return intern(i);
+    }
+    int bin(int op, int a, int b)
+    {
+        if (op == I_MUL) {
+            if (inst[a].op == I_CONST) return mulc(b, inst[a].imm);
+            if (inst[b].op == I_CONST) return mulc(a, inst[b].imm);
+            if (a == b) return un(I_SQR, a);
+            if (a > b) std::swap(a, b);
+        }
+        if (op == I_ADD) {
+            if (inst[a].op == I_CONST) return addc(b, inst[a].imm);
+            if (inst[b].op == I_CONST) return addc(a, inst[b].imm);
+            if (a > b) std::swap(a, b);
+        }
+        if (op == I_SUB && inst[b].op == I_CONST) return addc(a, -inst[b].imm);
+        if (op == I_DIV && inst[b].op == I_CONST) return mulc(a, 1.f / inst[b].imm);
+        Inst i; i.op = op; i.a = a; i.b = b; return intern(i);
+    }
+    int powi(int a, int n)
+    {
+        if (n == 0) return konst(1.f);
+        if (n == 1) return a;
+        if (n == 2) return un(I_SQR, a);
+        Inst i; i.op = I_POWI; i.a = a; i.ipow = n; return intern(i);
+    }
+
+    // -- loads: element offset affine in the kernel variables
+    int make_load(int ptr, const std::vector<int64_t> &A, const std::vector<int64_t> &off, int rank,
+                  const std::vector<int64_t> &shape, uint32_t free_set, uint32_t scope)
+    {
+        std::vector<int64_t> stride(rank, 1);
+        for (int r = rank - 2; r >= 0; --r) stride[r] = mul_ck(stride[r + 1], shape[r + 1]);
+        int64_t base = 0, elems = 1;
+        for (int r = 0; r < rank; ++r) { base = add_ck(base, mul_ck(stride[r], off[r])); elems *= shape[r]; }
+        std::vector<int64_t> coef(TADP_MAX_VARS, 0);
+        uint32_t adeps = 0;
+        const int nidx = n_idx();
+        for (int d = 0; d < nidx; ++d) {
+            int64_t flat = 0;
+            for (int r = 0; r < rank; ++r) flat = add_ck(flat, mul_ck(stride[r], A[size_t(r) * nidx + d]));
+            if (flat == 0) continue;
+            bool is_sum = d >= p.n_out;
+            int s = d - p.n_out;
+            if (is_sum && !(free_set & (1u << s))) {
+                if (!(scope & (1u << s))) throw BadExpr("internal: load reads a sum index outside its sum");
+                auto it = bound_var.find({s, free_set});
+                if (it == bound_var.end()) throw BadExpr("internal: bound sum variable missing");
+                coef[it->second] = add_ck(coef[it->second], flat);
+                adeps |= 1u << (16 + it->second);
+            } else {
+                if (!a_free_ok[d]) throw BadExpr("internal: free index without an affine map");
+                base = add_ck(base, mul_ck(flat, a_c0[d]));
+                for (size_t v = 0; v < a_coef[d].size(); ++v)
+                    coef[v] = add_ck(coef[v], mul_ck(flat, a_coef[d][v]));
+                adeps |= 1u << d;
+            }
+        }
+        TadpLoad L{};
+        L.ptr = ptr;
+        if (std::llabs(base) >= (int64_t(1) << 31)) throw Overflow();
+        L.base = (int32_t)base;
+        uint32_t deps = 0;
+        for (int v = 0; v < TADP_MAX_VARS; ++v) {
+            if (std::llabs(coef[v]) >= (int64_t(1) << 31)) throw Overflow();
+            L.coef[v] = (int32_t)coef[v];
+            if (coef[v]) deps |= 1u << v;
+        }
+        L.limit = (int32_t)elems;
+        int id = -1;
+        for (size_t i = 0; i < loads.size(); ++i)
+            if (!std::memcmp(&loads[i], &L, sizeof L)) id = (int)i;
+        if (id < 0) {
+            if ((int)loads.size() >= TADP_MAX_LOADS) throw Unsupported("too many distinct loads in one kernel");
+            loads.push_back(L); id = (int)loads.size() - 1;
+        }
+        Inst in; in.op = I_LOAD; in.load = id; in.deps = deps; in.adeps = adeps;
+        return intern(in);
+    }
+
+    int new_var(int kind, int64_t ext)
+    {
+        if ((int)vars.size() >= TADP_MAX_VARS) throw Unsupported("too many loop variables in one kernel");
+        vars.push_back({kind, ext, -1});
+        return (int)vars.size() - 1;
+    }
+
+    // -- value of an expression node with the sums of `free_set` liberated (taken from alpha_hat)
+    int val(int n, uint32_t free_set)
+    {
+        const NodeH &nd = p.nodes[n];
+        if (nd.op == TAD_OP_CONST) return konst((float)nd.imm);
+        auto key = std::make_pair(n, free_set);
+        auto it = val_memo.find(key);
+        if (it != val_memo.end()) return it->second;
+        int r = -1;
+        switch (nd.op) {
+        case TAD_OP_LOAD: {
+            int arg = p.accArg[nd.access];
+            r = make_load(arg, p.accA[nd.access], p.accOff[nd.access], (int)p.arg_shape[arg].size(),
+                          p.arg_shape[arg], free_set, nd.scope);
+            break;
+        }
+        case TAD_OP_NEG: r = neg(val(nd.in0, free_set)); break;
+        case TAD_OP_ADD: { int a = val(nd.in0, free_set), b = val(nd.in1, free_set); r = bin(I_ADD, a, b); break; }
+        case TAD_OP_SUB: { int a = val(nd.in0, free_set), b = val(nd.in1, free_set); r = bin(I_SUB, a, b); break; }
+        case TAD_OP_MUL: { int a = val(nd.in0, free_set), b = val(nd.in1, free_set); r = bin(I_MUL, a, b); break; }
+        case TAD_OP_DIV: { int a = val(nd.in0, free_set), b = val(nd.in1, free_set); r = bin(I_DIV, a, b); break; }
+        case TAD_OP_POWI: r = powi(val(nd.in0, free_set), nd.ipow); break;
+        case TAD_OP_EXP: r = un(I_EXP, val(nd.in0, free_set)); break;
+        case TAD_OP_LOG: r = un(I_LOG, val(nd.in0, free_set)); break;
+        case TAD_OP_SIN: r = un(I_SIN, val(nd.in0, free_set)); break;
+        case TAD_OP_COS: r = un(I_COS, val(nd.in0, free_set)); break;
+        case TAD_OP_TANH: r = un(I_TANH, val(nd.in0, free_set)); break;
+        case TAD_OP_SINH: r = un(I_SINH, val(nd.in0, free_set)); break;
+        case TAD_OP_COSH: r = un(I_COSH, val(nd.in0, free_set)); break;
+        case TAD_OP_SUM: {
+            int s = nd.sum_idx - p.n_out;
+            int v = new_var(2, nd.sum_hi - nd.sum_lo + 1);
+            bound_var[{s, free_set}] = v;
+            int body = val(nd.in0, free_set);
+            Inst in; in.op = I_SUM; in.a = body; in.var = v; in.lo = nd.sum_lo; in.hi = nd.sum_hi;
+            in.deps = inst[body].deps & ~(1u << v);
+            in.adeps = inst[body].adeps & ~(1u << (16 + v));
+            r = intern(in);
+            vars[v].sum_inst = r;
+            break;
+        }
+        default: throw BadExpr("unknown operation");
+        }
+        val_memo[key] = r;
+        return r;
+    }
+
+    // -- reverse accumulation (Sec. 2): the adjoint of the root is df; returns the term Delta
+    //    of Sec. 5.3, i.e. df * d f / d x^{pq} with every sum on the path to the leaf liberated
+    int differentiate(int df_inst)
+    {
+        const int root = (int)p.nodes.size() - 1;
+        std::vector<bool> active(p.nodes.size(), false);
+        for (int n = 0; n <= root; ++n) {
+            const NodeH &nd = p.nodes[n];
+            if (!nd.reachable) continue;
+            if (nd.op == TAD_OP_LOAD) active[n] = nd.access == q;
+            else active[n] = (nd.in0 >= 0 && active[nd.in0]) || (nd.in1 >= 0 && active[nd.in1]);
+        }
+        std::vector<int> adj(p.nodes.size(), -1);
+        if (!active[root]) return -1;
+        adj[root] = df_inst;
+        int total = -1;
+        auto push = [&](int c, int x) {
+            if (c < 0 || !active[c]) return;
+            adj[c] = adj[c] < 0 ? x : bin(I_ADD, adj[c], x);
+        };
+        for (int n = root; n >= 0; --n) {
+            if (!active[n] || adj[n] < 0) continue;
+            const NodeH &nd = p.nodes[n];
+            const uint32_t F = nd.scope;          // every enclosing sum lies on the path: liberated
+            const int g = adj[n];
+            switch (nd.op) {
+            case TAD_OP_LOAD: total = total < 0 ? g : bin(I_ADD, total, g); break;
+            case TAD_OP_NEG: push(nd.in0, neg(g)); break;
+            case TAD_OP_ADD: push(nd.in0, g); push(nd.in1, g); break;
+            case TAD_OP_SUB: push(nd.in0, g); push(nd.in1, neg(g)); break;
+            case TAD_OP_MUL:
+                if (active[nd.in0]) push(nd.in0, bin(I_MUL, g, val(nd.in1, F)));
+                if (active[nd.in1]) push(nd.in1, bin(I_MUL, g, val(nd.in0, F)));
+                break;
+            case TAD_OP_DIV:
+                if (active[nd.in0]) push(nd.in0, bin(I_DIV, g, val(nd.in1, F)));
+                if (active[nd.in1]) push(nd.in1, neg(bin(I_DIV, bin(I_MUL, g, val(n, F)), val(nd.in1, F))));
+                break;
+            case TAD_OP_POWI:
+                if (nd.ipow != 0)
+                    push(nd.in0, bin(I_MUL, g, mulc(powi(val(nd.in0, F), nd.ipow - 1), (float)nd.ipow)));
+                break;
+            case TAD_OP_EXP: push(nd.in0, bin(I_MUL, g, val(n, F))); break;
+            case TAD_OP_LOG: push(nd.in0, bin(I_DIV, g, val(nd.in0, F))); break;
+            case TAD_OP_SIN: push(nd.in0, bin(I_MUL, g, un(I_COS, val(nd.in0, F)))); break;
+            case TAD_OP_COS: push(nd.in0, neg(bin(I_MUL, g, un(I_SIN, val(nd.in0, F))))); break;
+            case TAD_OP_TANH: {
+                int t = val(n, F);
+                push(nd.in0, bin(I_MUL, g, addc(neg(un(I_SQR, t)), 1.f)));
+                break;
+            }
+            case TAD_OP_SINH: push(nd.in0, bin(I_MUL, g, un(I_COSH, val(nd.in0, F)))); break;
+            case TAD_OP_COSH: push(nd.in0, bin(I_MUL, g, un(I_SINH, val(nd.in0, F)))); break;
+            case TAD_OP_SUM: push(nd.in0, g); break;     // d s-bar / d s = 1 at the liberated index
+            default: break;
+            }
+        }
+        return total;
+    }
+};
+
+// ---- scheduling and emission ----------------------------------------------------------
+
+const char *op_name(int op)
+{
+    static const char *names[] = {"END", "CONST", "LOAD", "NEG", "EXP", "LOG", "SIN", "COS", "TANH", "SINH", "COSH",
+                                  "SQR", "POWI", "ADD", "SUB", "MUL", "DIV", "MULC", "ADDC", "FMA", "LDT", "STT",
+                                  "ZERO", "SUMADD", "SLOOP", "SEND", "ZLOOP", "ZEND", "ACC"};
+    return op < P_NUM_OPS ? names[op] : "?";
+}
+
+struct Emitter {
+    Gen &g;
+    std::vector<TadpInsn> code;
+    std::vector<TadpLoop> loops;
+    int depth = 0, max_depth = 0;
+    std::string listing;
+
+    explicit Emitter(Gen &gen) : g(gen) {}
+
+    int emit(int op, int a = 0, int b = 0, int32_t imm = 0, int delta = 0)
+    {
+        if (depth + delta > TADP_MAX_DEPTH - 1) throw Unsupported("expression needs a deeper operand stack");
+        TadpInsn w{};
+        w.handler = (uint16_t)(op * TADP_MAX_DEPTH + depth);
+        w.a = (uint8_t)a; w.b = (uint8_t)b; w.imm = imm;
+        code.push_back(w);
+        char line[160];
+        float f; std::memcpy(&f, &imm, 4);
+        std::snprintf(line, sizeof line, "%3zu  d=%d  %-7s a=%d imm=%d (%g)\n", code.size() - 1, depth, op_name(op), a, imm, (double)f);
+        listing += line;
+        depth += delta;
+        max_depth = std::max(max_depth, depth);
+        if ((int)code.size() >= TADP_MAX_CODE) throw Unsupported("program longer than TADP_MAX_CODE words");
+        return (int)code.size() - 1;
+    }
+    static int32_t fbits(float f) { int32_t b; std::memcpy(&b, &f, 4); return b; }
+
+    bool inline_ok(int i) const { return g.inst[i].temp < 0; }
+
+    // emits code that leaves the value of instance i on the stack
+    void expr(int i)
+    {
+        if (g.inst[i].temp >= 0) { emit(P_LDT, g.inst[i].temp, 0, 0, +1); return; }
+        body(i);
+    }
+    void body(int i)
+    {
+        const Inst in = g.inst[i];
+        switch (in.op) {
+        case I_CONST: emit(P_CONST, 0, 0, fbits(in.imm), +1); break;
+        case I_LOAD: emit(P_LOAD, in.load, 0, 0, +1); break;
+        case I_NEG: expr(in.a); emit(P_NEG); break;
+        case I_EXP: expr(in.a); emit(P_EXP); break;
+        case I_LOG: expr(in.a); emit(P_LOG); break;
+        case I_SIN: expr(in.a); emit(P_SIN); break;
+        case I_COS: expr(in.a); emit(P_COS); break;
+        case I_TANH: expr(in.a); emit(P_TANH); break;
+        case I_SINH: expr(in.a); emit(P_SINH); break;
+        case I_COSH: expr(in.a); emit(P_COSH); break;
+        case I_SQR: expr(in.a); emit(P_SQR); break;
+        case I_POWI: expr(in.a); emit(P_POWI, 0, 0, in.ipow); break;
+        case I_MULC: expr(in.a); emit(P_MULC, 0, 0, fbits(in.imm)); break;
+        case I_ADDC: expr(in.a); emit(P_ADDC, 0, 0, fbits(in.imm)); break;
+        case I_ADD: {
+            // a*b + c as one fused operation when the product is used only here
+            int m = -1, o = -1;
+            if (g.inst[in.a].op == I_MUL && inline_ok(in.a)) { m = in.a; o = in.b; }
+            else if (g.inst[in.b].op == I_MUL && inline_ok(in.b)) { m = in.b; o = in.a; }
+            if (m >= 0) { expr(g.inst[m].a); expr(g.inst[m].b); expr(o); emit(P_FMA, 0, 0, 0, -2); }
+            else { expr(in.a); expr(in.b); emit(P_ADD, 0, 0, 0, -1); }
+            break;
+        }
+        case I_SUB: expr(in.a); expr(in.b); emit(P_SUB, 0, 0, 0, -1); break;
+        case I_MUL: expr(in.a); expr(in.b); emit(P_MUL, 0, 0, 0, -1); break;
+        case I_DIV: expr(in.a); expr(in.b); emit(P_DIV, 0, 0, 0, -1); break;
+        case I_SUM: {
+            TadpLoop L{};
+            L.var = in.var; L.const_lo = (int32_t)in.lo; L.const_hi = (int32_t)in.hi;
+            if ((int)loops.size() >= TADP_MAX_LOOPS) throw Unsupported("too many loops in one kernel");
+            loops.push_back(L);
+            int id = (int)loops.size() - 1;
+            emit(P_ZERO, 0, 0, 0, +1);
+            int begin = emit(P_SLOOP, id);
+            temps_of_sum(i);
+            expr(in.a);
+            emit(P_SUMADD, 0, 0, 0, -1);
+            int end = emit(P_SEND, id, 0, begin + 1);
+            code[begin].imm = end + 1;
+            break;
+        }
+        }
+    }
+    void temps_of_sum(int sum_inst)
+    {
+        for (int i = 0; i < (int)g.inst.size(); ++i)
+            if (g.inst[i].temp >= 0 && g.inst[i].uses > 0 && g.inst[i].home_sum == sum_inst) { body(i); emit(P_STT, g.inst[i].temp, 0, 0, -1); }
+    }
+    void temps_of_level(int level)
+    {
+        for (int i = 0; i < (int)g.inst.size(); ++i)
+            if (g.inst[i].temp >= 0 && g.inst[i].uses > 0 && g.inst[i].home_sum < 0 && g.inst[i].zlevel == level) { body(i); emit(P_STT, g.inst[i].temp, 0, 0, -1); }
+    }
+};
+
+int64_t kernel_col_extent(const AccessPlan &ap, int col)
+{
+    int64_t best = INT64_MAX;
+    for (int d = 0; d < ap.n; ++d) {
+        int64_t k = std::llabs(ap.V(d, ap.R + col));
+        if (k) best = std::min(best, (ap.box_hi[d] - ap.box_lo[d]) / k + 1);
+    }
+    return best == INT64_MAX ? 1 : best;
+}
+
+double inst_weight(const Inst &in)
+{
+    switch (in.op) {
+    case I_CONST: return 0.0;
+    case I_LOAD: return 2.0;
+    case I_EXP: case I_LOG: case I_SIN: case I_COS: case I_TANH: case I_SINH: case I_COSH: return 8.0;
+    case I_DIV: return 4.0;
+    case I_POWI: return (double)std::max(1, std::abs(in.ipow) - 1);
+    default: return 1.0;
+    }
+}
+
+// marks use counts of everything reachable from `root`
+void count_uses(Gen &g, int root)
+{
+    for (Inst &in : g.inst) in.uses = 0;
+    std::vector<int> stack{root};
+    g.inst[root].uses = 1;
+    std::vector<bool> seen(g.inst.size(), false);
+    seen[root] = true;
+    while (!stack.empty()) {
+        int i = stack.back(); stack.pop_back();
+        for (int c : {g.inst[i].a, g.inst[i].b}) {
+            if (c < 0) continue;
+            g.inst[c].uses++;
+            if (!seen[c]) { seen[c] = true; stack.push_back(c); }
+        }
+    }
+}
+
+// home of every instance for the current loop order
+void place(Gen &g)
+{
+    std::vector<int> sum_depth(g.vars.size(), 0);
+    for (Inst &in : g.inst) {
+        in.zlevel = 0;
+        for (int col = 0; col < g.kappa; ++col)
+            if (in.deps & (1u << (g.n_outer + col))) in.zlevel = std::max(in.zlevel, g.zpos[col] + 1);
+    }
+    // depth of a bound sum = 1 + max depth of the bound variables its own instance depends on
+    bool changed = true;
+    while (changed) {
+        changed = false;
+        for (int v = 0; v < (int)g.vars.size(); ++v) {
+            if (g.vars[v].kind != 2 || g.vars[v].sum_inst < 0) continue;
+            int d = 1;
+            for (int w = 0; w < (int)g.vars.size(); ++w)
+                if (g.vars[w].kind == 2 && (g.inst[g.vars[v].sum_inst].deps & (1u << w))) d = std::max(d, sum_depth[w] + 1);
+            if (d != sum_depth[v]) { sum_depth[v] = d; changed = true; }
+        }
+    }
+    for (Inst &in : g.inst) {
+        in.home_sum = -1;
+        int best = 0;
+        for (int v = 0; v < (int)g.vars.size(); ++v)
+            if (g.vars[v].kind == 2 && (in.deps & (1u << v)) && sum_depth[v] > best) { best = sum_depth[v]; in.home_sum = g.vars[v].sum_inst; }
+    }
+}
+
+// estimated warp-instructions for the current loop order and a lane variable
+double schedule_cost(Gen &g, int root, int lane)
+{
+    place(g);
+    double total = 0;
+    for (int i = 0; i < (int)g.inst.size(); ++i) {
+        const Inst &in = g.inst[i];
+        if (!in.uses) continue;
+        double execs = 1;
+        for (int v = 0; v < g.n_outer; ++v) {
+            double e = (double)g.vars[v].ext;
+            if (v == lane) e = std::ceil(e / 32.0);
+            execs *= e;
+        }
+        int level = (i == root) ? g.kappa : in.zlevel;
+        if (in.home_sum >= 0) level = std::max(level, g.inst[in.home_sum].zlevel);
+        for (int l = 0; l < level; ++l) {
+            int v = g.n_outer + g.zorder[l];
+            double e = (double)g.vars[v].ext;
+            if (v == lane) e = std::ceil(e / 32.0);
+            execs *= e;
+        }
+        for (int v = 0; v < (int)g.vars.size(); ++v)
+            if (g.vars[v].kind == 2 && (in.deps & (1u << v))) execs *= (double)g.vars[v].ext;
+        double w = inst_weight(in);
+        if (in.op == I_LOAD) {
+            int64_t cl = std::llabs((int64_t)g.loads[in.load].coef[lane]);
+            double sectors = cl == 0 ? 1 : cl == 1 ? 4 : (double)std::min<int64_t>(32, 4 * cl);
+            w += sectors;
+        }
+        total += execs * w;
+    }
+    return total;
+}
+
+int32_t to_i32(int64_t v) { if (std::llabs(v) >= (int64_t(1) << 31)) throw Overflow(); return (int32_t)v; }
+
+// worst-case magnitude of a row numerator over the variable boxes must stay inside int32
+void check_row_range(const TadpRow &r, const std::vector<int64_t> &vlo, const std::vector<int64_t> &vhi)
+{
+    int64_t mn = r.c0, mx = r.c0;
+    for (int v = 0; v < TADP_MAX_VARS; ++v) {
+        int64_t c = r.coef[v];
+        if (!c) continue;
+        mn = add_ck(mn, mul_ck(c, c > 0 ? vlo[v] : vhi[v]));
+        mx = add_ck(mx, mul_ck(c, c > 0 ? vhi[v] : vlo[v]));
+    }
+    if (mn <= -(int64_t(1) << 30) || mx >= (int64_t(1) << 30)) throw Overflow();
+}
+
+void finish_stats(Gen &g, Kernel &k, bool backward, int64_t outputs, int64_t terms, bool zero_fill)
+{
+    tad_plan &p = g.p;
+    KernelStats &s = k.stats;
+    s.outputs = outputs; s.terms = terms;
+    s.bytecode_words = k.prog.n_code; s.n_launches = 1 + (zero_fill ? 1 : 0);
+    auto bindings = [&](uint32_t adeps) {
+        double n = 1;
+        for (int d = 0; d < p.n_out + p.n_sum; ++d)
+            if (adeps & (1u << d)) n *= d < p.n_out ? (double)p.out_shape[d] : (double)(p.sum_hi[d - p.n_out] - p.sum_lo[d - p.n_out] + 1);
+        for (int v = 0; v < (int)g.vars.size(); ++v)
+            if (adeps & (1u << (16 + v))) n *= (double)g.vars[v].ext;
+        return n;
+    };
+    std::map<int, double> ptr_bytes;
+    for (int i = 0; i < (int)g.inst.size(); ++i) {
+        const Inst &in = g.inst[i];
+        if (!in.uses) continue;
+        double n = bindings(in.adeps);
+        switch (in.op) {
+        case I_CONST: break;
+        case I_LOAD: {
+            const TadpLoad &L = g.loads[in.load];
+            bool contiguous = false;
+            for (int v = 0; v < TADP_MAX_VARS; ++v) if (std::abs(L.coef[v]) == 1) contiguous = true;
+            double bytes = std::min(n * (contiguous ? 4.0 : 32.0), 4.0 * L.limit);
+            ptr_bytes[L.ptr] = std::max(ptr_bytes[L.ptr], bytes);
+            break;
+        }
+        case I_EXP: case I_LOG: case I_SIN: case I_COS: case I_TANH: case I_SINH: case I_COSH:
+            s.alg_flops += n; s.alg_trans += n; break;
+        case I_POWI: s.alg_flops += n * std::max(1, std::abs(in.ipow) - 1); break;
+        case I_SUM: s.alg_flops += bindings(g.inst[in.a].adeps | (1u << (16 + in.var))); break;   // one add per summand
+        default: s.alg_flops += n; break;
+        }
+    }
+    if (backward) s.alg_flops += (double)terms;         // the accumulation of the terms
+    for (auto &kv : ptr_bytes) s.alg_bytes += kv.second;
+    s.alg_bytes += 4.0 * outputs;
+}
+
+// shared tail: choose temps, emit, fill the program
+void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<TadpRow>> &lower,
+                 const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards)
+{
+    TadpProgram &prog = k.prog;
+    place(g);
+    // temporaries: shared values and values hoisted out of the loop that consumes them
+    std::vector<bool> hoisted(g.inst.size(), false);
+    auto effective_level = [&](int i) { return i == root ? g.kappa : g.inst[i].zlevel; };
+    for (int i = 0; i < (int)g.inst.size(); ++i) {
+        const Inst &in = g.inst[i];
+        if (!in.uses) continue;
+        for (int c : {in.a, in.b}) {
+            if (c < 0 || g.inst[c].op == I_CONST) continue;
+            const Inst &ch = g.inst[c];
+            if (in.op == I_SUM) { if (ch.home_sum != i) hoisted[c] = true; }   // a sum's body is consumed inside its loop
+            else if (ch.home_sum != in.home_sum) hoisted[c] = true;
+            else if (ch.home_sum < 0 && ch.zlevel != effective_level(i)) hoisted[c] = true;
+        }
+    }
+    int n_temps = 0;
+    for (int i = 0; i < (int)g.inst.size(); ++i) {
+        Inst &in = g.inst[i];
+        in.temp = -1;
+        if (!in.uses || in.op == I_CONST || i == root) continue;
+        if (in.uses > 1 || hoisted[i]) {
+            if (n_temps >= TADP_NUM_TEMPS + TADP_MAX_SPILL) throw Unsupported("too many temporaries");
+            in.temp = n_temps++;
+        }
+    }
+    Emitter em(g);
+    em.temps_of_level(0);
+    std::vector<int> zbegin(g.kappa);
+    for (int l = 0; l < g.kappa; ++l) {
+        TadpLoop L{};
+        L.var = g.n_outer + g.zorder[l];
+        L.is_lane = L.var == g.lane_var;
+        L.mask_level = l + 1;
+        em.loops.push_back(L);
+        zbegin[l] = em.emit(P_ZLOOP, (int)em.loops.size() - 1);
+        em.temps_of_level(l + 1);
+    }
+    em.expr(root);
+    em.emit(P_ACC, 0, 0, 0, -1);
+    for (int l = g.kappa - 1; l >= 0; --l) {
+        int loop_id = em.code[zbegin[l]].a;
+        int end = em.emit(P_ZEND, loop_id, 0, zbegin[l] + 1);
+        em.code[zbegin[l]].imm = end + 1;
+    }
+    em.emit(P_END);
+    if (em.depth != 0) throw BadExpr("internal: unbalanced operand stack");
+    // rows
+    std::vector<TadpRow> rows;
+    for (TadpLoop &L : em.loops) {
+        if (g.vars[L.var].kind != 1) continue;
+        int zl = g.zpos[L.var - g.n_outer];
+        L.lower0 = (int16_t)rows.size(); L.n_lower = (int16_t)lower[zl].size();
+        for (const TadpRow &r : lower[zl]) rows.push_back(r);
+        L.upper0 = (int16_t)rows.size(); L.n_upper = (int16_t)upper[zl].size();
+        for (const TadpRow &r : upper[zl]) rows.push_back(r);
+        L.depends_on_lane = 0;
+        for (int r = L.lower0; r < L.upper0 + L.n_upper; ++r)
+            if (rows[r].coef[g.lane_var]) L.depends_on_lane = 1;
+    }
+    prog.guard0 = (int32_t)rows.size(); prog.n_guards = (int32_t)guards.size();
+    for (const TadpRow &r : guards) rows.push_back(r);
+    if ((int)rows.size() > TADP_MAX_ROWS) throw Unsupported("too many bound rows in one kernel");
+    prog.n_code = (int32_t)em.code.size();
+    std::copy(em.code.begin(), em.code.end(), prog.code);
+    prog.n_loads = (int32_t)g.loads.size();
+    std::copy(g.loads.begin(), g.loads.end(), prog.loads);
+    prog.n_loops = (int32_t)em.loops.size();
+    std::copy(em.loops.begin(), em.loops.end(), prog.loops);
+    prog.n_rows = (int32_t)rows.size();
+    std::copy(rows.begin(), rows.end(), prog.rows);
+    prog.n_outer = g.n_outer;
+    prog.lane_var = g.lane_var;
+    const int64_t lane_ext = g.vars[g.lane_var].ext;
+    k.vec = lane_ext >= 128 ? 4 : lane_ext >= 64 ? 2 : 1;
+    char head[256];
+    std::snprintf(head, sizeof head, "; vars=%zu outer=%d kappa=%d lane_var=%d vec=%d temps=%d max_depth=%d loads=%d rows=%d guards=%d\n",
+                  g.vars.size(), g.n_outer, g.kappa, g.lane_var, k.vec, n_temps, em.max_depth, prog.n_loads, prog.n_rows, prog.n_guards);
+    k.listing = head + em.listing;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+// forward: outer variables are the output indices, every sum is a bound loop
+// ---------------------------------------------------------------------------------------
+void generate_forward(tad_plan &p)
+{
+    Kernel &k = p.forward;
+    std::memset(&k.prog, 0, sizeof k.prog);
+    k.out_arg = -1; k.access = -1;
+    Gen g(p, -1);
+    g.n_outer = p.n_out; g.kappa = 0;
+    const int nidx = p.n_out + p.n_sum;
+    g.a_c0.assign(nidx, 0); g.a_coef.assign(nidx, std::vector<int64_t>(TADP_MAX_VARS, 0)); g.a_free_ok.assign(nidx, false);
+    for (int d = 0; d < p.n_out; ++d) {
+        g.new_var(0, p.out_shape[d]);
+        g.a_coef[d][d] = 1; g.a_free_ok[d] = true;
+    }
+    int root = g.val((int)p.nodes.size() - 1, 0);
+    count_uses(g, root);
+    g.lane_var = p.n_out - 1;
+    TadpProgram &prog = k.prog;
+    int64_t stride = 1;
+    for (int d = p.n_out - 1; d >= 0; --d) {
+        prog.outer_lo[d] = 0; prog.outer_ext[d] = to_i32(p.out_shape[d]);
+        prog.out_coef[d] = to_i32(stride);
+        stride *= p.out_shape[d];
+    }
+    prog.out_base = 0; prog.out_limit = to_i32(p.out_elems);
+    prog.accumulate = 0; prog.write_only_live = 0;
+    emit_kernel(g, k, root, {}, {}, {});
+    finish_stats(g, k, false, p.out_elems, 0, false);
+}
+
+// ---------------------------------------------------------------------------------------
+// backward of one index expression (Sec. 5.3: Delta, Omega, I/K/C, Omega', Sigma, accumulate)
+// ---------------------------------------------------------------------------------------
+void generate_backward(tad_plan &p, int q)
+{
+    AccessPlan &ap = p.access[q];
+    p.backward.emplace_back();
+    Kernel &k = p.backward.back();
+    std::memset(&k.prog, 0, sizeof k.prog);
+    k.out_arg = ap.arg; k.access = q;
+    const int kidx = (int)p.backward.size() - 1;
+    const bool first_of_arg = p.arg_kernels[ap.arg].empty();
+    p.arg_kernels[ap.arg].push_back(kidx);
+    const bool zero_fill = p.arg_zero_fill[ap.arg];
+
+    Gen g(p, q);
+    const int R = ap.R, kap = ap.kappa, n = ap.n, rank = ap.rank;
+    // outer variables: beta itself when the map is onto the whole argument lattice, else x'
+    const bool by_beta = !ap.masked;
+    g.n_outer = by_beta ? rank : R;
+    g.kappa = kap;
+    const int nidx = p.n_out + p.n_sum;
+    g.a_c0.assign(nidx, 0); g.a_coef.assign(nidx, std::vector<int64_t>(TADP_MAX_VARS, 0)); g.a_free_ok.assign(nidx, false);
+    // the affine map alpha_hat = c0 + Mu u + K z
+    Mat Mu(n, std::max(1, g.n_outer));
+    std::vector<int64_t> c0(n, 0);
+    std::vector<int64_t> ulo(g.n_outer), uhi(g.n_outer);
+    if (by_beta) {
+        // x' = U (beta - o)  =>  alpha_hat_0 = V_R U beta - V_R U o
+        for (int d = 0; d < n; ++d)
+            for (int c = 0; c < rank; ++c) {
+                int64_t s = 0;
+                for (int j = 0; j < R; ++j) s = add_ck(s, mul_ck(ap.V(d, j), ap.U(j, c)));
+                Mu(d, c) = s;
+                c0[d] = sub_ck(c0[d], mul_ck(s, ap.off[c]));
+            }
+        for (int c = 0; c < rank; ++c) { ulo[c] = 0; uhi[c] = p.arg_shape[ap.arg][c] - 1; }
+    } else {
+        for (int d = 0; d < n; ++d) for (int j = 0; j < R; ++j) Mu(d, j) = ap.V(d, j);
+        for (int j = 0; j < R; ++j) { ulo[j] = ap.xlo[j]; uhi[j] = ap.xhi[j]; }
+    }
+    if (g.n_outer == 0) throw Unsupported("index expression of rank 0 (constant element)");
+    for (int j = 0; j < g.n_outer; ++j) g.new_var(0, uhi[j] - ulo[j] + 1);
+    for (int col = 0; col < kap; ++col) g.new_var(1, kernel_col_extent(ap, col));
+    for (int c = 0; c < n; ++c) {
+        int d = ap.idx_pos[c];
+        g.a_free_ok[d] = true;
+        g.a_c0[d] = c0[c];
+        for (int j = 0; j < g.n_outer; ++j) g.a_coef[d][j] = Mu(c, j);
+        for (int col = 0; col < kap; ++col) g.a_coef[d][g.n_outer + col] = ap.V(c, R + col);
+    }
+    // df[alpha]: the sum indices are ignored when indexing df (Sec. 5.2)
+    std::vector<int64_t> dfA(size_t(p.n_out) * nidx, 0), dfOff(p.n_out, 0);
+    for (int d = 0; d < p.n_out; ++d) dfA[size_t(d) * nidx + d] = 1;
+    int df_inst = g.make_load(p.n_args, dfA, dfOff, p.n_out, p.out_shape, ap.scope, ap.scope);
+    int root = g.differentiate(df_inst);
+    if (root < 0) throw BadExpr("internal: index expression has no path to the root");
+    count_uses(g, root);
+
+    // Lane variable: a variable along which df is contiguous and which fills a warp, if there is
+    // one; otherwise (and for the loop order always) the smallest estimated cost.
+    const TadpLoad dfL = g.loads[g.inst[df_inst].load];
+    int forced_lane = -1;
+    for (int v = 0; v < g.n_outer + kap; ++v)
+        if (std::abs(dfL.coef[v]) == 1 && g.vars[v].ext >= 32 &&
+            (forced_lane < 0 || g.vars[v].ext > g.vars[forced_lane].ext ||
+             (g.vars[v].ext == g.vars[forced_lane].ext && g.vars[v].kind == 1)))
+            forced_lane = v;
+    std::vector<int> perm(kap);
+    for (int l = 0; l < kap; ++l) perm[l] = l;
+    double best = -1; std::vector<int> best_order = perm; int best_lane = -1;
+    do {
+        g.zorder = perm; g.zpos.assign(kap, 0);
+        for (int l = 0; l < kap; ++l) g.zpos[perm[l]] = l;
+        for (int v = 0; v < g.n_outer + kap; ++v) {
+            if (forced_lane >= 0 && v != forced_lane) continue;
+            if (g.vars[v].ext < 2 && g.n_outer + kap > 1) continue;
+            double c = schedule_cost(g, root, v);
+            c /= std::min(1.0, (double)g.vars[v].ext / 32.0);
+            if (std::abs(dfL.coef[v]) == 1) c *= 0.999;
+            if (g.vars[v].kind == 1) c *= 0.9999;
+            if (best < 0 || c < best) { best = c; best_order = perm; best_lane = v; }
+        }
+    } while (std::next_permutation(perm.begin(), perm.end()));
+    if (best_lane < 0) best_lane = 0;
+    g.zorder = best_order; g.zpos.assign(kap, 0);
+    for (int l = 0; l < kap; ++l) g.zpos[best_order[l]] = l;
+    g.lane_var = best_lane;
+    ap.lane_var = best_lane;
+    ap.zorder = best_order;
+    compute_bounds(ap);
+
+    // bound rows and guards over the kernel variables
+    std::vector<int64_t> vlo(TADP_MAX_VARS, 0), vhi(TADP_MAX_VARS, 0);
+    for (int j = 0; j < g.n_outer; ++j) { vlo[j] = ulo[j]; vhi[j] = uhi[j]; }
+    for (int col = 0; col < kap; ++col) {
+        // generous range of a kernel coordinate: z = (V^-1 alpha_hat)_{R+col} over the box, x' part aside
+        int64_t mag = 0;
+        for (int d = 0; d < n; ++d)
+            mag = add_ck(mag, mul_ck(std::llabs(ap.Vinv(R + col, d)), std::max(std::llabs(ap.box_lo[d]), std::llabs(ap.box_hi[d]))));
+        vlo[g.n_outer + col] = -mag; vhi[g.n_outer + col] = mag;
+    }
+    auto convert = [&](const BoundRowH &h, int loop) {
+        TadpRow r{};
+        r.den = to_i32(h.den);
+        int64_t c = h.c0;
+        std::vector<int64_t> cu(g.n_outer, 0);
+        if (by_beta) {
+            for (int col = 0; col < rank; ++col) {
+                int64_t s = 0;
+                for (int j = 0; j < R; ++j) s = add_ck(s, mul_ck(h.cx[j], ap.U(j, col)));
+                cu[col] = s;
+                c = sub_ck(c, mul_ck(s, ap.off[col]));
+            }
+        } else for (int j = 0; j < R; ++j) cu[j] = h.cx[j];
+        r.c0 = to_i32(c);
+        for (int j = 0; j < g.n_outer; ++j) r.coef[j] = to_i32(cu[j]);
+        for (int m = 0; m < loop; ++m) r.coef[g.n_outer + ap.zorder[m]] = to_i32(h.cz[m]);
+        check_row_range(r, vlo, vhi);
+        return r;
+    };
+    std::vector<std::vector<TadpRow>> lower(kap), upper(kap);
+    for (int l = 0; l < kap; ++l) {
+        for (const BoundRowH &h : ap.lower[l]) lower[l].push_back(convert(h, l));
+        for (const BoundRowH &h : ap.upper[l]) upper[l].push_back(convert(h, l));
+    }
+    std::vector<TadpRow> guards;
+    for (const BoundRowH &h : ap.guards) {
+        TadpRow r = convert(h, 0);
+        // drop guards that hold on the whole outer box
+        int64_t mx = r.c0;
+        for (int j = 0; j < g.n_outer; ++j) mx += (int64_t)r.coef[j] * (r.coef[j] > 0 ? uhi[j] : ulo[j]);
+        if (mx > 0) guards.push_back(r);
+    }
+
+    TadpProgram &prog = k.prog;
+    for (int j = 0; j < g.n_outer; ++j) { prog.outer_lo[j] = to_i32(ulo[j]); prog.outer_ext[j] = to_i32(uhi[j] - ulo[j] + 1); }
+    // output offset
+    std::vector<int64_t> ostride(rank, 1);
+    for (int r = rank - 2; r >= 0; --r) ostride[r] = ostride[r + 1] * p.arg_shape[ap.arg][r + 1];
+    if (by_beta) {
+        prog.out_base = 0;
+        for (int r = 0; r < rank; ++r) prog.out_coef[r] = to_i32(ostride[r]);
+    } else {
+        // beta = o + U^-1[:, :R] diag(alpha) x'
+        Mat Uinv = unimodular_inverse(ap.U);
+        int64_t base = 0;
+        for (int r = 0; r < rank; ++r) base = add_ck(base, mul_ck(ostride[r], ap.off[r]));
+        prog.out_base = to_i32(base);
+        for (int j = 0; j < R; ++j) {
+            int64_t s = 0;
+            for (int r = 0; r < rank; ++r) s = add_ck(s, mul_ck(ostride[r], mul_ck(Uinv(r, j), ap.inv[j])));
+            prog.out_coef[j] = to_i32(s);
+        }
+    }
+    prog.out_limit = to_i32(p.arg_elems[ap.arg]);
+    prog.accumulate = (zero_fill || !first_of_arg) ? 1 : 0;
+    prog.write_only_live = ap.masked ? 1 : 0;
+    emit_kernel(g, k, root, lower, upper, guards);
+    int64_t terms = 1;
+    for (int d = 0; d < n; ++d) terms = mul_ck(terms, ap.box_hi[d] - ap.box_lo[d] + 1);
+    finish_stats(g, k, true, p.arg_elems[ap.arg], terms, zero_fill && first_of_arg);
+}
+
+}  // namespace tad

@@ -1,0 +1,289 @@
+// Device side of the C ABI: the interpreter kernel, the zero-fill kernel and the launchers
+// behind tad_forward / tad_backward / tad_step_host.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <string>
+
+#include "plan.h"
+#include "vm.cuh"
+
+namespace tad {
+void set_error(const std::string &m);
+}
+
+namespace {
+
+using namespace tadvm;
+
+// One warp per work item, grid-stride over the items.  A work item fixes every outer variable
+// except the lane variable, which the warp covers 32 * T elements at a time.
+template <int T, bool DEBUG>
+__global__ void __launch_bounds__(WARPS_PER_BLOCK * 32)
+tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ TadpPointers ptrs, unsigned n_items)
+{
+    const unsigned lane = threadIdx.x & 31u;
+    const unsigned warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const unsigned n_warps = (gridDim.x * blockDim.x) >> 5;
+    const int lane_var = P.lane_var;
+    const bool lane_outer = lane_var < P.n_outer;
+    Vm<T> m;
+    for (unsigned item = warp; item < n_items; item += n_warps) {
+        // decode the outer variables (last one fastest)
+        unsigned rem = item;
+#pragma unroll
+        for (int k = 0; k < TADP_MAX_VARS; ++k) m.var[k] = 0;
+        unsigned mask0 = (1u << T) - 1u;
+#pragma unroll
+        for (int v = TADP_MAX_VARS - 1; v >= 0; --v) {
+            if (v < P.n_outer) {
+                const unsigned ext = (unsigned)P.outer_ext[v];
+                if (v == lane_var) {
+                    const unsigned chunks = (ext + 32u * T - 1u) / (32u * T);
+                    const unsigned c = rem % chunks; rem /= chunks;
+                    const unsigned first = c * 32u * T + lane;
+                    m.var[v] = P.outer_lo[v] + (int)first;
+                    mask0 = 0;
+#pragma unroll
+                    for (int t = 0; t < T; ++t) if (first + 32u * t < ext) mask0 |= 1u << t;
+                } else {
+                    const unsigned c = rem % ext; rem /= ext;
+                    m.var[v] = P.outer_lo[v] + (int)c;
+                }
+            }
+        }
+        const unsigned in_range = mask0;
+        // guards: rows over the outer variables that must be <= 0 for Gamma to be non-empty
+        for (int r = 0; r < P.n_guards; ++r) {
+            const TadpRow &R = P.rows[P.guard0 + r];
+            const int nmr = row_num(R, m.var);
+            const int step = lane_outer ? R.coef[lane_var] * 32 : 0;
+#pragma unroll
+            for (int t = 0; t < T; ++t) if (nmr + t * step > 0) mask0 &= ~(1u << t);
+        }
+        unsigned live = 0;
+        run_item<T, DEBUG>(P, ptrs, m, mask0, live);
+        // output
+        if (lane_outer) {
+            unsigned off = (unsigned)P.out_base;
+#pragma unroll
+            for (int k = 0; k < TADP_MAX_VARS; ++k) off += (unsigned)P.out_coef[k] * (unsigned)m.var[k];
+            const unsigned step = (unsigned)P.out_coef[lane_var] * 32u;
+#pragma unroll
+            for (int t = 0; t < T; ++t) {
+                if (!((in_range >> t) & 1u)) continue;
+                if (P.write_only_live && !((live >> t) & 1u)) continue;
+                const unsigned idx = off + (unsigned)t * step;
+                if (DEBUG && idx >= (unsigned)P.out_limit) { if (ptrs.debug) atomicCAS(ptrs.debug, 0, 0x20000); continue; }
+                ptrs.out[idx] = P.accumulate ? ptrs.out[idx] + m.acc[t] : m.acc[t];
+            }
+        } else {
+            // the lane variable is a kernel coordinate: one output per warp, fixed-order tree reduction
+            unsigned off = (unsigned)P.out_base;
+#pragma unroll
+            for (int k = 0; k < TADP_MAX_VARS; ++k) if (k < P.n_outer) off += (unsigned)P.out_coef[k] * (unsigned)m.var[k];
+            float total = 0.f;
+#pragma unroll
+            for (int t = 0; t < T; ++t) total += m.acc[t];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+            const unsigned any_live = __ballot_sync(0xffffffffu, live != 0);
+            if (lane == 0 && !(P.write_only_live && !any_live)) {
+                if (DEBUG && off >= (unsigned)P.out_limit) { if (ptrs.debug) atomicCAS(ptrs.debug, 0, 0x20000); }
+                else ptrs.out[off] = P.accumulate ? ptrs.out[off] + total : total;
+            }
+        }
+    }
+}
+
+__global__ void tad_fill_zero(float *out, unsigned n)
+{
+    const unsigned stride = gridDim.x * blockDim.x;
+    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) out[i] = 0.f;
+}
+
+int sm_count()
+{
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    return n;
+}
+
+unsigned long long item_count(const TadpProgram &P, int T)
+{
+    unsigned long long n = 1;
+    for (int v = 0; v < P.n_outer; ++v) {
+        unsigned long long e = (unsigned long long)P.outer_ext[v];
+        if (v == P.lane_var) e = (e + 32ull * T - 1) / (32ull * T);
+        n *= e;
+    }
+    return n;
+}
+
+template <int T>
+void launch_t(const tad::Kernel &k, const TadpPointers &ptrs, bool debug, unsigned items, unsigned blocks, cudaStream_t stream)
+{
+    if (debug) tad_vm_kernel<T, true><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items);
+    else tad_vm_kernel<T, false><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items);
+}
+
+tad_status launch(const tad::Kernel &k, const TadpPointers &ptrs, bool debug, cudaStream_t stream)
+{
+    const unsigned long long items64 = item_count(k.prog, k.vec);
+    if (items64 == 0) return TAD_OK;
+    if (items64 >= (1ull << 32)) { tad::set_error("too many work items"); return TAD_ERR_UNSUPPORTED; }
+    const unsigned items = (unsigned)items64;
+    const unsigned blocks_needed = (items + WARPS_PER_BLOCK - 1) / WARPS_PER_BLOCK;
+    const unsigned max_blocks = (unsigned)sm_count() * 16u;
+    const unsigned blocks = std::min(blocks_needed, max_blocks);
+    switch (k.vec) {
+    case 1: launch_t<1>(k, ptrs, debug, items, blocks, stream); break;
+    case 2: launch_t<2>(k, ptrs, debug, items, blocks, stream); break;
+    default: launch_t<4>(k, ptrs, debug, items, blocks, stream); break;
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { tad::set_error(std::string("kernel launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
+    return TAD_OK;
+}
+
+tad_status zero_fill(float *out, int64_t n, cudaStream_t stream)
+{
+    const unsigned blocks = (unsigned)std::min<int64_t>((n + 255) / 256, (int64_t)sm_count() * 16);
+    tad_fill_zero<<<blocks, 256, 0, stream>>>(out, (unsigned)n);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { tad::set_error(std::string("zero fill launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
+    return TAD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t tad_workspace_bytes(const tad_plan *plan)
+{
+    if (!plan) return 0;
+    return plan->opt.debug_bounds ? 256 : 0;
+}
+
+tad_status tad_forward(const tad_plan *plan, const float *const *args, float *f, void *cuda_stream)
+{
+    if (!plan || !f || (plan->n_args && !args)) { tad::set_error("NULL argument"); return TAD_ERR_INVALID_ARG; }
+    TadpPointers ptrs{};
+    for (int a = 0; a < plan->n_args; ++a) {
+        if (!args[a]) { tad::set_error("NULL argument tensor"); return TAD_ERR_INVALID_ARG; }
+        ptrs.in[a] = args[a];
+    }
+    ptrs.out = f;
+    ptrs.debug = nullptr;
+    return launch(plan->forward, ptrs, false, (cudaStream_t)cuda_stream);
+}
+
+tad_status tad_backward(const tad_plan *plan, const float *const *args, const float *df,
+                        float *const *dargs, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!plan || !df || !dargs || (plan->n_args && !args)) { tad::set_error("NULL argument"); return TAD_ERR_INVALID_ARG; }
+    const bool debug = plan->opt.debug_bounds != 0;
+    const size_t need = tad_workspace_bytes(plan);
+    if (need && (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))) {
+        tad::set_error("workspace missing, smaller than tad_workspace_bytes() or not 256-byte aligned");
+        return TAD_ERR_WORKSPACE;
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    TadpPointers ptrs{};
+    for (int a = 0; a < plan->n_args; ++a) {
+        if (!args[a]) { tad::set_error("NULL argument tensor"); return TAD_ERR_INVALID_ARG; }
+        ptrs.in[a] = args[a];
+    }
+    ptrs.in[plan->n_args] = df;
+    ptrs.debug = debug ? static_cast<int32_t *>(workspace) : nullptr;
+    for (int a = 0; a < plan->n_args; ++a) {
+        if (!dargs[a]) continue;
+        if (plan->arg_kernels[a].empty() || plan->arg_zero_fill[a]) {
+            tad_status st = zero_fill(dargs[a], plan->arg_elems[a], stream);
+            if (st != TAD_OK) return st;
+        }
+        for (int ki : plan->arg_kernels[a]) {
+            ptrs.out = dargs[a];
+            tad_status st = launch(plan->backward[ki], ptrs, debug, stream);
+            if (st != TAD_OK) return st;
+        }
+    }
+    return TAD_OK;
+}
+
+size_t tad_staging_bytes(const tad_plan *plan)
+{
+    if (!plan) return 0;
+    auto pad = [](size_t b) { return (b + 255) & ~size_t(255); };
+    size_t total = pad(tad_workspace_bytes(plan));
+    for (int a = 0; a < plan->n_args; ++a) total += 2 * pad(size_t(plan->arg_elems[a]) * 4);   // x^p and dx^p
+    total += 2 * pad(size_t(plan->out_elems) * 4);                                            // f and df
+    return total;
+}
+
+tad_status tad_step_host(const tad_plan *plan, const float *const *h_args, const float *h_df,
+                         float *h_f, float *const *h_dargs, void *staging, size_t staging_bytes, void *cuda_stream)
+{
+    if (!plan || !h_args || !h_df || !h_dargs || !staging) { tad::set_error("NULL argument"); return TAD_ERR_INVALID_ARG; }
+    if (staging_bytes < tad_staging_bytes(plan) || (reinterpret_cast<uintptr_t>(staging) & 255u)) {
+        tad::set_error("staging buffer too small or not 256-byte aligned");
+        return TAD_ERR_WORKSPACE;
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    auto pad = [](size_t b) { return (b + 255) & ~size_t(255); };
+    char *cur = static_cast<char *>(staging);
+    void *ws = cur; cur += pad(tad_workspace_bytes(plan));
+    const float *d_args[TADP_MAX_PTRS]; float *d_dargs[TADP_MAX_PTRS];
+    auto check = [](cudaError_t e, const char *what) {
+        if (e != cudaSuccess) { tad::set_error(std::string(what) + ": " + cudaGetErrorString(e)); return false; }
+        return true;
+    };
+    for (int a = 0; a < plan->n_args; ++a) {
+        const size_t bytes = size_t(plan->arg_elems[a]) * 4;
+        float *dx = reinterpret_cast<float *>(cur); cur += pad(bytes);
+        float *dg = reinterpret_cast<float *>(cur); cur += pad(bytes);
+        if (!h_args[a]) { tad::set_error("NULL host argument"); return TAD_ERR_INVALID_ARG; }
+        if (!check(cudaMemcpyAsync(dx, h_args[a], bytes, cudaMemcpyHostToDevice, stream), "copy of an argument")) return TAD_ERR_CUDA;
+        d_args[a] = dx; d_dargs[a] = h_dargs[a] ? dg : nullptr;
+    }
+    const size_t fbytes = size_t(plan->out_elems) * 4;
+    float *d_f = reinterpret_cast<float *>(cur); cur += pad(fbytes);
+    float *d_df = reinterpret_cast<float *>(cur); cur += pad(fbytes);
+    if (!check(cudaMemcpyAsync(d_df, h_df, fbytes, cudaMemcpyHostToDevice, stream), "copy of df")) return TAD_ERR_CUDA;
+    tad_status st = TAD_OK;
+    if (h_f) {
+        st = tad_forward(plan, d_args, d_f, stream);
+        if (st != TAD_OK) return st;
+        if (!check(cudaMemcpyAsync(h_f, d_f, fbytes, cudaMemcpyDeviceToHost, stream), "copy of f")) return TAD_ERR_CUDA;
+    }
+    if (plan->opt.debug_bounds && !check(cudaMemsetAsync(ws, 0, 256, stream), "clearing the debug word")) return TAD_ERR_CUDA;
+    st = tad_backward(plan, d_args, d_df, d_dargs, ws, tad_workspace_bytes(plan), stream);
+    if (st != TAD_OK) return st;
+    for (int a = 0; a < plan->n_args; ++a)
+        if (h_dargs[a] && !check(cudaMemcpyAsync(h_dargs[a], d_dargs[a], size_t(plan->arg_elems[a]) * 4, cudaMemcpyDeviceToHost, stream), "copy of a gradient")) return TAD_ERR_CUDA;
+    if (!check(cudaStreamSynchronize(stream), "stream synchronise")) return TAD_ERR_CUDA;
+    return TAD_OK;
+}
+
+tad_status tad_debug_status(const tad_plan *plan, void *workspace, void *cuda_stream)
+{
+    if (!plan) { tad::set_error("NULL plan"); return TAD_ERR_INVALID_ARG; }
+    if (!plan->opt.debug_bounds) return TAD_OK;
+    if (!workspace) { tad::set_error("NULL workspace"); return TAD_ERR_INVALID_ARG; }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    int32_t word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, workspace, sizeof word, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e == cudaSuccess && word != 0) e = cudaMemsetAsync(workspace, 0, sizeof word, stream);
+    if (e != cudaSuccess) { tad::set_error(std::string("reading the debug word: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
+    if (word != 0) {
+        char msg[96];
+        snprintf(msg, sizeof msg, "a kernel skipped an out-of-range access (code 0x%x)", word);
+        tad::set_error(msg);
+        return TAD_ERR_OUT_OF_RANGE;
+    }
+    return TAD_OK;
+}
+
+}  // extern "C"
