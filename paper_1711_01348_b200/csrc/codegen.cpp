@@ -709,7 +709,6 @@ void generate_backward(tad_plan &p, int q)
         for (int d = 0; d < n; ++d) for (int j = 0; j < R; ++j) Mu(d, j) = ap.V(d, j);
         for (int j = 0; j < R; ++j) { ulo[j] = ap.xlo[j]; uhi[j] = ap.xhi[j]; }
     }
-    if (g.n_outer == 0) throw Unsupported("index expression of rank 0 (constant element)");
     for (int j = 0; j < g.n_outer; ++j) g.new_var(0, uhi[j] - ulo[j] + 1);
     for (int col = 0; col < kap; ++col) g.new_var(1, kernel_col_extent(ap, col));
     for (int c = 0; c < n; ++c) {
