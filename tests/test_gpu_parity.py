@@ -1,0 +1,69 @@
+"""Parity of the CUDA path with the float64 oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle.oracle import Oracle, max_threads
+from workloads import configs as W
+
+pytestmark = pytest.mark.gpu
+
+from tests.gpu_util import GpuRun, assert_close, check_against_oracle  # noqa: E402
+
+SMALL = {
+    "sec6": (lambda: W.ex_section6(), ("uniform", -0.5, 0.5)),
+    "square_broadcast": (lambda: W.ex_square_broadcast(70, 133), ("uniform", -1, 1)),
+    "diag_square": (lambda: W.ex_diag_square(77), ("uniform", -1, 1)),
+    "exp_shift": (lambda: W.ex_exp_shift(150, 67), ("uniform", -1, 1)),
+    "sin": (lambda: W.ex_sin(1000), ("normal", 0, 1)),
+    "xy": (lambda: W.ex_xy(131), ("normal", 0, 1)),
+    "diag_cube": (lambda: W.ex_diag_cube(45), ("normal", 0, 1)),
+    "matmul": (lambda: W.ex_matmul(37, 150, 41), ("normal", 0, 1)),
+    "exp_flat": (lambda: W.ex_exp_flat(33, 7), ("uniform", -1, 1)),
+    "strided": (lambda: W.ex_strided(301, 2), ("normal", 0, 1)),
+    "strided3": (lambda: W.ex_strided(100, 3), ("normal", 0, 1)),
+    "strided2": (lambda: W.ex_strided2(40, 33), ("normal", 0, 1)),
+    "lattice2d": (lambda: W.ex_lattice2d(35, 44), ("normal", 0, 1)),
+    "all_ops": (lambda: W.ex_all_ops(300), ("uniform", -0.9, 0.9)),
+    "tiny": (lambda: W.intro(1, 1, 1), ("uniform", -0.5, 0.5)),
+    "one_row": (lambda: W.intro(1, 200, 3), ("uniform", -0.5, 0.5)),
+    "one_col": (lambda: W.intro(200, 1, 3), ("uniform", -0.5, 0.5)),
+}
+
+
+@pytest.mark.parametrize("name", sorted(SMALL))
+def test_small_expressions(name):
+    make, dist = SMALL[name]
+    e = make()
+    args, df = W.make_inputs(e, dist, seed=0)
+    check_against_oracle(e, args, df, debug_bounds=True)
+    check_against_oracle(e, args, df)
+
+
+@pytest.mark.parametrize("key", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+def test_reduced_workloads(key):
+    """Same structure as the full workloads, several tiles and ragged tails, full oracle run."""
+    e, args, df = W.workload(key, full=False)
+    check_against_oracle(e, args, df, nthreads=max_threads(), debug_bounds=True)
+    check_against_oracle(e, args, df, nthreads=max_threads())
+
+
+def test_gradient_subset_and_repeat_calls():
+    e, args, df = W.workload("cfg2", full=False)
+    run = GpuRun(e, args, df)
+    first = run.backward()
+    only_b = run.backward(wanted=[False, True, False, False])
+    np.testing.assert_array_equal(first[1], only_b[1])
+    second = run.backward()
+    for a, b in zip(first, second):
+        np.testing.assert_array_equal(a, b)       # fixed summation order: bitwise repeatable
+
+
+def test_null_pointer_is_rejected():
+    from paper_1711_01348_b200 import TadError
+    e, args, df = W.workload("cfg1", full=False)
+    run = GpuRun(e, args, df)
+    with pytest.raises(TadError):
+        run.plan.forward([a.data_ptr() for a in run.args], 0)
+    with pytest.raises(TadError):
+        run.plan.backward([0] * 4, run.df.data_ptr(), [d.data_ptr() for d in run.dargs])
