@@ -1,0 +1,324 @@
+#!/usr/bin/env python
+"""Benchmark: forward + all gradients of one synthetic workload through the C ABI.
+
+One step = tad_forward + tad_backward (every gradient) on device-resident inputs.  Prints ONE
+JSON line (rank 0).  With --gpus N > 1 (under torchrun) every rank runs an independent replica
+of the same workload on its own GPU; there is no data-path collective.
+`--impl reference` times the float64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fwd+bwd tensor elements/s"
+UNIT = "elements/s"
+
+# rows of the output the oracle sample covers, per workload (about 10-30 s of CPU work on 16 cores)
+ORACLE_SAMPLE_ROWS = {"cfg1": 64, "cfg2": 256, "cfg3": 4096, "cfg4": 96, "cfg5": 1}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "sm_max_mhz": float(d.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.samples = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 6:
+                self.samples.append(parts)
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        if self.thread is not None:
+            self.thread.join(timeout=5)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for p in self.samples:
+            try:
+                sm.append(float(p[0])); mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, p[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def elements_per_step(expr) -> int:
+    n = 1
+    for s in expr.out_shape:
+        n *= s
+    for shape in expr.arg_shapes:
+        m = 1
+        for s in shape:
+            m *= s
+        n += m
+    return n
+
+
+def oracle_sample(key, expr, args, df, nthreads):
+    """Runs the oracle, as it stands, on the first rows of the output; returns (seconds, elements)."""
+    from oracle.oracle import Oracle
+    rows = min(ORACLE_SAMPLE_ROWS[key], expr.out_shape[0])
+    lo = [0] * len(expr.out_shape)
+    hi = [rows] + list(expr.out_shape[1:])
+    orc = Oracle(expr)
+    t0 = time.perf_counter()
+    orc.forward(args, lo, hi, nthreads=nthreads)
+    orc.backward(args, df, lo, hi, nthreads=nthreads)
+    dt = time.perf_counter() - t0
+    frac = rows / expr.out_shape[0]
+    return dt, elements_per_step(expr) * frac, f"output rows [0, {rows}) of {expr.out_shape[0]} ({frac:.4%} of one step), forward + all gradients"
+
+
+def run_reference(opts):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle.oracle import build as build_oracle, max_threads
+    from workloads import configs as W
+    build_oracle()
+    expr, args, df = W.workload(opts.config, full=True)
+    cores = max_threads()
+    times = []
+    sample = ""
+    elems = 0.0
+    for i in range(opts.warmup + opts.steps):
+        dt, elems, sample = oracle_sample(opts.config, expr, args, df, cores)
+        if i >= opts.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = elems * len(times) / total
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": opts.gpus,
+            "steps": opts.steps, "warmup": opts.warmup, "ms_per_step": 1e3 * total / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": W.FULL[opts.config]().name, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(opts):
+    import torch
+    from paper_1711_01348_b200 import Plan
+    from workloads import configs as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    distributed = world > 1
+    if distributed:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl")
+    dev = torch.device(f"cuda:{local_rank}")
+    torch.cuda.set_device(dev)
+
+    expr, args, df = W.workload(opts.config, full=True)
+    plan = Plan(expr)
+    d_args = [a.to(dev) for a in args]
+    d_df = df.to(dev)
+    f = torch.empty(expr.out_shape, dtype=torch.float32, device=dev)
+    dargs = [torch.empty(s, dtype=torch.float32, device=dev) for s in expr.arg_shapes]
+    ws = torch.zeros(max(256, plan.workspace_bytes()), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream().cuda_stream
+    arg_ptrs = [a.data_ptr() for a in d_args]
+    darg_ptrs = [d.data_ptr() for d in dargs]
+    n_args = len(d_args)
+    parts = ["forward"] + [f"d{name}" for name in expr.arg_names]
+
+    def step(events=None):
+        if events is not None:
+            events[0].record()
+        plan.forward(arg_ptrs, f.data_ptr(), stream)
+        for p in range(n_args):
+            if events is not None:
+                events[p + 1].record()
+            only = [darg_ptrs[i] if i == p else 0 for i in range(n_args)]
+            plan.backward(arg_ptrs, d_df.data_ptr(), only, ws.data_ptr(), ws.numel(), stream)
+        if events is not None:
+            events[n_args + 1].record()
+
+    def barrier():
+        if distributed:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(opts.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    all_events = [[torch.cuda.Event(enable_timing=True) for _ in range(n_args + 2)] for _ in range(opts.steps)]
+    t_begin = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_begin.record()
+    for k in range(opts.steps):
+        step(all_events[k])
+    t_end.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t_begin.elapsed_time(t_end)
+    if distributed:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    part_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in all_events) / opts.steps for i in range(n_args + 1)]
+
+    # end to end: pinned host buffers in, results back, through tad_step_host
+    e2e = None
+    try:
+        h_args = [a.pin_memory() for a in args]
+        h_df = df.pin_memory()
+        h_f = torch.empty(expr.out_shape, dtype=torch.float32).pin_memory()
+        h_dargs = [torch.empty(s, dtype=torch.float32).pin_memory() for s in expr.arg_shapes]
+        staging = torch.empty(plan.staging_bytes(), dtype=torch.uint8, device=dev)
+        e2e_steps = max(1, min(opts.steps, 3))
+
+        def host_step():
+            plan.step_host([a.data_ptr() for a in h_args], h_df.data_ptr(), h_f.data_ptr(),
+                           [d.data_ptr() for d in h_dargs], staging.data_ptr(), staging.numel(), stream)
+        host_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            host_step()
+        torch.cuda.synchronize()
+        e2e_s = (time.perf_counter() - t0) / e2e_steps
+        if distributed:
+            t = torch.tensor([e2e_s], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        h2d = sum(a.numel() * 4 for a in args) + df.numel() * 4
+        d2h = h_f.numel() * 4 + sum(d.numel() * 4 for d in h_dargs)
+        e2e = {"value": world * elements_per_step(expr) / e2e_s, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * e2e_s}
+        del staging
+    except RuntimeError as exc:                       # e.g. not enough pinned memory
+        e2e = {"value": None, "unit": UNIT, "error": str(exc)[:200]}
+
+    if rank == 0:
+        peaks = load_peaks()
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        fp32_peak_tflops = 2 * 128 * sms * peaks["sm_max_mhz"] * 1e6 / 1e12
+        stats = [plan.kernel_stats(-1)]
+        first_access = {}
+        for q, a in enumerate(expr.accesses):
+            first_access.setdefault(a.arg, []).append(q)
+        per_part = []
+        launches = 0
+        for i, name in enumerate(parts):
+            if i == 0:
+                qs = [-1]
+            else:
+                qs = first_access.get(i - 1, [])
+            flops = sum(plan.kernel_stats(q).alg_flops for q in qs)
+            byts = sum(plan.kernel_stats(q).alg_bytes for q in qs)
+            nl = sum(plan.kernel_stats(q).n_launches for q in qs)
+            launches += nl
+            ms = part_ms[i]
+            t_alu = flops / (fp32_peak_tflops * 1e12)
+            t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
+            per_part.append({"part": name, "ms": ms, "alg_gflop": flops / 1e9, "alg_gb": byts / 1e9,
+                             "bound": "alu" if t_alu >= t_hbm else "hbm",
+                             "frac": max(t_alu, t_hbm) / (ms * 1e-3) if ms > 0 else None})
+        dom = max(range(len(parts)), key=lambda i: part_ms[i])
+        d = per_part[dom]
+        if d["bound"] == "alu":
+            achieved = d["alg_gflop"] / 1e3 / (d["ms"] * 1e-3)
+            roof = {"bound": "alu", "achieved": achieved, "peak": fp32_peak_tflops, "unit": "TFLOP/s",
+                    "frac": achieved / fp32_peak_tflops, "traffic": None,
+                    "peak_source": f"2 x 128 lanes x {sms} SMs x {peaks['sm_max_mhz']:.0f} MHz ({peaks['source']} clock)"}
+        else:
+            achieved = d["alg_gb"] / (d["ms"] * 1e-3)
+            roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
+        roof["kernel"] = d["part"]
+        cpu = None
+        if not distributed and not opts.no_cpu_baseline:
+            from oracle.oracle import build as build_oracle, max_threads
+            build_oracle()
+            cores = max_threads()
+            dt, elems, sample = oracle_sample(opts.config, expr, args, df, cores)
+            cpu = {"value": elems / dt, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                   "seconds": dt}
+        ms_per_step = total_ms / opts.steps
+        line = {"metric": METRIC, "value": world * elements_per_step(expr) / (ms_per_step * 1e-3), "unit": UNIT,
+                "n_gpus": world, "steps": opts.steps, "warmup": opts.warmup, "ms_per_step": ms_per_step,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+                "data": "synthetic",
+                "config": {"workload": expr.name, "out_shape": expr.out_shape, "arg_shapes": expr.arg_shapes,
+                           "l2": "inputs larger than L2 (df and c are 268 MB each)" if opts.config == "cfg2" else "see DESIGN.md",
+                           "parallelism": "replicas" if world > 1 else "single"},
+                "roofline": roof, "parts": per_part, "cpu_baseline": cpu, "e2e": e2e,
+                "gpu_launches": launches * opts.steps, "clocks": clocks}
+        print(json.dumps(line), flush=True)
+    if distributed:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    opts = ap.parse_args()
+    if opts.impl == "reference":
+        run_reference(opts)
+    else:
+        run_ours(opts)
+
+
+if __name__ == "__main__":
+    main()
