@@ -161,6 +161,12 @@ def run_ours(opts):
     torch.cuda.set_device(dev)
 
     expr, args, df = W.workload(opts.config, full=True)
+    if opts.rows:
+        # profiler captures only: the same workload with fewer rows of the first output index
+        if opts.config != "cfg2":
+            raise SystemExit("--rows is implemented for cfg2 only")
+        expr = W.intro(opts.rows, 8192, 32, name=f"cfg2_intro_scaled_rows{opts.rows}")
+        args, df = W.make_inputs(expr, W.DIST["cfg2"], seed=0)
     plan = Plan(expr)
     d_args = [a.to(dev) for a in args]
     d_df = df.to(dev)
@@ -215,6 +221,8 @@ def run_ours(opts):
     # end to end: pinned host buffers in, results back, through tad_step_host
     e2e = None
     try:
+        if opts.no_e2e:
+            raise RuntimeError("skipped (--no-e2e)")
         h_args = [a.pin_memory() for a in args]
         h_df = df.pin_memory()
         h_f = torch.empty(expr.out_shape, dtype=torch.float32).pin_memory()
@@ -282,7 +290,7 @@ def run_ours(opts):
                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
         roof["kernel"] = d["part"]
         cpu = None
-        if not distributed and not opts.no_cpu_baseline:
+        if not distributed and not opts.no_cpu_baseline and not opts.rows:
             from oracle.oracle import build as build_oracle, max_threads
             build_oracle()
             cores = max_threads()
@@ -313,6 +321,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--rows", type=int, default=0,
+                    help="profiler captures only: shrink the first output extent of cfg2 (not a bench number)")
     opts = ap.parse_args()
     if opts.impl == "reference":
         run_reference(opts)
