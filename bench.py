@@ -177,19 +177,26 @@ def run_ours(opts):
     arg_ptrs = [a.data_ptr() for a in d_args]
     darg_ptrs = [d.data_ptr() for d in dargs]
     n_args = len(d_args)
-    parts = ["forward"] + [f"d{name}" for name in expr.arg_names]
+    n_stages = plan.num_stages()
+    parts = ["forward"] + (["stage"] if n_stages else []) + [f"d{name}" for name in expr.arg_names]
+    n_parts = len(parts)
 
     def step(events=None):
+        """forward, then exactly what tad_backward does: staging kernels, then every gradient."""
+        e = 0
         if events is not None:
-            events[0].record()
+            events[e].record(); e += 1
         plan.forward(arg_ptrs, f.data_ptr(), stream)
+        if n_stages:
+            if events is not None:
+                events[e].record(); e += 1
+            plan.backward_stage(arg_ptrs, d_df.data_ptr(), ws.data_ptr(), ws.numel(), stream)
         for p in range(n_args):
             if events is not None:
-                events[p + 1].record()
-            only = [darg_ptrs[i] if i == p else 0 for i in range(n_args)]
-            plan.backward(arg_ptrs, d_df.data_ptr(), only, ws.data_ptr(), ws.numel(), stream)
+                events[e].record(); e += 1
+            plan.backward_arg(arg_ptrs, d_df.data_ptr(), p, darg_ptrs[p], ws.data_ptr(), ws.numel(), stream)
         if events is not None:
-            events[n_args + 1].record()
+            events[e].record()
 
     def barrier():
         if distributed:
@@ -202,7 +209,7 @@ def run_ours(opts):
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    all_events = [[torch.cuda.Event(enable_timing=True) for _ in range(n_args + 2)] for _ in range(opts.steps)]
+    all_events = [[torch.cuda.Event(enable_timing=True) for _ in range(n_parts + 1)] for _ in range(opts.steps)]
     t_begin = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
     barrier()
     t_begin.record()
@@ -216,7 +223,7 @@ def run_ours(opts):
         t = torch.tensor([total_ms], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         total_ms = float(t.item())
-    part_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in all_events) / opts.steps for i in range(n_args + 1)]
+    part_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in all_events) / opts.steps for i in range(n_parts)]
 
     # end to end: pinned host buffers in, results back, through tad_step_host
     e2e = None
@@ -263,10 +270,12 @@ def run_ours(opts):
         per_part = []
         launches = 0
         for i, name in enumerate(parts):
-            if i == 0:
+            if name == "forward":
                 qs = [-1]
+            elif name == "stage":
+                qs = [-2 - st for st in range(n_stages)]
             else:
-                qs = first_access.get(i - 1, [])
+                qs = first_access.get(expr.arg_names.index(name[1:]), [])
             flops = sum(plan.kernel_stats(q).alg_flops for q in qs)
             byts = sum(plan.kernel_stats(q).alg_bytes for q in qs)
             nl = sum(plan.kernel_stats(q).n_launches for q in qs)

@@ -163,6 +163,23 @@ tad_status tad_backward(const tad_plan *plan, const float *const *args, const fl
                         void *cuda_stream);
 
 /*
+ * The two halves of tad_backward, for callers that want gradients one at a time.
+ * tad_backward_stage evaluates, once per output element, the adjoints of the top-level sums
+ * that several gradients share (the factor df * d fbar / d s-bar of Sec. 5.2) into the
+ * workspace; tad_backward_arg then evaluates the gradient of ONE argument and expects the
+ * staged values of the same args / df to be in the workspace.  tad_backward is exactly
+ * tad_backward_stage (when a requested gradient reads a staged value) followed by
+ * tad_backward_arg for every requested argument.  The paper evaluates the derivative without
+ * temporary memory (Sec. 7); staging trades |f| floats per staged sum for not repeating the
+ * inner sum in every term.
+ */
+tad_status tad_backward_stage(const tad_plan *plan, const float *const *args, const float *df,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream);
+tad_status tad_backward_arg(const tad_plan *plan, const float *const *args, const float *df,
+                            int32_t arg, float *darg, void *workspace, size_t workspace_bytes,
+                            void *cuda_stream);
+
+/*
  * tad_step_host: one forward and one backward pass with HOST buffers (same meaning as
  * tad_forward followed by tad_backward).  Inputs are copied to the device staging area,
  * results copied back; all copies and launches are enqueued on the stream and the call
@@ -236,7 +253,11 @@ typedef struct {
     int32_t n_launches;     /* kernel launches this part issues */
 } tad_kernel_stats;
 
-/* which = -1: forward kernel; which = q: backward kernel of index expression q. */
+/* Number of staged adjoints (|f| floats of workspace each). */
+int32_t tad_plan_num_stages(const tad_plan *plan);
+
+/* which = -1: forward kernel; which = q >= 0: backward kernel of index expression q;
+ * which = -2 - s: staging kernel s. */
 tad_status tad_plan_kernel_stats(const tad_plan *plan, int32_t which, tad_kernel_stats *out);
 
 /* Human-readable listing of the compiled program (`which` as above); returns bytes needed. */

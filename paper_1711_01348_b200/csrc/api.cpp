@@ -40,6 +40,7 @@ tad_status tad_compile(const tad_expr *expr, const tad_options *opt, tad_plan **
         for (int q = 0; q < (int)p->access.size(); ++q)
             if (p->access[q].used) analyse_access(*p, q);
         generate_forward(*p);
+        generate_stages(*p);
         p->arg_kernels.assign(p->n_args, {});
         p->arg_zero_fill.assign(p->n_args, false);
         for (int q = 0; q < (int)p->access.size(); ++q)
@@ -54,6 +55,8 @@ tad_status tad_compile(const tad_expr *expr, const tad_options *opt, tad_plan **
 }
 
 void tad_destroy(tad_plan *plan) { delete plan; }
+
+int32_t tad_plan_num_stages(const tad_plan *plan) { return plan ? (int32_t)plan->stages.size() : 0; }
 
 tad_status tad_plan_access_info(const tad_plan *plan, int32_t access, tad_access_info *out)
 {
@@ -113,6 +116,7 @@ tad_status tad_plan_enumerate(const tad_plan *plan, int32_t access, const int64_
 static const Kernel *pick_kernel(const tad_plan *plan, int32_t which)
 {
     if (which == -1) return &plan->forward;
+    if (which <= -2 && -2 - which < (int)plan->stages.size()) return &plan->stages[-2 - which];
     for (const Kernel &k : plan->backward) if (k.access == which) return &k;
     return nullptr;
 }

@@ -57,6 +57,8 @@ struct Gen {
     std::vector<int> zorder;                                  // loop l -> kernel column
     std::vector<int> zpos;                                    // kernel column -> loop position
     int lane_var = -1;
+    std::map<int, int> staged;                                // sum node -> pointer slot of its staged adjoint
+    std::vector<int> stages_used;                             // pointer slots the derivative reads
 
     Gen(tad_plan &pl, int acc) : p(pl), q(acc) {}
 
@@ -226,58 +228,80 @@ struct Gen {
 
     // -- reverse accumulation (Sec. 2): the adjoint of the root is df; returns the term Delta
     //    of Sec. 5.3, i.e. df * d f / d x^{pq} with every sum on the path to the leaf liberated
-    int differentiate(int df_inst)
+    //    With target >= 0 the accumulation stops at that node and its adjoint is returned.
+    int differentiate(int df_inst, int target = -1)
     {
         const int root = (int)p.nodes.size() - 1;
         std::vector<bool> active(p.nodes.size(), false);
         for (int n = 0; n <= root; ++n) {
             const NodeH &nd = p.nodes[n];
             if (!nd.reachable) continue;
-            if (nd.op == TAD_OP_LOAD) active[n] = nd.access == q;
-            else active[n] = (nd.in0 >= 0 && active[nd.in0]) || (nd.in1 >= 0 && active[nd.in1]);
+            if (target >= 0) { if (n == target) { active[n] = true; continue; } }
+            else if (nd.op == TAD_OP_LOAD) { active[n] = nd.access == q; continue; }
+            active[n] = (nd.in0 >= 0 && active[nd.in0]) || (nd.in1 >= 0 && active[nd.in1]);
+        }
+        // need[n]: the adjoint of n has to be built from its consumers (it is not staged and
+        // some path from it reaches a wanted leaf without crossing a staged node first)
+        std::vector<bool> need(p.nodes.size(), false);
+        for (int n = 0; n <= root; ++n) {
+            if (!active[n]) continue;
+            const NodeH &nd = p.nodes[n];
+            bool leaf = target >= 0 ? n == target : (nd.op == TAD_OP_LOAD && nd.access == q);
+            bool below = false;
+            for (int c : {nd.in0, nd.in1})
+                if (c >= 0 && active[c] && need[c]) below = true;
+            need[n] = !staged.count(n) && (leaf || below);
         }
         std::vector<int> adj(p.nodes.size(), -1);
         if (!active[root]) return -1;
         adj[root] = df_inst;
         int total = -1;
-        auto push = [&](int c, int x) {
-            if (c < 0 || !active[c]) return;
-            adj[c] = adj[c] < 0 ? x : bin(I_ADD, adj[c], x);
-        };
+        auto wants = [&](int c) { return c >= 0 && active[c] && need[c]; };
+        auto push = [&](int c, int x) { adj[c] = adj[c] < 0 ? x : bin(I_ADD, adj[c], x); };
         for (int n = root; n >= 0; --n) {
-            if (!active[n] || adj[n] < 0) continue;
+            if (!active[n]) continue;
             const NodeH &nd = p.nodes[n];
             const uint32_t F = nd.scope;          // every enclosing sum lies on the path: liberated
-            const int g = adj[n];
+            int g = adj[n];
+            auto st = staged.find(n);
+            if (st != staged.end()) {
+                // the adjoint of this sum was evaluated once per alpha by a staging kernel
+                std::vector<int64_t> A(size_t(p.n_out) * n_idx(), 0), off(p.n_out, 0);
+                for (int d = 0; d < p.n_out; ++d) A[size_t(d) * n_idx() + d] = 1;
+                g = make_load(st->second, A, off, p.n_out, p.out_shape, F, F);
+                if (std::find(stages_used.begin(), stages_used.end(), st->second) == stages_used.end())
+                    stages_used.push_back(st->second);
+            }
+            if (g < 0) continue;
+            if (n == target) return g;
+            const int a = nd.in0, b = nd.in1;
             switch (nd.op) {
-            case TAD_OP_LOAD: total = total < 0 ? g : bin(I_ADD, total, g); break;
-            case TAD_OP_NEG: push(nd.in0, neg(g)); break;
-            case TAD_OP_ADD: push(nd.in0, g); push(nd.in1, g); break;
-            case TAD_OP_SUB: push(nd.in0, g); push(nd.in1, neg(g)); break;
+            case TAD_OP_LOAD: if (nd.access == q && target < 0) total = total < 0 ? g : bin(I_ADD, total, g); break;
+            case TAD_OP_NEG: if (wants(a)) push(a, neg(g)); break;
+            case TAD_OP_ADD: if (wants(a)) push(a, g); if (wants(b)) push(b, g); break;
+            case TAD_OP_SUB: if (wants(a)) push(a, g); if (wants(b)) push(b, neg(g)); break;
             case TAD_OP_MUL:
-                if (active[nd.in0]) push(nd.in0, bin(I_MUL, g, val(nd.in1, F)));
-                if (active[nd.in1]) push(nd.in1, bin(I_MUL, g, val(nd.in0, F)));
+                if (wants(a)) push(a, bin(I_MUL, g, val(b, F)));
+                if (wants(b)) push(b, bin(I_MUL, g, val(a, F)));
                 break;
             case TAD_OP_DIV:
-                if (active[nd.in0]) push(nd.in0, bin(I_DIV, g, val(nd.in1, F)));
-                if (active[nd.in1]) push(nd.in1, neg(bin(I_DIV, bin(I_MUL, g, val(n, F)), val(nd.in1, F))));
+                if (wants(a)) push(a, bin(I_DIV, g, val(b, F)));
+                if (wants(b)) push(b, neg(bin(I_DIV, bin(I_MUL, g, val(n, F)), val(b, F))));
                 break;
             case TAD_OP_POWI:
-                if (nd.ipow != 0)
-                    push(nd.in0, bin(I_MUL, g, mulc(powi(val(nd.in0, F), nd.ipow - 1), (float)nd.ipow)));
+                if (nd.ipow != 0 && wants(a))
+                    push(a, bin(I_MUL, g, mulc(powi(val(a, F), nd.ipow - 1), (float)nd.ipow)));
                 break;
-            case TAD_OP_EXP: push(nd.in0, bin(I_MUL, g, val(n, F))); break;
-            case TAD_OP_LOG: push(nd.in0, bin(I_DIV, g, val(nd.in0, F))); break;
-            case TAD_OP_SIN: push(nd.in0, bin(I_MUL, g, un(I_COS, val(nd.in0, F)))); break;
-            case TAD_OP_COS: push(nd.in0, neg(bin(I_MUL, g, un(I_SIN, val(nd.in0, F))))); break;
-            case TAD_OP_TANH: {
-                int t = val(n, F);
-                push(nd.in0, bin(I_MUL, g, addc(neg(un(I_SQR, t)), 1.f)));
+            case TAD_OP_EXP: if (wants(a)) push(a, bin(I_MUL, g, val(n, F))); break;
+            case TAD_OP_LOG: if (wants(a)) push(a, bin(I_DIV, g, val(a, F))); break;
+            case TAD_OP_SIN: if (wants(a)) push(a, bin(I_MUL, g, un(I_COS, val(a, F)))); break;
+            case TAD_OP_COS: if (wants(a)) push(a, neg(bin(I_MUL, g, un(I_SIN, val(a, F))))); break;
+            case TAD_OP_TANH:
+                if (wants(a)) { int t = val(n, F); push(a, bin(I_MUL, g, addc(neg(un(I_SQR, t)), 1.f))); }
                 break;
-            }
-            case TAD_OP_SINH: push(nd.in0, bin(I_MUL, g, un(I_COSH, val(nd.in0, F)))); break;
-            case TAD_OP_COSH: push(nd.in0, bin(I_MUL, g, un(I_SINH, val(nd.in0, F)))); break;
-            case TAD_OP_SUM: push(nd.in0, g); break;     // d s-bar / d s = 1 at the liberated index
+            case TAD_OP_SINH: if (wants(a)) push(a, bin(I_MUL, g, un(I_COSH, val(a, F)))); break;
+            case TAD_OP_COSH: if (wants(a)) push(a, bin(I_MUL, g, un(I_SINH, val(a, F)))); break;
+            case TAD_OP_SUM: if (wants(a)) push(a, g); break;     // d s-bar / d s = 1 at the liberated index
             default: break;
             }
         }
@@ -639,12 +663,11 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
 // ---------------------------------------------------------------------------------------
 // forward: outer variables are the output indices, every sum is a bound loop
 // ---------------------------------------------------------------------------------------
-void generate_forward(tad_plan &p)
+namespace {
+
+// kernels that run over the output box: outer variables are the output indices alpha
+void setup_alpha_gen(tad_plan &p, Gen &g)
 {
-    Kernel &k = p.forward;
-    std::memset(&k.prog, 0, sizeof k.prog);
-    k.out_arg = -1; k.access = -1;
-    Gen g(p, -1);
     g.n_outer = p.n_out; g.kappa = 0;
     const int nidx = p.n_out + p.n_sum;
     g.a_c0.assign(nidx, 0); g.a_coef.assign(nidx, std::vector<int64_t>(TADP_MAX_VARS, 0)); g.a_free_ok.assign(nidx, false);
@@ -652,7 +675,10 @@ void generate_forward(tad_plan &p)
         g.new_var(0, p.out_shape[d]);
         g.a_coef[d][d] = 1; g.a_free_ok[d] = true;
     }
-    int root = g.val((int)p.nodes.size() - 1, 0);
+}
+
+void finish_alpha_kernel(tad_plan &p, Gen &g, Kernel &k, int root)
+{
     count_uses(g, root);
     g.lane_var = p.n_out - 1;
     TadpProgram &prog = k.prog;
@@ -666,6 +692,56 @@ void generate_forward(tad_plan &p)
     prog.accumulate = 0; prog.write_only_live = 0;
     emit_kernel(g, k, root, {}, {}, {});
     finish_stats(g, k, false, p.out_elems, 0, false);
+}
+
+}  // namespace
+
+void generate_forward(tad_plan &p)
+{
+    Kernel &k = p.forward;
+    std::memset(&k.prog, 0, sizeof k.prog);
+    k.out_arg = -1; k.access = -1;
+    Gen g(p, -1);
+    setup_alpha_gen(p, g);
+    int root = g.val((int)p.nodes.size() - 1, 0);
+    finish_alpha_kernel(p, g, k, root);
+}
+
+// ---------------------------------------------------------------------------------------
+// staging: the adjoint  df * d f / d s  of a top-level sum node s depends on alpha only and
+// is shared by every gradient whose leaf sits inside that sum.  When it contains a sum of its
+// own (so that re-evaluating it per term would repeat a whole inner loop) it is evaluated
+// once per alpha by a kernel of its own into the workspace and read like df afterwards.
+// ---------------------------------------------------------------------------------------
+void generate_stages(tad_plan &p)
+{
+    const int root = (int)p.nodes.size() - 1;
+    for (int n = 0; n < root; ++n) {
+        const NodeH &nd = p.nodes[n];
+        if (!nd.reachable || nd.op != TAD_OP_SUM || nd.scope != 0) continue;
+        if (p.n_args + 1 + (int)p.stages.size() >= TADP_MAX_PTRS) break;
+        Gen g(p, -1);
+        try {
+            setup_alpha_gen(p, g);
+            std::vector<int64_t> dfA(size_t(p.n_out) * g.n_idx(), 0), dfOff(p.n_out, 0);
+            for (int d = 0; d < p.n_out; ++d) dfA[size_t(d) * g.n_idx() + d] = 1;
+            int df_inst = g.make_load(p.n_args, dfA, dfOff, p.n_out, p.out_shape, 0, 0);
+            int adj = g.differentiate(df_inst, n);
+            if (adj < 0 || adj == df_inst) continue;
+            count_uses(g, adj);
+            bool has_sum = false;
+            for (const Inst &in : g.inst) if (in.uses && in.op == I_SUM) has_sum = true;
+            if (!has_sum) continue;
+            Kernel k;
+            std::memset(&k.prog, 0, sizeof k.prog);
+            k.out_arg = -1; k.access = -1;
+            finish_alpha_kernel(p, g, k, adj);
+            p.stages.push_back(k);
+            p.stage_node.push_back(n);
+        } catch (const Unsupported &) {
+            continue;      // too large to stage: the gradients recompute it
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -722,8 +798,10 @@ void generate_backward(tad_plan &p, int q)
     std::vector<int64_t> dfA(size_t(p.n_out) * nidx, 0), dfOff(p.n_out, 0);
     for (int d = 0; d < p.n_out; ++d) dfA[size_t(d) * nidx + d] = 1;
     int df_inst = g.make_load(p.n_args, dfA, dfOff, p.n_out, p.out_shape, ap.scope, ap.scope);
+    for (size_t st = 0; st < p.stages.size(); ++st) g.staged[p.stage_node[st]] = p.n_args + 1 + (int)st;
     int root = g.differentiate(df_inst);
     if (root < 0) throw BadExpr("internal: index expression has no path to the root");
+    for (int slot : g.stages_used) k.stages_used.push_back(slot - p.n_args - 1);
     count_uses(g, root);
 
     // Lane variable: a variable along which df is contiguous and which fills a warp, if there is

@@ -64,6 +64,7 @@ struct Kernel {
     int out_arg = -1;          // -1: forward (writes f); else the argument whose gradient it writes
     int access = -1;
     int vec = 4;               // vector elements per lane the launcher instantiates
+    std::vector<int> stages_used;   // backward: staged adjoints it reads (indices into tad_plan::stages)
     KernelStats stats;
     std::string listing;
 };
@@ -87,6 +88,8 @@ struct tad_plan {
     // analysis + programs
     std::vector<tad::AccessPlan> access;
     tad::Kernel forward;
+    std::vector<tad::Kernel> stages;            // staged adjoints of top-level sums, one |f|-sized buffer each
+    std::vector<int> stage_node;                // the sum node each stage belongs to
     std::vector<tad::Kernel> backward;          // one per used index expression
     std::vector<std::vector<int>> arg_kernels;  // per argument: indices into backward, launch order
     std::vector<bool> arg_zero_fill;            // the gradient is cleared before its kernels add into it
@@ -103,6 +106,7 @@ size_t enumerate_access(const tad_plan &p, int q, const int64_t *beta, std::vect
 
 // codegen.cpp
 void generate_forward(tad_plan &p);
+void generate_stages(tad_plan &p);
 void generate_backward(tad_plan &p, int q);
 
 }  // namespace tad

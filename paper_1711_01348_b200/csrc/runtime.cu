@@ -158,12 +158,47 @@ tad_status zero_fill(float *out, int64_t n, cudaStream_t stream)
 
 }  // namespace
 
+namespace {
+
+size_t pad256(size_t b) { return (b + 255) & ~size_t(255); }
+
+// workspace layout: [256 B debug word, debug_bounds plans only][stage 0][stage 1]...
+size_t stage_offset(const tad_plan *plan, int s)
+{
+    return (plan->opt.debug_bounds ? 256 : 0) + size_t(s) * pad256(size_t(plan->out_elems) * 4);
+}
+
+bool check_workspace(const tad_plan *plan, void *workspace, size_t workspace_bytes)
+{
+    const size_t need = tad_workspace_bytes(plan);
+    if (need && (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))) {
+        tad::set_error("workspace missing, smaller than tad_workspace_bytes() or not 256-byte aligned");
+        return false;
+    }
+    return true;
+}
+
+bool fill_inputs(const tad_plan *plan, const float *const *args, const float *df, void *workspace, TadpPointers &ptrs)
+{
+    for (int a = 0; a < plan->n_args; ++a) {
+        if (!args[a]) { tad::set_error("NULL argument tensor"); return false; }
+        ptrs.in[a] = args[a];
+    }
+    ptrs.in[plan->n_args] = df;
+    for (int s = 0; s < (int)plan->stages.size(); ++s)
+        ptrs.in[plan->n_args + 1 + s] = reinterpret_cast<const float *>(static_cast<char *>(workspace) + stage_offset(plan, s));
+    ptrs.debug = plan->opt.debug_bounds ? static_cast<int32_t *>(workspace) : nullptr;
+    return true;
+}
+
+}  // namespace
+
 extern "C" {
 
 size_t tad_workspace_bytes(const tad_plan *plan)
 {
     if (!plan) return 0;
-    return plan->opt.debug_bounds ? 256 : 0;
+    return stage_offset(plan, (int)plan->stages.size());
 }
 
 tad_status tad_forward(const tad_plan *plan, const float *const *args, float *f, void *cuda_stream)
@@ -179,35 +214,58 @@ tad_status tad_forward(const tad_plan *plan, const float *const *args, float *f,
     return launch(plan->forward, ptrs, false, (cudaStream_t)cuda_stream);
 }
 
+tad_status tad_backward_stage(const tad_plan *plan, const float *const *args, const float *df,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!plan || !df || (plan->n_args && !args)) { tad::set_error("NULL argument"); return TAD_ERR_INVALID_ARG; }
+    if (!check_workspace(plan, workspace, workspace_bytes)) return TAD_ERR_WORKSPACE;
+    TadpPointers ptrs{};
+    if (!fill_inputs(plan, args, df, workspace, ptrs)) return TAD_ERR_INVALID_ARG;
+    for (int s = 0; s < (int)plan->stages.size(); ++s) {
+        ptrs.out = reinterpret_cast<float *>(static_cast<char *>(workspace) + stage_offset(plan, s));
+        tad_status st = launch(plan->stages[s], ptrs, plan->opt.debug_bounds != 0, (cudaStream_t)cuda_stream);
+        if (st != TAD_OK) return st;
+    }
+    return TAD_OK;
+}
+
+tad_status tad_backward_arg(const tad_plan *plan, const float *const *args, const float *df,
+                            int32_t arg, float *darg, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!plan || !df || !darg || (plan->n_args && !args)) { tad::set_error("NULL argument"); return TAD_ERR_INVALID_ARG; }
+    if (arg < 0 || arg >= plan->n_args) { tad::set_error("no such argument"); return TAD_ERR_INVALID_ARG; }
+    if (!check_workspace(plan, workspace, workspace_bytes)) return TAD_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    TadpPointers ptrs{};
+    if (!fill_inputs(plan, args, df, workspace, ptrs)) return TAD_ERR_INVALID_ARG;
+    if (plan->arg_kernels[arg].empty() || plan->arg_zero_fill[arg]) {
+        tad_status st = zero_fill(darg, plan->arg_elems[arg], stream);
+        if (st != TAD_OK) return st;
+    }
+    ptrs.out = darg;
+    for (int ki : plan->arg_kernels[arg]) {
+        tad_status st = launch(plan->backward[ki], ptrs, plan->opt.debug_bounds != 0, stream);
+        if (st != TAD_OK) return st;
+    }
+    return TAD_OK;
+}
+
 tad_status tad_backward(const tad_plan *plan, const float *const *args, const float *df,
                         float *const *dargs, void *workspace, size_t workspace_bytes, void *cuda_stream)
 {
     if (!plan || !df || !dargs || (plan->n_args && !args)) { tad::set_error("NULL argument"); return TAD_ERR_INVALID_ARG; }
-    const bool debug = plan->opt.debug_bounds != 0;
-    const size_t need = tad_workspace_bytes(plan);
-    if (need && (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u))) {
-        tad::set_error("workspace missing, smaller than tad_workspace_bytes() or not 256-byte aligned");
-        return TAD_ERR_WORKSPACE;
+    bool need_stage = false;
+    for (int a = 0; a < plan->n_args; ++a)
+        if (dargs[a])
+            for (int ki : plan->arg_kernels[a]) if (!plan->backward[ki].stages_used.empty()) need_stage = true;
+    if (need_stage) {
+        tad_status st = tad_backward_stage(plan, args, df, workspace, workspace_bytes, cuda_stream);
+        if (st != TAD_OK) return st;
     }
-    cudaStream_t stream = (cudaStream_t)cuda_stream;
-    TadpPointers ptrs{};
-    for (int a = 0; a < plan->n_args; ++a) {
-        if (!args[a]) { tad::set_error("NULL argument tensor"); return TAD_ERR_INVALID_ARG; }
-        ptrs.in[a] = args[a];
-    }
-    ptrs.in[plan->n_args] = df;
-    ptrs.debug = debug ? static_cast<int32_t *>(workspace) : nullptr;
     for (int a = 0; a < plan->n_args; ++a) {
         if (!dargs[a]) continue;
-        if (plan->arg_kernels[a].empty() || plan->arg_zero_fill[a]) {
-            tad_status st = zero_fill(dargs[a], plan->arg_elems[a], stream);
-            if (st != TAD_OK) return st;
-        }
-        for (int ki : plan->arg_kernels[a]) {
-            ptrs.out = dargs[a];
-            tad_status st = launch(plan->backward[ki], ptrs, debug, stream);
-            if (st != TAD_OK) return st;
-        }
+        tad_status st = tad_backward_arg(plan, args, df, a, dargs[a], workspace, workspace_bytes, cuda_stream);
+        if (st != TAD_OK) return st;
     }
     return TAD_OK;
 }
