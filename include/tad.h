@@ -180,6 +180,32 @@ tad_status tad_backward_arg(const tad_plan *plan, const float *const *args, cons
                             void *cuda_stream);
 
 /*
+ * tad_backward_noalloc: tad_backward for callers that cannot hand over a workspace because
+ * they cannot allocate device memory themselves - for instance a plug-in called from inside
+ * a host application's own memory pool, a callback that runs while allocation is forbidden,
+ * or a process whose device-memory budget is fixed at start-up.  (The paper has no
+ * counterpart: it evaluates derivatives without temporary memory, Sec. 7; this library
+ * stages shared adjoints and therefore needs scratch.)
+ *
+ * The scratch is a fixed array of TAD_NOALLOC_SCRATCH_BYTES inside the library image; every
+ * GPU that loads the library holds that much memory until the process exits.  A plan whose
+ * tad_workspace_bytes() is larger is rejected with TAD_ERR_WORKSPACE and a message; nothing
+ * is launched in that case.  The call allocates nothing (no cudaMalloc / cudaFree, no
+ * allocating library routine); inputs and outputs are still the caller's buffers, with the
+ * same meaning as in tad_backward.
+ *
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call outside any stream capture.  All calls on one device share
+ * the one array, which still holds whatever the previous call wrote: the entry point clears
+ * the part that must start at zero (the debug word of debug_bounds plans) and overwrites the
+ * rest before reading it, but two calls whose work overlaps on the GPU (different streams,
+ * or different plans in flight at once) race on it and give wrong gradients.  Serialise them.
+ */
+#define TAD_NOALLOC_SCRATCH_BYTES (32u * 1024u * 1024u)
+tad_status tad_backward_noalloc(const tad_plan *plan, const float *const *args, const float *df,
+                                float *const *dargs, void *cuda_stream);
+
+/*
  * tad_step_host: one forward and one backward pass with HOST buffers (same meaning as
  * tad_forward followed by tad_backward).  Inputs are copied to the device staging area,
  * results copied back; all copies and launches are enqueued on the stream and the call

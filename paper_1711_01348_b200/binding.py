@@ -23,7 +23,7 @@ STATUS = {0: "TAD_OK", 1: "TAD_ERR_INVALID_ARG", 2: "TAD_ERR_BAD_EXPR", 3: "TAD_
 MAX_IDX, MAX_RANK, MAX_KAPPA = 8, 4, 4
 
 EXPORTS = ["tad_compile", "tad_destroy", "tad_workspace_bytes", "tad_forward", "tad_backward",
-           "tad_backward_stage", "tad_backward_arg", "tad_plan_num_stages",
+           "tad_backward_stage", "tad_backward_arg", "tad_plan_num_stages", "tad_backward_noalloc",
            "tad_staging_bytes", "tad_step_host", "tad_last_error", "tad_debug_status",
            "tad_plan_access_info", "tad_plan_bound_row", "tad_plan_enumerate", "tad_plan_kernel_stats",
            "tad_plan_disassemble", "tad_extended_euclid", "tad_smith_normal_form", "tad_fourier_motzkin"]
@@ -89,6 +89,7 @@ def _load() -> C.CDLL:
     lib.tad_backward.argtypes = [vp, C.POINTER(vp), vp, C.POINTER(vp), vp, C.c_size_t, vp]
     lib.tad_backward_stage.argtypes = [vp, C.POINTER(vp), vp, vp, C.c_size_t, vp]
     lib.tad_backward_arg.argtypes = [vp, C.POINTER(vp), vp, C.c_int32, vp, vp, C.c_size_t, vp]
+    lib.tad_backward_noalloc.argtypes = [vp, C.POINTER(vp), vp, C.POINTER(vp), vp]
     lib.tad_plan_num_stages.argtypes = [vp]; lib.tad_plan_num_stages.restype = C.c_int32
     lib.tad_step_host.argtypes = [vp, C.POINTER(vp), vp, vp, C.POINTER(vp), vp, C.c_size_t, vp]
     lib.tad_last_error.restype = C.c_char_p
@@ -201,6 +202,11 @@ class Plan:
                      stream=0) -> None:
         _check(lib.tad_backward_arg(self._h, self._ptr_array(arg_ptrs), df_ptr, arg, darg_ptr,
                                     workspace_ptr or None, workspace_bytes, stream or None))
+
+    def backward_noalloc(self, arg_ptrs, df_ptr, darg_ptrs, stream: int = 0) -> None:
+        """tad_backward with the library's built-in scratch array instead of a caller workspace."""
+        _check(lib.tad_backward_noalloc(self._h, self._ptr_array(arg_ptrs), df_ptr,
+                                        self._ptr_array(darg_ptrs), stream or None))
 
     def num_stages(self) -> int:
         return int(lib.tad_plan_num_stages(self._h))

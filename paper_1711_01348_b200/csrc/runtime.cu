@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdio>
+#include <mutex>
 #include <string>
 
 #include "plan.h"
@@ -158,7 +160,14 @@ tad_status zero_fill(float *out, int64_t n, cudaStream_t stream)
 
 }  // namespace
 
+// Scratch of tad_backward_noalloc: lives in the library image, one copy per GPU that loads it.
+static __device__ __align__(256) unsigned char tad_noalloc_scratch[TAD_NOALLOC_SCRATCH_BYTES];
+
 namespace {
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+void *g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {};
+std::mutex g_noalloc_mutex;
 
 size_t pad256(size_t b) { return (b + 255) & ~size_t(255); }
 
@@ -322,6 +331,48 @@ tad_status tad_step_host(const tad_plan *plan, const float *const *h_args, const
         if (h_dargs[a] && !check(cudaMemcpyAsync(h_dargs[a], d_dargs[a], size_t(plan->arg_elems[a]) * 4, cudaMemcpyDeviceToHost, stream), "copy of a gradient")) return TAD_ERR_CUDA;
     if (!check(cudaStreamSynchronize(stream), "stream synchronise")) return TAD_ERR_CUDA;
     return TAD_OK;
+}
+
+tad_status tad_backward_noalloc(const tad_plan *plan, const float *const *args, const float *df,
+                                float *const *dargs, void *cuda_stream)
+{
+    if (!plan) { tad::set_error("NULL plan"); return TAD_ERR_INVALID_ARG; }
+    const size_t need = tad_workspace_bytes(plan);
+    if (need > TAD_NOALLOC_SCRATCH_BYTES) {
+        char msg[160];
+        snprintf(msg, sizeof msg, "this plan needs %zu bytes of scratch, tad_backward_noalloc holds at most %zu; "
+                                  "use tad_backward with a caller-provided workspace", need, (size_t)TAD_NOALLOC_SCRATCH_BYTES);
+        tad::set_error(msg);
+        return TAD_ERR_WORKSPACE;
+    }
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) {
+        tad::set_error(e != cudaSuccess ? std::string("cudaGetDevice: ") + cudaGetErrorString(e) : "device ordinal out of range");
+        return TAD_ERR_CUDA;
+    }
+    void *scratch = nullptr;
+    {
+        // once per device, with that device current: the array's name is only a host-side handle,
+        // the device address has to be asked for
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_ptr[dev]) {
+            void *p = nullptr;
+            e = cudaGetSymbolAddress(&p, tad_noalloc_scratch);
+            if (e != cudaSuccess || !p) {
+                tad::set_error(std::string("cudaGetSymbolAddress: ") + cudaGetErrorString(e));
+                return TAD_ERR_CUDA;
+            }
+            g_noalloc_ptr[dev] = p;
+        }
+        scratch = g_noalloc_ptr[dev];
+    }
+    if (plan->opt.debug_bounds) {
+        // the array keeps what the last call left: the debug word has to start at zero
+        e = cudaMemsetAsync(scratch, 0, 256, (cudaStream_t)cuda_stream);
+        if (e != cudaSuccess) { tad::set_error(std::string("clearing the debug word: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
+    }
+    return tad_backward(plan, args, df, dargs, scratch, TAD_NOALLOC_SCRATCH_BYTES, cuda_stream);
 }
 
 tad_status tad_debug_status(const tad_plan *plan, void *workspace, void *cuda_stream)
