@@ -313,9 +313,9 @@ struct Gen {
 
 const char *op_name(int op)
 {
-    static const char *names[] = {"END", "CONST", "LOAD", "NEG", "EXP", "LOG", "SIN", "COS", "TANH", "SINH", "COSH",
-                                  "SQR", "POWI", "ADD", "SUB", "MUL", "DIV", "MULC", "ADDC", "FMA", "LDT", "STT",
-                                  "ZERO", "SUMADD", "SLOOP", "SEND", "ZLOOP", "ZEND", "ACC"};
+    static const char *names[] = {"END", "CONST", "ZERO", "LOAD", "LDT", "NEG", "SQR", "CUBE", "MULC", "ADDC",
+                                  "LDADD", "LDMUL", "FN", "STT", "ACC", "ADD", "SUB", "MUL", "DIV", "SUMADD",
+                                  "MACC", "FMA", "SLOOP", "SEND", "ZLOOP", "ZEND"};
     return op < P_NUM_OPS ? names[op] : "?";
 }
 
@@ -328,16 +328,17 @@ struct Emitter {
 
     explicit Emitter(Gen &gen) : g(gen) {}
 
-    int emit(int op, int a = 0, int b = 0, int32_t imm = 0, int delta = 0)
+    // k_override >= 0: the handler number carries a loop variable instead of the stack depth
+    int emit(int op, int a = 0, int b = 0, int32_t imm = 0, int delta = 0, int k_override = -1)
     {
         if (depth + delta > TADP_MAX_DEPTH - 1) throw Unsupported("expression needs a deeper operand stack");
         TadpInsn w{};
-        w.handler = (uint16_t)(op * TADP_MAX_DEPTH + depth);
+        w.handler = (uint16_t)(op * 8 + (k_override >= 0 ? k_override : depth));
         w.a = (uint8_t)a; w.b = (uint8_t)b; w.imm = imm;
         code.push_back(w);
         char line[160];
         float f; std::memcpy(&f, &imm, 4);
-        std::snprintf(line, sizeof line, "%3zu  d=%d  %-7s a=%d imm=%d (%g)\n", code.size() - 1, depth, op_name(op), a, imm, (double)f);
+        std::snprintf(line, sizeof line, "%3zu  d=%d  %-7s a=%d b=%d imm=%d (%g)\n", code.size() - 1, depth, op_name(op), a, b, imm, (double)f);
         listing += line;
         depth += delta;
         max_depth = std::max(max_depth, depth);
@@ -347,6 +348,7 @@ struct Emitter {
     static int32_t fbits(float f) { int32_t b; std::memcpy(&b, &f, 4); return b; }
 
     bool inline_ok(int i) const { return g.inst[i].temp < 0; }
+    bool is_inline_load(int i) const { return g.inst[i].op == I_LOAD && g.inst[i].temp < 0; }
 
     // emits code that leaves the value of instance i on the stack
     void expr(int i)
@@ -361,15 +363,18 @@ struct Emitter {
         case I_CONST: emit(P_CONST, 0, 0, fbits(in.imm), +1); break;
         case I_LOAD: emit(P_LOAD, in.load, 0, 0, +1); break;
         case I_NEG: expr(in.a); emit(P_NEG); break;
-        case I_EXP: expr(in.a); emit(P_EXP); break;
-        case I_LOG: expr(in.a); emit(P_LOG); break;
-        case I_SIN: expr(in.a); emit(P_SIN); break;
-        case I_COS: expr(in.a); emit(P_COS); break;
-        case I_TANH: expr(in.a); emit(P_TANH); break;
-        case I_SINH: expr(in.a); emit(P_SINH); break;
-        case I_COSH: expr(in.a); emit(P_COSH); break;
+        case I_EXP: expr(in.a); emit(P_FN, 0, F_EXP); break;
+        case I_LOG: expr(in.a); emit(P_FN, 0, F_LOG); break;
+        case I_SIN: expr(in.a); emit(P_FN, 0, F_SIN); break;
+        case I_COS: expr(in.a); emit(P_FN, 0, F_COS); break;
+        case I_TANH: expr(in.a); emit(P_FN, 0, F_TANH); break;
+        case I_SINH: expr(in.a); emit(P_FN, 0, F_SINH); break;
+        case I_COSH: expr(in.a); emit(P_FN, 0, F_COSH); break;
         case I_SQR: expr(in.a); emit(P_SQR); break;
-        case I_POWI: expr(in.a); emit(P_POWI, 0, 0, in.ipow); break;
+        case I_POWI:
+            expr(in.a);
+            if (in.ipow == 3) emit(P_CUBE); else emit(P_FN, 0, F_POWI, in.ipow);
+            break;
         case I_MULC: expr(in.a); emit(P_MULC, 0, 0, fbits(in.imm)); break;
         case I_ADDC: expr(in.a); emit(P_ADDC, 0, 0, fbits(in.imm)); break;
         case I_ADD: {
@@ -378,11 +383,17 @@ struct Emitter {
             if (g.inst[in.a].op == I_MUL && inline_ok(in.a)) { m = in.a; o = in.b; }
             else if (g.inst[in.b].op == I_MUL && inline_ok(in.b)) { m = in.b; o = in.a; }
             if (m >= 0) { expr(g.inst[m].a); expr(g.inst[m].b); expr(o); emit(P_FMA, 0, 0, 0, -2); }
+            else if (is_inline_load(in.b)) { expr(in.a); emit(P_LDADD, g.inst[in.b].load); }
+            else if (is_inline_load(in.a)) { expr(in.b); emit(P_LDADD, g.inst[in.a].load); }
             else { expr(in.a); expr(in.b); emit(P_ADD, 0, 0, 0, -1); }
             break;
         }
         case I_SUB: expr(in.a); expr(in.b); emit(P_SUB, 0, 0, 0, -1); break;
-        case I_MUL: expr(in.a); expr(in.b); emit(P_MUL, 0, 0, 0, -1); break;
+        case I_MUL:
+            if (is_inline_load(in.b)) { expr(in.a); emit(P_LDMUL, g.inst[in.b].load); }
+            else if (is_inline_load(in.a)) { expr(in.b); emit(P_LDMUL, g.inst[in.a].load); }
+            else { expr(in.a); expr(in.b); emit(P_MUL, 0, 0, 0, -1); }
+            break;
         case I_DIV: expr(in.a); expr(in.b); emit(P_DIV, 0, 0, 0, -1); break;
         case I_SUM: {
             TadpLoop L{};
@@ -391,11 +402,11 @@ struct Emitter {
             loops.push_back(L);
             int id = (int)loops.size() - 1;
             emit(P_ZERO, 0, 0, 0, +1);
-            int begin = emit(P_SLOOP, id);
+            int begin = emit(P_SLOOP, id, 0, 0, 0, in.var);
             temps_of_sum(i);
             expr(in.a);
             emit(P_SUMADD, 0, 0, 0, -1);
-            int end = emit(P_SEND, id, 0, begin + 1);
+            int end = emit(P_SEND, id, 0, begin + 1, 0, in.var);
             code[begin].imm = end + 1;
             break;
         }
@@ -612,14 +623,19 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
         L.is_lane = L.var == g.lane_var;
         L.mask_level = l + 1;
         em.loops.push_back(L);
-        zbegin[l] = em.emit(P_ZLOOP, (int)em.loops.size() - 1);
+        zbegin[l] = em.emit(P_ZLOOP, (int)em.loops.size() - 1, 0, 0, 0, L.var);
         em.temps_of_level(l + 1);
     }
-    em.expr(root);
-    em.emit(P_ACC, 0, 0, 0, -1);
+    if (g.inst[root].op == I_MUL && g.inst[root].temp < 0) {
+        em.expr(g.inst[root].a); em.expr(g.inst[root].b);
+        em.emit(P_MACC, 0, 0, 0, -2);
+    } else {
+        em.expr(root);
+        em.emit(P_ACC, 0, 0, 0, -1);
+    }
     for (int l = g.kappa - 1; l >= 0; --l) {
         int loop_id = em.code[zbegin[l]].a;
-        int end = em.emit(P_ZEND, loop_id, 0, zbegin[l] + 1);
+        int end = em.emit(P_ZEND, loop_id, 0, zbegin[l] + 1, 0, em.loops[loop_id].var);
         em.code[zbegin[l]].imm = end + 1;
     }
     em.emit(P_END);
@@ -644,6 +660,7 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     std::copy(em.code.begin(), em.code.end(), prog.code);
     prog.n_loads = (int32_t)g.loads.size();
     std::copy(g.loads.begin(), g.loads.end(), prog.loads);
+    for (int i = 0; i < prog.n_loads; ++i) prog.loads[i].lane_step = to_i32(32 * (int64_t)prog.loads[i].coef[g.lane_var]);
     prog.n_loops = (int32_t)em.loops.size();
     std::copy(em.loops.begin(), em.loops.end(), prog.loops);
     prog.n_rows = (int32_t)rows.size();
@@ -651,7 +668,8 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     prog.n_outer = g.n_outer;
     prog.lane_var = g.lane_var;
     const int64_t lane_ext = g.vars[g.lane_var].ext;
-    k.vec = lane_ext >= 128 ? 4 : lane_ext >= 64 ? 2 : 1;
+    k.vec = lane_ext >= 256 ? 8 : lane_ext >= 128 ? 4 : lane_ext >= 64 ? 2 : 1;
+    if (lane_ext >= 512 && em.max_depth <= TADP_WIDE_DEPTH) k.vec = 16;
     char head[256];
     std::snprintf(head, sizeof head, "; vars=%zu outer=%d kappa=%d lane_var=%d vec=%d temps=%d max_depth=%d loads=%d rows=%d guards=%d\n",
                   g.vars.size(), g.n_outer, g.kappa, g.lane_var, k.vec, n_temps, em.max_depth, prog.n_loads, prog.n_rows, prog.n_guards);

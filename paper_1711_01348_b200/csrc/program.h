@@ -15,43 +15,54 @@
 #define TADP_NUM_TEMPS 8      // temporaries held in registers; further ones spill to local memory
 #define TADP_MAX_SPILL 16
 #define TADP_MAX_ZLOOPS 4     // kernel-coordinate loops per kernel
+#define TADP_WIDE_DEPTH 4     // operand stack depth of the 16-element interpreter variant
 
-// Interpreter operations.  The handler a word selects is op * TADP_MAX_DEPTH + d where d is
-// the operand stack depth BEFORE the instruction, known to the host at emission time; this
-// lets every handler name its operand registers statically.
+// Interpreter operations.  The handler a word selects is op * 8 + k.  For operations on the
+// operand stack k is the stack depth BEFORE the instruction, known to the host at emission
+// time, so that every handler names its operand registers statically; for loop control k is
+// the loop variable.
 enum TadpOp : int {
     P_END = 0,
-    P_CONST,      // push imm (float bits)
-    P_LOAD,       // push element-wise load through loads[a]
-    P_NEG, P_EXP, P_LOG, P_SIN, P_COS, P_TANH, P_SINH, P_COSH,
-    P_SQR,        // top <- top^2
-    P_POWI,       // top <- top ** imm (signed integer)
-    P_ADD, P_SUB, P_MUL, P_DIV,   // second <- second op top ; pop
+    // push one value (k = 0..6)
+    P_CONST,      // imm (float bits)
+    P_ZERO,       // 0 (accumulator of a value sum)
+    P_LOAD,       // element-wise load through loads[a]
+    P_LDT,        // temp[a]
+    // replace the top (k = 1..7)
+    P_NEG, P_SQR, P_CUBE,
     P_MULC, P_ADDC,               // top <- top op imm(float)
-    P_FMA,        // third <- third * second + top ; pop 2
-    P_LDT,        // push temp[a]
+    P_LDADD, P_LDMUL,             // top <- top op load(loads[a])
+    P_FN,         // top <- function b of top: TadpFn; P_FN_POWI takes its exponent from imm
     P_STT,        // temp[a] <- top ; pop
-    P_ZERO,       // push 0 (accumulator of a value sum)
+    P_ACC,        // acc += active ? top : 0 ; pop
+    // two operands (k = 2..7): second <- second op top ; pop
+    P_ADD, P_SUB, P_MUL, P_DIV,
     P_SUMADD,     // second += top ; pop
+    P_MACC,       // acc += active ? second * top : 0 ; pop 2
+    // three operands (k = 3..7)
+    P_FMA,        // third <- third * second + top ; pop 2
+    // loop control (k = loop variable)
     P_SLOOP,      // bound sum loop begin: loops[a]; jumps to imm when the range is empty
     P_SEND,       // bound sum loop end: increments, jumps back to imm while in range
     P_ZLOOP,      // kernel-coordinate loop begin: loops[a]; computes the range from its bound rows
     P_ZEND,       // kernel-coordinate loop end
-    P_ACC,        // acc += active ? top : 0 ; pop
     P_NUM_OPS
 };
 
-struct TadpInsn {          // 8 bytes
-    uint16_t handler;      // op * TADP_MAX_DEPTH + depth
+enum TadpFn : int { F_EXP = 0, F_LOG, F_SIN, F_COS, F_TANH, F_SINH, F_COSH, F_POWI };
+
+struct alignas(8) TadpInsn {   // 8 bytes, fetched as one 64-bit constant load
+    uint16_t handler;      // op * 8 + k
     uint8_t a, b;
     int32_t imm;
 };
 
-struct TadpLoad {
-    int32_t ptr;                       // which pointer slot (arguments first, then df)
-    int32_t base;                      // constant element offset
+struct alignas(16) TadpLoad {         // 48 bytes, 16-byte aligned: three 128-bit constant loads
     int32_t coef[TADP_MAX_VARS];       // element offset = base + sum_v coef[v] * var[v]  (mod 2^32)
+    int32_t base;                      // constant element offset
+    int32_t ptr;                       // which pointer slot (arguments first, then df, then staged adjoints)
     int32_t limit;                     // elements in the tensor (debug bounds)
+    int32_t lane_step;                 // 32 * coef[lane variable]: offset step between vector elements
 };
 
 struct TadpRow {                       // value = (c0 + sum_v coef[v] * var[v]) / den, den > 0
@@ -70,7 +81,7 @@ struct TadpLoop {
     int32_t mask_level;                // position of its activity mask in the mask word (1..)
 };
 
-struct TadpProgram {
+struct alignas(16) TadpProgram {
     int32_t n_code, n_loads, n_loops, n_rows;
     int32_t n_outer;                   // outer variables 0 .. n_outer-1 (decoded from the work item)
     int32_t lane_var;                  // variable spread over lanes; < n_outer: distinct outputs per lane

@@ -21,7 +21,7 @@ using namespace tadvm;
 // One warp per work item, grid-stride over the items.  A work item fixes every outer variable
 // except the lane variable, which the warp covers 32 * T elements at a time.
 template <int T, bool DEBUG>
-__global__ void __launch_bounds__(WARPS_PER_BLOCK * 32)
+__global__ void __launch_bounds__(WARPS_PER_BLOCK * 32, 2)
 tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ TadpPointers ptrs, unsigned n_items)
 {
     const unsigned lane = threadIdx.x & 31u;
@@ -142,6 +142,8 @@ tad_status launch(const tad::Kernel &k, const TadpPointers &ptrs, bool debug, cu
     switch (k.vec) {
     case 1: launch_t<1>(k, ptrs, debug, items, blocks, stream); break;
     case 2: launch_t<2>(k, ptrs, debug, items, blocks, stream); break;
+    case 8: launch_t<8>(k, ptrs, debug, items, blocks, stream); break;
+    case 16: launch_t<16>(k, ptrs, debug, items, blocks, stream); break;
     default: launch_t<4>(k, ptrs, debug, items, blocks, stream); break;
     }
     cudaError_t e = cudaGetLastError();
