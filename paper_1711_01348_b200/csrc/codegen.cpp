@@ -667,12 +667,48 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     std::copy(rows.begin(), rows.end(), prog.rows);
     prog.n_outer = g.n_outer;
     prog.lane_var = g.lane_var;
+    // Vector width and summation split.  Wide vectors amortise the interpreter's dispatch cost,
+    // but only while enough warps remain to fill the GPU; when even the narrowest shape leaves
+    // too few, the outermost kernel-coordinate loop is divided among several warps per output,
+    // each writing a partial sum that a second launch adds up in a fixed order.
     const int64_t lane_ext = g.vars[g.lane_var].ext;
-    k.vec = lane_ext >= 256 ? 8 : lane_ext >= 128 ? 4 : lane_ext >= 64 ? 2 : 1;
-    if (lane_ext >= 512 && em.max_depth <= TADP_WIDE_DEPTH) k.vec = 16;
+    const double target_warps = 148.0 * 16.0 * 2.0;
+    auto items_for = [&](int T) {
+        double n = 1;
+        for (int v = 0; v < g.n_outer; ++v) {
+            double e = (double)prog.outer_ext[v];
+            if (v == g.lane_var) e = std::ceil(e / (32.0 * T));
+            n *= e;
+        }
+        return n;
+    };
+    const bool debug = g.p.opt.debug_bounds != 0;
+    auto allowed = [&](int T) {
+        if (T == 16 && em.max_depth > TADP_WIDE_DEPTH) return false;
+        if (debug && T > 4) return false;
+        return T == 1 || lane_ext >= 32 * T;
+    };
+    prog.zsplit = 1;
+    k.vec = 1;
+    if (g.kappa >= 1) {
+        // a summation that can be split: take the widest vector and split to fill the GPU
+        for (int T : {16, 8, 4, 2, 1}) if (allowed(T)) { k.vec = T; break; }
+        // splitting costs a pass over zsplit x outputs: only for small gradients that starve the GPU
+        if (items_for(k.vec) < target_warps / 2 && prog.out_limit <= (1 << 22)) {
+            TadpLoop &L0 = prog.loops[em.code[zbegin[0]].a];
+            const int64_t ext0 = std::max<int64_t>(1, g.vars[L0.var].ext / (L0.is_lane ? 32 * k.vec : 1));
+            int64_t S = (int64_t)std::ceil(target_warps / items_for(k.vec));
+            S = std::min<int64_t>(std::min<int64_t>(S, ext0), 4096);
+            while (S > 1 && S * (int64_t)prog.out_limit > (int64_t(1) << 25)) S /= 2;   // <= 128 MB of partial sums
+            if (S >= 2) { prog.zsplit = (int32_t)S; L0.is_split = 1; }
+        }
+    } else {
+        // element-wise kernel: the widest vector that still leaves enough warps
+        for (int T : {16, 8, 4, 2, 1}) if (allowed(T) && (items_for(T) >= target_warps || T == 1)) { k.vec = T; break; }
+    }
     char head[256];
-    std::snprintf(head, sizeof head, "; vars=%zu outer=%d kappa=%d lane_var=%d vec=%d temps=%d max_depth=%d loads=%d rows=%d guards=%d\n",
-                  g.vars.size(), g.n_outer, g.kappa, g.lane_var, k.vec, n_temps, em.max_depth, prog.n_loads, prog.n_rows, prog.n_guards);
+    std::snprintf(head, sizeof head, "; vars=%zu outer=%d kappa=%d lane_var=%d vec=%d zsplit=%d temps=%d max_depth=%d loads=%d rows=%d guards=%d\n",
+                  g.vars.size(), g.n_outer, g.kappa, g.lane_var, k.vec, prog.zsplit, n_temps, em.max_depth, prog.n_loads, prog.n_rows, prog.n_guards);
     k.listing = head + em.listing;
 }
 
@@ -925,6 +961,10 @@ void generate_backward(tad_plan &p, int q)
     int64_t terms = 1;
     for (int d = 0; d < n; ++d) terms = mul_ck(terms, ap.box_hi[d] - ap.box_lo[d] + 1);
     finish_stats(g, k, true, p.arg_elems[ap.arg], terms, zero_fill && first_of_arg);
+    if (prog.zsplit > 1) {
+        p.partial_bytes = std::max(p.partial_bytes, size_t(prog.zsplit) * size_t(prog.out_limit) * 4);
+        k.stats.n_launches += 1 + (prog.write_only_live ? 1 : 0);
+    }
 }
 
 }  // namespace tad

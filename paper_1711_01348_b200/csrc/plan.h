@@ -93,6 +93,7 @@ struct tad_plan {
     std::vector<tad::Kernel> backward;          // one per used index expression
     std::vector<std::vector<int>> arg_kernels;  // per argument: indices into backward, launch order
     std::vector<bool> arg_zero_fill;            // the gradient is cleared before its kernels add into it
+    size_t partial_bytes = 0;                   // workspace for the partial sums of split summations (largest kernel)
 };
 
 namespace tad {

@@ -78,7 +78,8 @@ struct TadpLoop {
     int32_t const_lo, const_hi;        // bound-sum loops: inclusive constant range
     int16_t lower0, n_lower;           // rows[lower0 .. lower0 + n_lower)
     int16_t upper0, n_upper;
-    int32_t mask_level;                // position of its activity mask in the mask word (1..)
+    int32_t mask_level;                // position of its activity mask in the mask stack (1..)
+    int32_t is_split;                  // 1: its range is divided among the zsplit warps that share an output
 };
 
 struct alignas(16) TadpProgram {
@@ -93,6 +94,7 @@ struct alignas(16) TadpProgram {
     int32_t out_limit;
     int32_t accumulate;                // 0: out = acc ; 1: out += acc
     int32_t write_only_live;           // 1: skip elements whose Gamma is empty (output pre-zeroed)
+    int32_t zsplit;                    // > 1: that many warps share every output; each writes a partial sum
     TadpInsn code[TADP_MAX_CODE];
     TadpLoad loads[TADP_MAX_LOADS];
     TadpLoop loops[TADP_MAX_LOOPS];
@@ -102,5 +104,6 @@ struct alignas(16) TadpProgram {
 struct TadpPointers {
     const float *in[TADP_MAX_PTRS];
     float *out;
+    float *part;                       // zsplit > 1: partial sums, zsplit planes of out_limit floats
     int32_t *debug;                    // NULL unless the plan was compiled with debug_bounds
 };

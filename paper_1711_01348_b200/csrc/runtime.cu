@@ -30,7 +30,11 @@ tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ Tad
     const int lane_var = P.lane_var;
     const bool lane_outer = lane_var < P.n_outer;
     Vm<T> m;
-    for (unsigned item = warp; item < n_items; item += n_warps) {
+    const unsigned zsplit = P.zsplit > 1 ? (unsigned)P.zsplit : 1u;
+    for (unsigned witem = warp; witem < n_items; witem += n_warps) {
+        // warps witem = item * zsplit + s share the outputs of `item`
+        const unsigned item = witem / zsplit;
+        const int split = (int)(witem % zsplit);
         // decode the outer variables (last one fastest)
         unsigned rem = item;
 #pragma unroll
@@ -64,7 +68,7 @@ tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ Tad
             for (int t = 0; t < T; ++t) if (nmr + t * step > 0) mask0 &= ~(1u << t);
         }
         unsigned live = 0;
-        run_item<T, DEBUG>(P, ptrs, m, mask0, live);
+        run_item<T, DEBUG>(P, ptrs, m, mask0, split, live);
         // output
         if (lane_outer) {
             unsigned off = (unsigned)P.out_base;
@@ -77,7 +81,8 @@ tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ Tad
                 if (P.write_only_live && !((live >> t) & 1u)) continue;
                 const unsigned idx = off + (unsigned)t * step;
                 if (DEBUG && idx >= (unsigned)P.out_limit) { if (ptrs.debug) atomicCAS(ptrs.debug, 0, 0x20000); continue; }
-                ptrs.out[idx] = P.accumulate ? ptrs.out[idx] + m.acc[t] : m.acc[t];
+                if (zsplit > 1) ptrs.part[(size_t)split * (unsigned)P.out_limit + idx] = m.acc[t];
+                else ptrs.out[idx] = P.accumulate ? ptrs.out[idx] + m.acc[t] : m.acc[t];
             }
         } else {
             // the lane variable is a kernel coordinate: one output per warp, fixed-order tree reduction
@@ -92,9 +97,21 @@ tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ Tad
             const unsigned any_live = __ballot_sync(0xffffffffu, live != 0);
             if (lane == 0 && !(P.write_only_live && !any_live)) {
                 if (DEBUG && off >= (unsigned)P.out_limit) { if (ptrs.debug) atomicCAS(ptrs.debug, 0, 0x20000); }
+                else if (zsplit > 1) ptrs.part[(size_t)split * (unsigned)P.out_limit + off] = total;
                 else ptrs.out[off] = P.accumulate ? ptrs.out[off] + total : total;
             }
         }
+    }
+}
+
+// out[i] (+)= part[0][i] + part[1][i] + ... in that order
+__global__ void tad_reduce_partials(float *out, const float *part, unsigned n, int planes, int accumulate)
+{
+    const unsigned stride = gridDim.x * blockDim.x;
+    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        float sum = accumulate ? out[i] : 0.f;
+        for (int s = 0; s < planes; ++s) sum += part[(size_t)s * n + i];
+        out[i] = sum;
     }
 }
 
@@ -130,9 +147,20 @@ void launch_t(const tad::Kernel &k, const TadpPointers &ptrs, bool debug, unsign
     else tad_vm_kernel<T, false><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items);
 }
 
-tad_status launch(const tad::Kernel &k, const TadpPointers &ptrs, bool debug, cudaStream_t stream)
+tad_status zero_fill(float *out, int64_t n, cudaStream_t stream);
+
+tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStream_t stream)
 {
-    const unsigned long long items64 = item_count(k.prog, k.vec);
+    const int zsplit = k.prog.zsplit > 1 ? k.prog.zsplit : 1;
+    if (zsplit > 1) {
+        if (!ptrs.part) { tad::set_error("internal: partial-sum buffer missing"); return TAD_ERR_WORKSPACE; }
+        if (k.prog.write_only_live) {
+            // masked gradients leave elements unvisited: their partial sums must read as zero
+            tad_status st = zero_fill(ptrs.part, (int64_t)zsplit * k.prog.out_limit, stream);
+            if (st != TAD_OK) return st;
+        }
+    }
+    const unsigned long long items64 = item_count(k.prog, k.vec) * (unsigned long long)zsplit;
     if (items64 == 0) return TAD_OK;
     if (items64 >= (1ull << 32)) { tad::set_error("too many work items"); return TAD_ERR_UNSUPPORTED; }
     const unsigned items = (unsigned)items64;
@@ -148,6 +176,13 @@ tad_status launch(const tad::Kernel &k, const TadpPointers &ptrs, bool debug, cu
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { tad::set_error(std::string("kernel launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
+    if (zsplit > 1) {
+        const unsigned n = (unsigned)k.prog.out_limit;
+        const unsigned rblocks = std::min((n + 255u) / 256u, (unsigned)sm_count() * 16u);
+        tad_reduce_partials<<<rblocks, 256, 0, stream>>>(ptrs.out, ptrs.part, n, zsplit, k.prog.accumulate);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { tad::set_error(std::string("reduce launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
+    }
     return TAD_OK;
 }
 
@@ -199,6 +234,8 @@ bool fill_inputs(const tad_plan *plan, const float *const *args, const float *df
     for (int s = 0; s < (int)plan->stages.size(); ++s)
         ptrs.in[plan->n_args + 1 + s] = reinterpret_cast<const float *>(static_cast<char *>(workspace) + stage_offset(plan, s));
     ptrs.debug = plan->opt.debug_bounds ? static_cast<int32_t *>(workspace) : nullptr;
+    ptrs.part = plan->partial_bytes
+        ? reinterpret_cast<float *>(static_cast<char *>(workspace) + stage_offset(plan, (int)plan->stages.size())) : nullptr;
     return true;
 }
 
@@ -209,7 +246,7 @@ extern "C" {
 size_t tad_workspace_bytes(const tad_plan *plan)
 {
     if (!plan) return 0;
-    return stage_offset(plan, (int)plan->stages.size());
+    return stage_offset(plan, (int)plan->stages.size()) + pad256(plan->partial_bytes);
 }
 
 tad_status tad_forward(const tad_plan *plan, const float *const *args, float *f, void *cuda_stream)

@@ -116,7 +116,7 @@ __device__ __forceinline__ unsigned load_offset(const TadpLoad &L, const int (&v
 // the outermost level.  Returns in live_out the elements that accumulated at least one term.
 template <int T, bool DEBUG>
 __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointers &ptrs, Vm<T> &m,
-                                         unsigned mask0, unsigned &live_out)
+                                         unsigned mask0, int split, unsigned &live_out)
 {
     const int lane_var = P.lane_var;
     unsigned cur = mask0;                 // activity mask of the vector elements at the current loop level
@@ -237,6 +237,11 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                 for (int r = 0; r < L.n_lower; ++r) { const TadpRow &R = P.rows[L.lower0 + r]; const int nmr = row_num(R, m.var); lo = max(lo, R.den == 1 ? nmr : ceil_div_i(nmr, R.den)); } \
                 for (int r = 0; r < L.n_upper; ++r) { const TadpRow &R = P.rows[L.upper0 + r]; const int nmr = row_num(R, m.var); hi = min(hi, R.den == 1 ? nmr : floor_div_i(nmr, R.den)); } \
                 wlo = lo; whi = hi; \
+                if (L.is_split && lo <= hi) { \
+                    /* this warp's contiguous share of the range (fixed chunking: repeatable sums) */ \
+                    const int chunk = (hi - lo + P.zsplit) / P.zsplit; \
+                    wlo = lo + split * chunk; whi = min(hi, wlo + chunk - 1); \
+                } \
                 if (__ballot_sync(0xffffffffu, parent != 0) == 0) { wlo = 1; whi = 0; } \
             } else { \
                 int lo_w = INT_MAX, hi_w = INT_MIN; \
@@ -250,6 +255,13 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                     const TadpRow &R = P.rows[L.upper0 + r]; \
                     const int nmr = row_num(R, m.var); const int step = R.coef[lane_var] * 32; \
                     _Pragma("unroll") for (int t = 0; t < T; ++t) { int v = nmr + t * step; v = R.den == 1 ? v : floor_div_i(v, R.den); ehi[lvl - 1][t] = min(ehi[lvl - 1][t], v); } \
+                } \
+                if (L.is_split) { \
+                    /* every element's own range is divided into zsplit contiguous shares */ \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) if (elo[lvl - 1][t] <= ehi[lvl - 1][t]) { \
+                        const int chunk = (ehi[lvl - 1][t] - elo[lvl - 1][t] + P.zsplit) / P.zsplit; \
+                        elo[lvl - 1][t] += split * chunk; ehi[lvl - 1][t] = min(ehi[lvl - 1][t], elo[lvl - 1][t] + chunk - 1); \
+                    } \
                 } \
                 _Pragma("unroll") for (int t = 0; t < T; ++t) \
                     if (((parent >> t) & 1u) && elo[lvl - 1][t] <= ehi[lvl - 1][t]) { lo_w = min(lo_w, elo[lvl - 1][t]); hi_w = max(hi_w, ehi[lvl - 1][t]); } \
