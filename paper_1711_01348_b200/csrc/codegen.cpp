@@ -660,7 +660,27 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     std::copy(em.code.begin(), em.code.end(), prog.code);
     prog.n_loads = (int32_t)g.loads.size();
     std::copy(g.loads.begin(), g.loads.end(), prog.loads);
-    for (int i = 0; i < prog.n_loads; ++i) prog.loads[i].lane_step = to_i32(32 * (int64_t)prog.loads[i].coef[g.lane_var]);
+    // relative loop: a kernel-coordinate loop whose range is short but starts at a different value
+    // for every lane (the taps of a strided convolution's transpose): walking the union of all
+    // lanes' ranges would leave almost every element idle
+    prog.rel_var = -1;
+    for (int li = (int)em.loops.size() - 1; li >= 0; --li) {
+        TadpLoop &L = em.loops[li];
+        if (g.vars[L.var].kind != 1 || L.is_lane || !L.depends_on_lane) continue;
+        if (g.vars[L.var].ext > 16) continue;
+        // no other loop's bounds may read this variable through a warp-uniform path
+        bool inner_reads = false;
+        for (const TadpLoop &M : em.loops)
+            if (&M != &L && g.vars[M.var].kind == 1)
+                for (int r = M.lower0; r < M.upper0 + M.n_upper; ++r) if (rows[r].coef[L.var] && !M.depends_on_lane) inner_reads = true;
+        if (inner_reads) continue;
+        L.is_relative = 1; prog.rel_var = L.var;
+        break;
+    }
+    for (int i = 0; i < prog.n_loads; ++i) {
+        prog.loads[i].lane_step = to_i32(32 * (int64_t)prog.loads[i].coef[g.lane_var]);
+        prog.loads[i].rel_step = prog.rel_var >= 0 ? prog.loads[i].coef[prog.rel_var] : 0;
+    }
     prog.n_loops = (int32_t)em.loops.size();
     std::copy(em.loops.begin(), em.loops.end(), prog.loops);
     prog.n_rows = (int32_t)rows.size();

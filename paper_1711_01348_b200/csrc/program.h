@@ -57,12 +57,14 @@ struct alignas(8) TadpInsn {   // 8 bytes, fetched as one 64-bit constant load
     int32_t imm;
 };
 
-struct alignas(16) TadpLoad {         // 48 bytes, 16-byte aligned: three 128-bit constant loads
+struct alignas(16) TadpLoad {         // 64 bytes, 16-byte aligned: 128-bit constant loads
     int32_t coef[TADP_MAX_VARS];       // element offset = base + sum_v coef[v] * var[v]  (mod 2^32)
     int32_t base;                      // constant element offset
     int32_t ptr;                       // which pointer slot (arguments first, then df, then staged adjoints)
     int32_t limit;                     // elements in the tensor (debug bounds)
     int32_t lane_step;                 // 32 * coef[lane variable]: offset step between vector elements
+    int32_t rel_step;                  // coef[variable of the relative loop]
+    int32_t pad[3];
 };
 
 struct TadpRow {                       // value = (c0 + sum_v coef[v] * var[v]) / den, den > 0
@@ -80,6 +82,7 @@ struct TadpLoop {
     int16_t upper0, n_upper;
     int32_t mask_level;                // position of its activity mask in the mask stack (1..)
     int32_t is_split;                  // 1: its range is divided among the zsplit warps that share an output
+    int32_t is_relative;               // 1: every element walks its own short range, trip r visits lo_e + r
 };
 
 struct alignas(16) TadpProgram {
@@ -95,6 +98,7 @@ struct alignas(16) TadpProgram {
     int32_t accumulate;                // 0: out = acc ; 1: out += acc
     int32_t write_only_live;           // 1: skip elements whose Gamma is empty (output pre-zeroed)
     int32_t zsplit;                    // > 1: that many warps share every output; each writes a partial sum
+    int32_t rel_var;                   // variable of the relative loop, or -1
     TadpInsn code[TADP_MAX_CODE];
     TadpLoad loads[TADP_MAX_LOADS];
     TadpLoop loops[TADP_MAX_LOOPS];

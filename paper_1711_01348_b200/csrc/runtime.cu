@@ -20,7 +20,7 @@ using namespace tadvm;
 
 // One warp per work item, grid-stride over the items.  A work item fixes every outer variable
 // except the lane variable, which the warp covers 32 * T elements at a time.
-template <int T, bool DEBUG>
+template <int T, bool DEBUG, bool REL>
 __global__ void __launch_bounds__(WARPS_PER_BLOCK * 32, 2)
 tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ TadpPointers ptrs, unsigned n_items)
 {
@@ -68,7 +68,7 @@ tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ Tad
             for (int t = 0; t < T; ++t) if (nmr + t * step > 0) mask0 &= ~(1u << t);
         }
         unsigned live = 0;
-        run_item<T, DEBUG>(P, ptrs, m, mask0, split, live);
+        run_item<T, DEBUG, REL>(P, ptrs, m, mask0, split, live);
         // output
         if (lane_outer) {
             unsigned off = (unsigned)P.out_base;
@@ -143,8 +143,10 @@ unsigned long long item_count(const TadpProgram &P, int T)
 template <int T>
 void launch_t(const tad::Kernel &k, const TadpPointers &ptrs, bool debug, unsigned items, unsigned blocks, cudaStream_t stream)
 {
-    if (debug) tad_vm_kernel<T, true><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items);
-    else tad_vm_kernel<T, false><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items);
+    // three builds of the interpreter per vector width: plain, with the relative-loop support, with bounds checks
+    if (debug) { if constexpr (T <= 4) tad_vm_kernel<T, true, true><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items); }
+    else if (k.prog.rel_var >= 0) tad_vm_kernel<T, false, true><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items);
+    else tad_vm_kernel<T, false, false><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items);
 }
 
 tad_status zero_fill(float *out, int64_t n, cudaStream_t stream);

@@ -114,7 +114,7 @@ __device__ __forceinline__ unsigned load_offset(const TadpLoad &L, const int (&v
 
 // Runs the program of one work item.  mask0: which vector elements of this lane are live at
 // the outermost level.  Returns in live_out the elements that accumulated at least one term.
-template <int T, bool DEBUG>
+template <int T, bool DEBUG, bool REL>
 __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointers &ptrs, Vm<T> &m,
                                          unsigned mask0, int split, unsigned &live_out)
 {
@@ -125,6 +125,11 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
     unsigned live = 0;
     int loop_hi[TADP_MAX_LOOPS];
     int elo[TADP_MAX_ZLOOPS][T], ehi[TADP_MAX_ZLOOPS][T];
+    // per-element start of the relative loop; in shared memory (one column per thread) because it is
+    // rarely touched and would otherwise cost T registers in every kernel
+    __shared__ int zrel_s[REL ? T : 1][WARPS_PER_BLOCK * 32];
+#define zrel(t) zrel_s[t][threadIdx.x]
+    const int rel_var = REL ? P.rel_var : -1;
     constexpr int NTR = VmCfg<T>::NTR;
     float spill[TADP_MAX_SPILL + TADP_NUM_TEMPS - NTR][T];
 #pragma unroll
@@ -152,13 +157,14 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
             const unsigned off = load_offset(L, m.var); \
             const unsigned lc = (unsigned)L.lane_step; \
             const float *base = ptrs.in[L.ptr]; \
-            if (lc == 0 && !DEBUG) { \
+            if (lc == 0 && (!REL || L.rel_step == 0) && !DEBUG) { \
                 /* the same element for every vector element of this lane: one load */ \
                 const float v = cur ? __ldg(base + off) : 0.f; \
                 _Pragma("unroll") for (int t = 0; t < T; ++t) { DST_EXPR; } \
             } else { \
+                const unsigned rs = REL ? (unsigned)L.rel_step : 0u; \
                 _Pragma("unroll") for (int t = 0; t < T; ++t) { \
-                    const unsigned idx = off + (unsigned)t * lc; \
+                    const unsigned idx = off + (unsigned)t * lc + (REL && rs ? rs * (unsigned)zrel(t) : 0u); \
                     bool ok = (cur >> t) & 1u; \
                     if (DEBUG && ok && idx >= (unsigned)L.limit) { ok = false; if (ptrs.debug) atomicCAS(ptrs.debug, 0, 0x10000 + a); } \
                     const float v = ok ? __ldg(base + idx) : 0.f; \
@@ -249,12 +255,14 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                 for (int r = 0; r < L.n_lower; ++r) { \
                     const TadpRow &R = P.rows[L.lower0 + r]; \
                     const int nmr = row_num(R, m.var); const int step = R.coef[lane_var] * 32; \
-                    _Pragma("unroll") for (int t = 0; t < T; ++t) { int v = nmr + t * step; v = R.den == 1 ? v : ceil_div_i(v, R.den); elo[lvl - 1][t] = max(elo[lvl - 1][t], v); } \
+                    const int rstep = rel_var >= 0 ? R.coef[rel_var] : 0; \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) { int v = nmr + t * step + (REL && rstep ? rstep * zrel(t) : 0); v = R.den == 1 ? v : ceil_div_i(v, R.den); elo[lvl - 1][t] = max(elo[lvl - 1][t], v); } \
                 } \
                 for (int r = 0; r < L.n_upper; ++r) { \
                     const TadpRow &R = P.rows[L.upper0 + r]; \
                     const int nmr = row_num(R, m.var); const int step = R.coef[lane_var] * 32; \
-                    _Pragma("unroll") for (int t = 0; t < T; ++t) { int v = nmr + t * step; v = R.den == 1 ? v : floor_div_i(v, R.den); ehi[lvl - 1][t] = min(ehi[lvl - 1][t], v); } \
+                    const int rstep = rel_var >= 0 ? R.coef[rel_var] : 0; \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) { int v = nmr + t * step + (REL && rstep ? rstep * zrel(t) : 0); v = R.den == 1 ? v : floor_div_i(v, R.den); ehi[lvl - 1][t] = min(ehi[lvl - 1][t], v); } \
                 } \
                 if (L.is_split) { \
                     /* every element's own range is divided into zsplit contiguous shares */ \
@@ -265,10 +273,22 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                 } \
                 _Pragma("unroll") for (int t = 0; t < T; ++t) \
                     if (((parent >> t) & 1u) && elo[lvl - 1][t] <= ehi[lvl - 1][t]) { lo_w = min(lo_w, elo[lvl - 1][t]); hi_w = max(hi_w, ehi[lvl - 1][t]); } \
+                if (REL && L.is_relative) { \
+                    /* trip r visits lo_e + r: the warp runs as many trips as its longest element range */ \
+                    int len = 0; \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) { \
+                        if (((parent >> t) & 1u) && elo[lvl - 1][t] <= ehi[lvl - 1][t]) len = max(len, ehi[lvl - 1][t] - elo[lvl - 1][t] + 1); \
+                        else { ehi[lvl - 1][t] = -1; elo[lvl - 1][t] = 0; } \
+                        zrel(t) = elo[lvl - 1][t]; ehi[lvl - 1][t] -= elo[lvl - 1][t]; elo[lvl - 1][t] = 0; \
+                    } \
+                    _Pragma("unroll") for (int o = 16; o > 0; o >>= 1) len = max(len, __shfl_xor_sync(0xffffffffu, len, o)); \
+                    lo_w = 0; hi_w = len - 1; \
+                } else { \
                 _Pragma("unroll") for (int o = 16; o > 0; o >>= 1) { lo_w = min(lo_w, __shfl_xor_sync(0xffffffffu, lo_w, o)); hi_w = max(hi_w, __shfl_xor_sync(0xffffffffu, hi_w, o)); } \
+                } \
                 wlo = lo_w; whi = hi_w; \
             } \
-            if (wlo > whi) { pc = imm; } \
+            if (wlo > whi) { pc = imm; if (REL && L.is_relative) { _Pragma("unroll") for (int t = 0; t < T; ++t) zrel(t) = 0; } } \
             else { \
                 loop_hi[a] = whi; \
                 unsigned mk; \
@@ -315,6 +335,7 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                 pc = imm; \
             } else { \
                 cur = parent; \
+                if (REL && L.is_relative) { _Pragma("unroll") for (int t = 0; t < T; ++t) zrel(t) = 0; set_var(m.var, V, 0); } \
             } }
         default: {
             const int op = (raw.x & 0xffffu) >> 3;
