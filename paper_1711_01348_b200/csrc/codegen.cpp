@@ -57,6 +57,7 @@ struct Gen {
     std::vector<int> zorder;                                  // loop l -> kernel column
     std::vector<int> zpos;                                    // kernel column -> loop position
     int lane_var = -1;
+    int unroll_var = -1;                                      // element variable B (-1: none)
     std::map<int, int> staged;                                // sum node -> pointer slot of its staged adjoint
     std::vector<int> stages_used;                             // pointer slots the derivative reads
 
@@ -313,9 +314,9 @@ struct Gen {
 
 const char *op_name(int op)
 {
-    static const char *names[] = {"END", "CONST", "ZERO", "LOAD", "LDT", "NEG", "SQR", "CUBE", "MULC", "ADDC",
+    static const char *names[] = {"END", "CONST", "ZERO", "LOAD", "LDT", "NEG", "SQR", "CUBE", "HSUM", "MULC", "ADDC",
                                   "LDADD", "LDMUL", "FN", "STT", "ACC", "ADD", "SUB", "MUL", "DIV", "SUMADD",
-                                  "MACC", "FMA", "SLOOP", "SEND", "ZLOOP", "ZEND"};
+                                  "MACC", "FMA", "SLOOP", "SEND", "USLOOP", "USEND", "ZLOOP", "ZEND"};
     return op < P_NUM_OPS ? names[op] : "?";
 }
 
@@ -348,6 +349,8 @@ struct Emitter {
     static int32_t fbits(float f) { int32_t b; std::memcpy(&b, &f, 4); return b; }
 
     bool inline_ok(int i) const { return g.inst[i].temp < 0; }
+    // the value does not vary along the element variable (and is not computed inside its sum loop)
+    int same_for_all_u(int i) const { return g.unroll_var >= 0 && !(g.inst[i].deps & (1u << g.unroll_var)) ? 1 : 0; }
     bool is_inline_load(int i) const { return g.inst[i].op == I_LOAD && g.inst[i].temp < 0; }
 
     // emits code that leaves the value of instance i on the stack
@@ -363,17 +366,17 @@ struct Emitter {
         case I_CONST: emit(P_CONST, 0, 0, fbits(in.imm), +1); break;
         case I_LOAD: emit(P_LOAD, in.load, 0, 0, +1); break;
         case I_NEG: expr(in.a); emit(P_NEG); break;
-        case I_EXP: expr(in.a); emit(P_FN, 0, F_EXP); break;
-        case I_LOG: expr(in.a); emit(P_FN, 0, F_LOG); break;
-        case I_SIN: expr(in.a); emit(P_FN, 0, F_SIN); break;
-        case I_COS: expr(in.a); emit(P_FN, 0, F_COS); break;
-        case I_TANH: expr(in.a); emit(P_FN, 0, F_TANH); break;
-        case I_SINH: expr(in.a); emit(P_FN, 0, F_SINH); break;
-        case I_COSH: expr(in.a); emit(P_FN, 0, F_COSH); break;
+        case I_EXP: expr(in.a); emit(P_FN, same_for_all_u(in.a), F_EXP); break;
+        case I_LOG: expr(in.a); emit(P_FN, same_for_all_u(in.a), F_LOG); break;
+        case I_SIN: expr(in.a); emit(P_FN, same_for_all_u(in.a), F_SIN); break;
+        case I_COS: expr(in.a); emit(P_FN, same_for_all_u(in.a), F_COS); break;
+        case I_TANH: expr(in.a); emit(P_FN, same_for_all_u(in.a), F_TANH); break;
+        case I_SINH: expr(in.a); emit(P_FN, same_for_all_u(in.a), F_SINH); break;
+        case I_COSH: expr(in.a); emit(P_FN, same_for_all_u(in.a), F_COSH); break;
         case I_SQR: expr(in.a); emit(P_SQR); break;
         case I_POWI:
             expr(in.a);
-            if (in.ipow == 3) emit(P_CUBE); else emit(P_FN, 0, F_POWI, in.ipow);
+            if (in.ipow == 3) emit(P_CUBE); else emit(P_FN, same_for_all_u(in.a), F_POWI, in.ipow);
             break;
         case I_MULC: expr(in.a); emit(P_MULC, 0, 0, fbits(in.imm)); break;
         case I_ADDC: expr(in.a); emit(P_ADDC, 0, 0, fbits(in.imm)); break;
@@ -401,12 +404,14 @@ struct Emitter {
             if ((int)loops.size() >= TADP_MAX_LOOPS) throw Unsupported("too many loops in one kernel");
             loops.push_back(L);
             int id = (int)loops.size() - 1;
+            const bool over_elements = in.var == g.unroll_var;   // the element variable runs over this sum
             emit(P_ZERO, 0, 0, 0, +1);
-            int begin = emit(P_SLOOP, id, 0, 0, 0, in.var);
+            int begin = emit(over_elements ? P_USLOOP : P_SLOOP, id, 0, 0, 0, in.var);
             temps_of_sum(i);
             expr(in.a);
             emit(P_SUMADD, 0, 0, 0, -1);
-            int end = emit(P_SEND, id, 0, begin + 1, 0, in.var);
+            int end = emit(over_elements ? P_USEND : P_SEND, id, 0, begin + 1, 0, in.var);
+            if (over_elements) emit(P_HSUM);
             code[begin].imm = end + 1;
             break;
         }
@@ -584,12 +589,47 @@ void finish_stats(Gen &g, Kernel &k, bool backward, int64_t outputs, int64_t ter
     s.alg_bytes += 4.0 * outputs;
 }
 
+// Element variable B: a second loop variable spread over further elements of each thread.
+// It pays when some load is strided across the lanes (every lane touches its own 32-byte
+// sector) but contiguous along B: the thread then reads its own row with 128-bit loads and
+// uses the sector in full; a strided load that does not depend on B is fetched once for all its
+// elements.  Candidates: outer variables (a tile of gradient elements per thread) and bound
+// sums (several summands per trip).
+void choose_element_variable(Gen &g)
+{
+    g.unroll_var = -1;
+    if (g.p.opt.debug_bounds) return;            // debug plans use the narrow kernels
+    const int A = g.lane_var;
+    double best = 0;
+    for (int v = 0; v < (int)g.vars.size(); ++v) {
+        if (v == A || g.vars[v].ext < 4 || g.vars[v].kind == 1) continue;
+        if (g.vars[v].kind == 2 && (g.vars[v].sum_inst < 0 || !g.inst[g.vars[v].sum_inst].uses)) continue;
+        double score = 0;
+        bool fixes_strided = false;
+        for (const Inst &in : g.inst) {
+            if (!in.uses || in.op != I_LOAD) continue;
+            const TadpLoad &L = g.loads[in.load];
+            const int64_t ca = std::llabs((int64_t)L.coef[A]), cb = std::llabs((int64_t)L.coef[v]);
+            // weight: how often the load runs (loads inside bound sums and inner loops dominate)
+            double w = 1;
+            for (int x = g.n_outer; x < (int)g.vars.size(); ++x)
+                if (x != v && (in.deps & (1u << x))) w *= (double)g.vars[x].ext;
+            if (cb == 1 && ca >= 8) { score += 4 * w; fixes_strided = true; }          // strided load becomes row reads
+            else if (cb == 0 && ca >= 8) { score += 3 * w; fixes_strided = true; }     // strided load shared by all u
+            else if (cb == 0) score += w;
+            else if (cb == 1 && ca == 0) score += 0.5 * w;
+        }
+        if (fixes_strided && score > best) { best = score; g.unroll_var = v; }
+    }
+}
+
 // shared tail: choose temps, emit, fill the program
 void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<TadpRow>> &lower,
                  const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards)
 {
     TadpProgram &prog = k.prog;
     place(g);
+    choose_element_variable(g);
     // temporaries: shared values and values hoisted out of the loop that consumes them
     std::vector<bool> hoisted(g.inst.size(), false);
     auto effective_level = [&](int i) { return i == root ? g.kappa : g.inst[i].zlevel; };
@@ -651,7 +691,7 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
         for (const TadpRow &r : upper[zl]) rows.push_back(r);
         L.depends_on_lane = 0;
         for (int r = L.lower0; r < L.upper0 + L.n_upper; ++r)
-            if (rows[r].coef[g.lane_var]) L.depends_on_lane = 1;
+            if (rows[r].coef[g.lane_var] || (g.unroll_var >= 0 && rows[r].coef[g.unroll_var])) L.depends_on_lane = 1;
     }
     prog.guard0 = (int32_t)rows.size(); prog.n_guards = (int32_t)guards.size();
     for (const TadpRow &r : guards) rows.push_back(r);
@@ -666,6 +706,7 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     prog.rel_var = -1;
     for (int li = (int)em.loops.size() - 1; li >= 0; --li) {
         TadpLoop &L = em.loops[li];
+        if (g.unroll_var >= 0) break;
         if (g.vars[L.var].kind != 1 || L.is_lane || !L.depends_on_lane) continue;
         if (g.vars[L.var].ext > 16) continue;
         // no other loop's bounds may read this variable through a warp-uniform path
@@ -680,6 +721,7 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     for (int i = 0; i < prog.n_loads; ++i) {
         prog.loads[i].lane_step = to_i32(32 * (int64_t)prog.loads[i].coef[g.lane_var]);
         prog.loads[i].rel_step = prog.rel_var >= 0 ? prog.loads[i].coef[prog.rel_var] : 0;
+        prog.loads[i].unroll_step = g.unroll_var >= 0 ? prog.loads[i].coef[g.unroll_var] : 0;
     }
     prog.n_loops = (int32_t)em.loops.size();
     std::copy(em.loops.begin(), em.loops.end(), prog.loops);
@@ -687,48 +729,65 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     std::copy(rows.begin(), rows.end(), prog.rows);
     prog.n_outer = g.n_outer;
     prog.lane_var = g.lane_var;
+    prog.unroll_var = g.unroll_var;
+    prog.unroll_kind = g.unroll_var < 0 ? 0 : g.unroll_var < g.n_outer ? 1 : 3;
     // Vector width and summation split.  Wide vectors amortise the interpreter's dispatch cost,
     // but only while enough warps remain to fill the GPU; when even the narrowest shape leaves
     // too few, the outermost kernel-coordinate loop is divided among several warps per output,
     // each writing a partial sum that a second launch adds up in a fixed order.
     const int64_t lane_ext = g.vars[g.lane_var].ext;
     const double target_warps = 148.0 * 16.0 * 2.0;
-    auto items_for = [&](int T) {
+    const int64_t uext = g.unroll_var >= 0 ? g.vars[g.unroll_var].ext : 1;
+    const bool shallow = em.max_depth <= TADP_WIDE_DEPTH;
+    const bool debug = g.p.opt.debug_bounds != 0;
+    // candidate shapes (TA, UB), widest first; 16 values per thread need the shallow stack
+    struct Shape { int ta, ub; };
+    std::vector<Shape> shapes;
+    if (g.unroll_var >= 0 && !debug) {
+        if (uext >= 8 && shallow && lane_ext >= 64) shapes.push_back({2, 8});     // measured best on the intro expression
+        if (uext >= 16 && shallow) shapes.push_back({1, 16});
+        if (uext >= 8) shapes.push_back({1, 8});
+        shapes.push_back({1, 4});
+    } else {
+        for (int T : {16, 8, 4, 2, 1}) {
+            if (T == 16 && !shallow) continue;
+            if (debug && T > 4) continue;
+            if (T > 1 && lane_ext < 32 * T) continue;
+            shapes.push_back({T, 1});
+        }
+    }
+    auto items_for = [&](const Shape &sh) {
         double n = 1;
         for (int v = 0; v < g.n_outer; ++v) {
             double e = (double)prog.outer_ext[v];
-            if (v == g.lane_var) e = std::ceil(e / (32.0 * T));
+            if (v == g.lane_var) e = std::ceil(e / (32.0 * sh.ta));
+            else if (v == g.unroll_var) e = std::ceil(e / (double)sh.ub);
             n *= e;
         }
         return n;
     };
-    const bool debug = g.p.opt.debug_bounds != 0;
-    auto allowed = [&](int T) {
-        if (T == 16 && em.max_depth > TADP_WIDE_DEPTH) return false;
-        if (debug && T > 4) return false;
-        return T == 1 || lane_ext >= 32 * T;
-    };
     prog.zsplit = 1;
-    k.vec = 1;
+    Shape pick = shapes.back();
     if (g.kappa >= 1) {
-        // a summation that can be split: take the widest vector and split to fill the GPU
-        for (int T : {16, 8, 4, 2, 1}) if (allowed(T)) { k.vec = T; break; }
+        // a summation that can be split: take the widest shape and split to fill the GPU
+        pick = shapes.front();
         // splitting costs a pass over zsplit x outputs: only for small gradients that starve the GPU
-        if (items_for(k.vec) < target_warps / 2 && prog.out_limit <= (1 << 22)) {
+        if (items_for(pick) < target_warps / 2 && prog.out_limit <= (1 << 22)) {
             TadpLoop &L0 = prog.loops[em.code[zbegin[0]].a];
-            const int64_t ext0 = std::max<int64_t>(1, g.vars[L0.var].ext / (L0.is_lane ? 32 * k.vec : 1));
-            int64_t S = (int64_t)std::ceil(target_warps / items_for(k.vec));
+            const int64_t ext0 = std::max<int64_t>(1, g.vars[L0.var].ext / (L0.is_lane ? 32 * pick.ta : 1));
+            int64_t S = (int64_t)std::ceil(target_warps / items_for(pick));
             S = std::min<int64_t>(std::min<int64_t>(S, ext0), 4096);
             while (S > 1 && S * (int64_t)prog.out_limit > (int64_t(1) << 25)) S /= 2;   // <= 128 MB of partial sums
             if (S >= 2) { prog.zsplit = (int32_t)S; L0.is_split = 1; }
         }
     } else {
-        // element-wise kernel: the widest vector that still leaves enough warps
-        for (int T : {16, 8, 4, 2, 1}) if (allowed(T) && (items_for(T) >= target_warps || T == 1)) { k.vec = T; break; }
+        // element-wise kernel: the widest shape that still leaves enough warps
+        for (const Shape &sh : shapes) if (items_for(sh) >= target_warps) { pick = sh; break; }
     }
+    k.vec = pick.ta; k.vec_u = pick.ub;
     char head[256];
-    std::snprintf(head, sizeof head, "; vars=%zu outer=%d kappa=%d lane_var=%d vec=%d zsplit=%d temps=%d max_depth=%d loads=%d rows=%d guards=%d\n",
-                  g.vars.size(), g.n_outer, g.kappa, g.lane_var, k.vec, prog.zsplit, n_temps, em.max_depth, prog.n_loads, prog.n_rows, prog.n_guards);
+    std::snprintf(head, sizeof head, "; vars=%zu outer=%d kappa=%d lane_var=%d unroll_var=%d vec=%dx%d zsplit=%d temps=%d max_depth=%d loads=%d rows=%d guards=%d\n",
+                  g.vars.size(), g.n_outer, g.kappa, g.lane_var, g.unroll_var, k.vec, k.vec_u, prog.zsplit, n_temps, em.max_depth, prog.n_loads, prog.n_rows, prog.n_guards);
     k.listing = head + em.listing;
 }
 

@@ -63,7 +63,8 @@ struct Kernel {
     TadpProgram prog;
     int out_arg = -1;          // -1: forward (writes f); else the argument whose gradient it writes
     int access = -1;
-    int vec = 4;               // vector elements per lane the launcher instantiates
+    int vec = 4;               // elements per thread along the lane variable (TA)
+    int vec_u = 1;             // elements per thread along the element variable (UB)
     std::vector<int> stages_used;   // backward: staged adjoints it reads (indices into tad_plan::stages)
     KernelStats stats;
     std::string listing;

@@ -30,9 +30,11 @@ enum TadpOp : int {
     P_LDT,        // temp[a]
     // replace the top (k = 1..7)
     P_NEG, P_SQR, P_CUBE,
+    P_HSUM,       // top[t][u] <- sum over u' of top[t][u'] (closes a sum loop that runs over the element variable)
     P_MULC, P_ADDC,               // top <- top op imm(float)
     P_LDADD, P_LDMUL,             // top <- top op load(loads[a])
-    P_FN,         // top <- function b of top: TadpFn; P_FN_POWI takes its exponent from imm
+    P_FN,         // top <- function b of top: TadpFn; F_POWI takes its exponent from imm; a != 0: the value is
+                  // the same for every u, evaluate it once per lane-variable element
     P_STT,        // temp[a] <- top ; pop
     P_ACC,        // acc += active ? top : 0 ; pop
     // two operands (k = 2..7): second <- second op top ; pop
@@ -44,6 +46,8 @@ enum TadpOp : int {
     // loop control (k = loop variable)
     P_SLOOP,      // bound sum loop begin: loops[a]; jumps to imm when the range is empty
     P_SEND,       // bound sum loop end: increments, jumps back to imm while in range
+    P_USLOOP,     // the same for the sum whose index is the element variable: steps by UB, masks the tail
+    P_USEND,
     P_ZLOOP,      // kernel-coordinate loop begin: loops[a]; computes the range from its bound rows
     P_ZEND,       // kernel-coordinate loop end
     P_NUM_OPS
@@ -64,7 +68,8 @@ struct alignas(16) TadpLoad {         // 64 bytes, 16-byte aligned: 128-bit cons
     int32_t limit;                     // elements in the tensor (debug bounds)
     int32_t lane_step;                 // 32 * coef[lane variable]: offset step between vector elements
     int32_t rel_step;                  // coef[variable of the relative loop]
-    int32_t pad[3];
+    int32_t unroll_step;               // coef[element variable]: offset step between elements u and u+1
+    int32_t pad[2];
 };
 
 struct TadpRow {                       // value = (c0 + sum_v coef[v] * var[v]) / den, den > 0
@@ -88,7 +93,9 @@ struct TadpLoop {
 struct alignas(16) TadpProgram {
     int32_t n_code, n_loads, n_loops, n_rows;
     int32_t n_outer;                   // outer variables 0 .. n_outer-1 (decoded from the work item)
-    int32_t lane_var;                  // variable spread over lanes; < n_outer: distinct outputs per lane
+    int32_t lane_var;                  // variable A spread over lanes (and elements t); < n_outer: distinct outputs per lane
+    int32_t unroll_var;                // variable B spread over the elements u of each thread, or -1
+    int32_t unroll_kind;               // 0 none, 1 outer variable (distinct outputs per u), 3 bound sum
     int32_t outer_lo[TADP_MAX_VARS];   // inclusive box of the outer variables
     int32_t outer_ext[TADP_MAX_VARS];  // extents (>= 1)
     int32_t n_guards, guard0;          // rows[guard0 ..): element is live iff every row value <= 0 (den = 1)

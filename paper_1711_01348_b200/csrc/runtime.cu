@@ -19,17 +19,21 @@ namespace {
 using namespace tadvm;
 
 // One warp per work item, grid-stride over the items.  A work item fixes every outer variable
-// except the lane variable, which the warp covers 32 * T elements at a time.
-template <int T, bool DEBUG, bool REL>
+// except the lane variable A, which the warp covers 32 * TA values at a time, and the element
+// variable B when that is an outer variable, which it covers UB values at a time.
+template <int TA, int UB, bool DEBUG, bool REL>
 __global__ void __launch_bounds__(WARPS_PER_BLOCK * 32, 2)
 tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ TadpPointers ptrs, unsigned n_items)
 {
+    constexpr int E = TA * UB;
     const unsigned lane = threadIdx.x & 31u;
     const unsigned warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const unsigned n_warps = (gridDim.x * blockDim.x) >> 5;
     const int lane_var = P.lane_var;
+    const int unroll_var = P.unroll_var;
     const bool lane_outer = lane_var < P.n_outer;
-    Vm<T> m;
+    const bool unroll_outer = UB > 1 && P.unroll_kind == 1;
+    Vm<TA, UB> m;
     const unsigned zsplit = P.zsplit > 1 ? (unsigned)P.zsplit : 1u;
     for (unsigned witem = warp; witem < n_items; witem += n_warps) {
         // warps witem = item * zsplit + s share the outputs of `item`
@@ -39,66 +43,82 @@ tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ Tad
         unsigned rem = item;
 #pragma unroll
         for (int k = 0; k < TADP_MAX_VARS; ++k) m.var[k] = 0;
-        unsigned mask0 = (1u << T) - 1u;
+        unsigned first_a = 0, ext_a = 0xffffffffu, first_b = 0, ext_b = 0xffffffffu;
 #pragma unroll
         for (int v = TADP_MAX_VARS - 1; v >= 0; --v) {
             if (v < P.n_outer) {
                 const unsigned ext = (unsigned)P.outer_ext[v];
                 if (v == lane_var) {
-                    const unsigned chunks = (ext + 32u * T - 1u) / (32u * T);
+                    const unsigned chunks = (ext + 32u * TA - 1u) / (32u * TA);
                     const unsigned c = rem % chunks; rem /= chunks;
-                    const unsigned first = c * 32u * T + lane;
-                    m.var[v] = P.outer_lo[v] + (int)first;
-                    mask0 = 0;
-#pragma unroll
-                    for (int t = 0; t < T; ++t) if (first + 32u * t < ext) mask0 |= 1u << t;
+                    first_a = c * 32u * TA + lane; ext_a = ext;
+                    m.var[v] = P.outer_lo[v] + (int)first_a;
+                } else if (unroll_outer && v == unroll_var) {
+                    const unsigned chunks = (ext + UB - 1u) / UB;
+                    const unsigned c = rem % chunks; rem /= chunks;
+                    first_b = c * UB; ext_b = ext;
+                    m.var[v] = P.outer_lo[v] + (int)first_b;
                 } else {
                     const unsigned c = rem % ext; rem /= ext;
                     m.var[v] = P.outer_lo[v] + (int)c;
                 }
             }
         }
+        unsigned mask0 = 0;
+#pragma unroll
+        for (int e = 0; e < E; ++e)
+            if (first_a + 32u * (e / UB) < ext_a && first_b + (unsigned)(e % UB) < ext_b) mask0 |= 1u << e;
         const unsigned in_range = mask0;
         // guards: rows over the outer variables that must be <= 0 for Gamma to be non-empty
         for (int r = 0; r < P.n_guards; ++r) {
             const TadpRow &R = P.rows[P.guard0 + r];
             const int nmr = row_num(R, m.var);
-            const int step = lane_outer ? R.coef[lane_var] * 32 : 0;
+            const int sa = lane_outer ? R.coef[lane_var] * 32 : 0;
+            const int sb = unroll_outer ? R.coef[unroll_var] : 0;
 #pragma unroll
-            for (int t = 0; t < T; ++t) if (nmr + t * step > 0) mask0 &= ~(1u << t);
+            for (int e = 0; e < E; ++e) if (nmr + (e / UB) * sa + (e % UB) * sb > 0) mask0 &= ~(1u << e);
         }
         unsigned live = 0;
-        run_item<T, DEBUG, REL>(P, ptrs, m, mask0, split, live);
-        // output
+        run_item<TA, UB, DEBUG, REL>(P, ptrs, m, mask0, split, live);
+
+        // ---- output: distinct elements along t when A is an outer variable, along u when B is ----
+        const int n_u = unroll_outer ? UB : 1;
+        unsigned off = (unsigned)P.out_base;
+#pragma unroll
+        for (int k = 0; k < TADP_MAX_VARS; ++k) if (k < P.n_outer) off += (unsigned)P.out_coef[k] * (unsigned)m.var[k];
+        const unsigned step_a = lane_outer ? (unsigned)P.out_coef[lane_var] * 32u : 0u;
+        const unsigned step_b = unroll_outer ? (unsigned)P.out_coef[unroll_var] : 0u;
+        float *dst = zsplit > 1 ? ptrs.part + (size_t)split * (unsigned)P.out_limit : ptrs.out;
+        const bool accumulate = zsplit > 1 ? false : P.accumulate != 0;
+        const bool only_live = zsplit > 1 ? false : P.write_only_live != 0;
         if (lane_outer) {
-            unsigned off = (unsigned)P.out_base;
 #pragma unroll
-            for (int k = 0; k < TADP_MAX_VARS; ++k) off += (unsigned)P.out_coef[k] * (unsigned)m.var[k];
-            const unsigned step = (unsigned)P.out_coef[lane_var] * 32u;
-#pragma unroll
-            for (int t = 0; t < T; ++t) {
-                if (!((in_range >> t) & 1u)) continue;
-                if (P.write_only_live && !((live >> t) & 1u)) continue;
-                const unsigned idx = off + (unsigned)t * step;
+            for (int e = 0; e < E; ++e) {
+                if ((e % UB) >= n_u) continue;
+                if (!((in_range >> e) & 1u)) continue;
+                if (only_live && !((live >> e) & 1u)) continue;
+                const unsigned idx = off + (unsigned)(e / UB) * step_a + (unsigned)(e % UB) * step_b;
                 if (DEBUG && idx >= (unsigned)P.out_limit) { if (ptrs.debug) atomicCAS(ptrs.debug, 0, 0x20000); continue; }
-                if (zsplit > 1) ptrs.part[(size_t)split * (unsigned)P.out_limit + idx] = m.acc[t];
-                else ptrs.out[idx] = P.accumulate ? ptrs.out[idx] + m.acc[t] : m.acc[t];
+                dst[idx] = accumulate ? dst[idx] + m.acc[e] : m.acc[e];
             }
         } else {
-            // the lane variable is a kernel coordinate: one output per warp, fixed-order tree reduction
-            unsigned off = (unsigned)P.out_base;
+            // the lane variable is a kernel coordinate: fixed-order tree reduction over t and the lanes
 #pragma unroll
-            for (int k = 0; k < TADP_MAX_VARS; ++k) if (k < P.n_outer) off += (unsigned)P.out_coef[k] * (unsigned)m.var[k];
-            float total = 0.f;
+            for (int u = 0; u < UB; ++u) {
+                if (u >= n_u) continue;
+                float total = 0.f;
+                unsigned lv = 0;
 #pragma unroll
-            for (int t = 0; t < T; ++t) total += m.acc[t];
+                for (int t = 0; t < TA; ++t) { total += m.acc[t * UB + u]; lv |= (live >> (t * UB + u)) & 1u; }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
-            const unsigned any_live = __ballot_sync(0xffffffffu, live != 0);
-            if (lane == 0 && !(P.write_only_live && !any_live)) {
-                if (DEBUG && off >= (unsigned)P.out_limit) { if (ptrs.debug) atomicCAS(ptrs.debug, 0, 0x20000); }
-                else if (zsplit > 1) ptrs.part[(size_t)split * (unsigned)P.out_limit + off] = total;
-                else ptrs.out[off] = P.accumulate ? ptrs.out[off] + total : total;
+                for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+                const unsigned any_live = __ballot_sync(0xffffffffu, lv != 0);
+                const bool inside = first_b + (unsigned)u < ext_b;
+                if (lane == 0 && inside && !(only_live && !any_live)) {
+                    const unsigned idx = off + (unsigned)u * step_b;
+                    if (DEBUG && idx >= (unsigned)P.out_limit) { if (ptrs.debug) atomicCAS(ptrs.debug, 0, 0x20000); }
+                    else dst[idx] = accumulate ? dst[idx] + total : total;
+                }
             }
         }
     }
@@ -129,24 +149,26 @@ int sm_count()
     return n;
 }
 
-unsigned long long item_count(const TadpProgram &P, int T)
+unsigned long long item_count(const TadpProgram &P, int ta, int ub)
 {
     unsigned long long n = 1;
     for (int v = 0; v < P.n_outer; ++v) {
         unsigned long long e = (unsigned long long)P.outer_ext[v];
-        if (v == P.lane_var) e = (e + 32ull * T - 1) / (32ull * T);
+        if (v == P.lane_var) e = (e + 32ull * ta - 1) / (32ull * ta);
+        else if (ub > 1 && P.unroll_kind == 1 && v == P.unroll_var) e = (e + ub - 1) / ub;
         n *= e;
     }
     return n;
 }
 
-template <int T>
+// Builds of the interpreter per vector shape: plain, with the relative-loop support and (narrow
+// shapes only) with bounds checks.
+template <int TA, int UB>
 void launch_t(const tad::Kernel &k, const TadpPointers &ptrs, bool debug, unsigned items, unsigned blocks, cudaStream_t stream)
 {
-    // three builds of the interpreter per vector width: plain, with the relative-loop support, with bounds checks
-    if (debug) { if constexpr (T <= 4) tad_vm_kernel<T, true, true><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items); }
-    else if (k.prog.rel_var >= 0) tad_vm_kernel<T, false, true><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items);
-    else tad_vm_kernel<T, false, false><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items);
+    if (debug) { if constexpr (TA <= 4 && UB == 1) tad_vm_kernel<TA, UB, true, true><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items); }
+    else if (k.prog.rel_var >= 0) { if constexpr (UB == 1) tad_vm_kernel<TA, UB, false, true><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items); }
+    else tad_vm_kernel<TA, UB, false, false><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items);
 }
 
 tad_status zero_fill(float *out, int64_t n, cudaStream_t stream);
@@ -162,19 +184,24 @@ tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStrea
             if (st != TAD_OK) return st;
         }
     }
-    const unsigned long long items64 = item_count(k.prog, k.vec) * (unsigned long long)zsplit;
+    const unsigned long long items64 = item_count(k.prog, k.vec, k.vec_u) * (unsigned long long)zsplit;
     if (items64 == 0) return TAD_OK;
     if (items64 >= (1ull << 32)) { tad::set_error("too many work items"); return TAD_ERR_UNSUPPORTED; }
     const unsigned items = (unsigned)items64;
     const unsigned blocks_needed = (items + WARPS_PER_BLOCK - 1) / WARPS_PER_BLOCK;
     const unsigned max_blocks = (unsigned)sm_count() * 16u;
     const unsigned blocks = std::min(blocks_needed, max_blocks);
-    switch (k.vec) {
-    case 1: launch_t<1>(k, ptrs, debug, items, blocks, stream); break;
-    case 2: launch_t<2>(k, ptrs, debug, items, blocks, stream); break;
-    case 8: launch_t<8>(k, ptrs, debug, items, blocks, stream); break;
-    case 16: launch_t<16>(k, ptrs, debug, items, blocks, stream); break;
-    default: launch_t<4>(k, ptrs, debug, items, blocks, stream); break;
+    switch (k.vec * 100 + k.vec_u) {
+    case 101: launch_t<1, 1>(k, ptrs, debug, items, blocks, stream); break;
+    case 201: launch_t<2, 1>(k, ptrs, debug, items, blocks, stream); break;
+    case 401: launch_t<4, 1>(k, ptrs, debug, items, blocks, stream); break;
+    case 801: launch_t<8, 1>(k, ptrs, debug, items, blocks, stream); break;
+    case 1601: launch_t<16, 1>(k, ptrs, debug, items, blocks, stream); break;
+    case 104: launch_t<1, 4>(k, ptrs, debug, items, blocks, stream); break;
+    case 108: launch_t<1, 8>(k, ptrs, debug, items, blocks, stream); break;
+    case 208: launch_t<2, 8>(k, ptrs, debug, items, blocks, stream); break;
+    case 116: launch_t<1, 16>(k, ptrs, debug, items, blocks, stream); break;
+    default: tad::set_error("internal: no kernel for this vector shape"); return TAD_ERR_UNSUPPORTED;
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { tad::set_error(std::string("kernel launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }

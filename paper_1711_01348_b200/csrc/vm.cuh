@@ -59,17 +59,19 @@ __device__ __noinline__ float apply_fn(int fn, float x, int n)
 // Per vector width: NTR temporaries kept in registers (the rest spill to local memory) and the
 // usable operand stack depth.  Wide vectors amortise the dispatch cost over more elements and
 // pay for it with a shallower stack; the host picks the widest variant a program fits.
-template <int T>
+template <int TA, int UB>
 struct VmCfg {
-    static constexpr int NTR = T >= 16 ? 0 : T >= 8 ? 2 : TADP_NUM_TEMPS;
-    static constexpr int DEPTH = T >= 16 ? TADP_WIDE_DEPTH : STACK;
+    static constexpr int E = TA * UB;           // values per thread and operand
+    static constexpr int NTR = E >= 16 ? 0 : E >= 8 ? 2 : TADP_NUM_TEMPS;
+    static constexpr int DEPTH = E >= 16 ? TADP_WIDE_DEPTH : STACK;
 };
 
-template <int T>
+template <int TA, int UB>
 struct Vm {
-    float s[VmCfg<T>::DEPTH][T];
-    float tmp[VmCfg<T>::NTR > 0 ? VmCfg<T>::NTR : 1][T];
-    float acc[T];
+    static constexpr int E = TA * UB;
+    float s[VmCfg<TA, UB>::DEPTH][E];
+    float tmp[VmCfg<TA, UB>::NTR > 0 ? VmCfg<TA, UB>::NTR : 1][E];
+    float acc[E];
     int var[TADP_MAX_VARS];
 };
 
@@ -110,14 +112,17 @@ __device__ __forceinline__ unsigned load_offset(const TadpLoad &L, const int (&v
 #define TADV_V8(M, OP) M(OP, 0) M(OP, 1) M(OP, 2) M(OP, 3) M(OP, 4) M(OP, 5) M(OP, 6) M(OP, 7)
 #define TADV_H(OP, K) ((OP) * 8 + (K))
 // a handler exists only if the depths it touches fit the variant's stack
-#define TADV_CASE(OP, D, TOP) case TADV_H(OP, D): if constexpr ((TOP) <= VmCfg<T>::DEPTH)
+#define TADV_CASE(OP, D, TOP) case TADV_H(OP, D): if constexpr ((TOP) <= VmCfg<TA, UB>::DEPTH)
 
 // Runs the program of one work item.  mask0: which vector elements of this lane are live at
 // the outermost level.  Returns in live_out the elements that accumulated at least one term.
-template <int T, bool DEBUG, bool REL>
-__device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointers &ptrs, Vm<T> &m,
+template <int TA, int UB, bool DEBUG, bool REL>
+__device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointers &ptrs, Vm<TA, UB> &m,
                                          unsigned mask0, int split, unsigned &live_out)
 {
+    constexpr int T = TA * UB;             // element e = t * UB + u: t along the lane variable, u along the element variable
+    const int unroll_var = P.unroll_var;
+    unsigned sum_parent = mask0;           // mask outside the sum loop that runs over the element variable
     const int lane_var = P.lane_var;
     unsigned cur = mask0;                 // activity mask of the vector elements at the current loop level
     unsigned mstack[TADP_MAX_ZLOOPS + 1];  // activity mask per loop level
@@ -130,7 +135,7 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
     __shared__ int zrel_s[REL ? T : 1][WARPS_PER_BLOCK * 32];
 #define zrel(t) zrel_s[t][threadIdx.x]
     const int rel_var = REL ? P.rel_var : -1;
-    constexpr int NTR = VmCfg<T>::NTR;
+    constexpr int NTR = VmCfg<TA, UB>::NTR;
     float spill[TADP_MAX_SPILL + TADP_NUM_TEMPS - NTR][T];
 #pragma unroll
     for (int t = 0; t < T; ++t) m.acc[t] = 0.f;
@@ -156,15 +161,39 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
             const TadpLoad &L = P.loads[a]; \
             const unsigned off = load_offset(L, m.var); \
             const unsigned lc = (unsigned)L.lane_step; \
+            const unsigned uc = UB > 1 ? (unsigned)L.unroll_step : 0u; \
             const float *base = ptrs.in[L.ptr]; \
-            if (lc == 0 && (!REL || L.rel_step == 0) && !DEBUG) { \
-                /* the same element for every vector element of this lane: one load */ \
+            if (lc == 0 && uc == 0 && (!REL || L.rel_step == 0) && !DEBUG) { \
+                /* the same element for every value of this lane: one load */ \
                 const float v = cur ? __ldg(base + off) : 0.f; \
                 _Pragma("unroll") for (int t = 0; t < T; ++t) { DST_EXPR; } \
+            } else if (UB > 1 && uc == 0 && (!REL || L.rel_step == 0) && !DEBUG) { \
+                /* constant along the element variable: one load per lane-variable element */ \
+                _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { \
+                    const unsigned mm = (cur >> (ta * UB)) & ((1u << UB) - 1u); \
+                    const float v = mm ? __ldg(base + off + (unsigned)ta * lc) : 0.f; \
+                    _Pragma("unroll") for (int u = 0; u < UB; ++u) { const int t = ta * UB + u; DST_EXPR; } \
+                } \
+            } else if (UB % 4 == 0 && uc == 1 && (!REL || L.rel_step == 0) && !DEBUG && (reinterpret_cast<uintptr_t>(base) & 15u) == 0) { \
+                /* contiguous along the element variable: 128-bit loads of this lane's own row */ \
+                _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { \
+                    const unsigned o = off + (unsigned)ta * lc; \
+                    _Pragma("unroll") for (int g4 = 0; g4 < UB / 4; ++g4) { \
+                        const unsigned mm = (cur >> (ta * UB + 4 * g4)) & 0xfu; \
+                        float q[4]; \
+                        if (mm == 0xfu && ((o + 4u * g4) & 3u) == 0) { \
+                            const float4 f4 = __ldg(reinterpret_cast<const float4 *>(base + o + 4 * g4)); \
+                            q[0] = f4.x; q[1] = f4.y; q[2] = f4.z; q[3] = f4.w; \
+                        } else { \
+                            _Pragma("unroll") for (int i = 0; i < 4; ++i) q[i] = ((mm >> i) & 1u) ? __ldg(base + o + 4 * g4 + i) : 0.f; \
+                        } \
+                        _Pragma("unroll") for (int i = 0; i < 4; ++i) { const int t = ta * UB + 4 * g4 + i; const float v = q[i]; DST_EXPR; } \
+                    } \
+                } \
             } else { \
                 const unsigned rs = REL ? (unsigned)L.rel_step : 0u; \
                 _Pragma("unroll") for (int t = 0; t < T; ++t) { \
-                    const unsigned idx = off + (unsigned)t * lc + (REL && rs ? rs * (unsigned)zrel(t) : 0u); \
+                    const unsigned idx = off + (unsigned)(t / UB) * lc + (unsigned)(t % UB) * uc + (REL && rs ? rs * (unsigned)zrel(t) : 0u); \
                     bool ok = (cur >> t) & 1u; \
                     if (DEBUG && ok && idx >= (unsigned)L.limit) { ok = false; if (ptrs.debug) atomicCAS(ptrs.debug, 0, 0x10000 + a); } \
                     const float v = ok ? __ldg(base + idx) : 0.f; \
@@ -189,13 +218,32 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
         TADV_D1(TADV_MULC, P_MULC)
 #define TADV_ADDC(OP, D) TADV_CASE(OP, D, D) { const float c = __int_as_float(imm); TADV_UNARY(D, op_add(x, c)) }
         TADV_D1(TADV_ADDC, P_ADDC)
-#define TADV_FN(OP, D) TADV_CASE(OP, D, D) { TADV_UNARY(D, apply_fn(fn_code, x, imm)) }
+#define TADV_FN(OP, D) TADV_CASE(OP, D, D) { \
+            if (UB > 1 && a) { \
+                _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { \
+                    const float r = apply_fn(fn_code, m.s[D - 1][ta * UB], imm); \
+                    _Pragma("unroll") for (int u = 0; u < UB; ++u) m.s[D - 1][ta * UB + u] = r; \
+                } \
+                break; \
+            } \
+            TADV_UNARY(D, apply_fn(fn_code, x, imm)) }
         TADV_D1(TADV_FN, P_FN)
 
 #define TADV_BINARY(D, EXPR) { _Pragma("unroll") for (int t = 0; t < T; ++t) { const float x = m.s[D - 2][t], y = m.s[D - 1][t]; m.s[D - 2][t] = (EXPR); } } break;
 #define TADV_ADD(OP, D) TADV_CASE(OP, D, D) TADV_BINARY(D, op_add(x, y))
         TADV_D2(TADV_ADD, P_ADD)
-        TADV_D2(TADV_ADD, P_SUMADD)
+        // summand into the accumulator of a value sum; elements masked off (the tail of a sum that
+        // runs over the element variable) leave it unchanged
+#define TADV_SUMADD(OP, D) TADV_CASE(OP, D, D) { _Pragma("unroll") for (int t = 0; t < T; ++t) if (UB == 1 || ((cur >> t) & 1u)) m.s[D - 2][t] = op_add(m.s[D - 2][t], m.s[D - 1][t]); } break;
+        TADV_D2(TADV_SUMADD, P_SUMADD)
+        // closes a sum over the element variable: add up the UB partial sums, replicate the result
+#define TADV_HSUM(OP, D) TADV_CASE(OP, D, D) { \
+            _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { \
+                float sum = m.s[D - 1][ta * UB]; \
+                _Pragma("unroll") for (int u = 1; u < UB; ++u) sum = op_add(sum, m.s[D - 1][ta * UB + u]); \
+                _Pragma("unroll") for (int u = 0; u < UB; ++u) m.s[D - 1][ta * UB + u] = op_mov(sum); \
+            } } break;
+        TADV_D1(TADV_HSUM, P_HSUM)
 #define TADV_SUB(OP, D) TADV_CASE(OP, D, D) TADV_BINARY(D, op_sub(x, y))
         TADV_D2(TADV_SUB, P_SUB)
 #define TADV_MUL(OP, D) TADV_CASE(OP, D, D) TADV_BINARY(D, op_mul(x, y))
@@ -232,6 +280,26 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
         TADV_V8(TADV_SLOOP, P_SLOOP)
 #define TADV_SEND(OP, V) case TADV_H(OP, V): { const int k = m.var[V] + 1; if (k <= P.loops[a].const_hi) { m.var[V] = k; pc = imm; } } break;
         TADV_V8(TADV_SEND, P_SEND)
+        // the sum whose index is the element variable: UB summands per trip, tail masked
+#define TADV_USLOOP(OP, V) case TADV_H(OP, V): { \
+            const TadpLoop &L = P.loops[a]; \
+            if (L.const_lo > L.const_hi) pc = imm; \
+            else { \
+                m.var[V] = L.const_lo; sum_parent = cur; \
+                unsigned mk = 0; \
+                _Pragma("unroll") for (int t = 0; t < T; ++t) if (L.const_lo + (t % UB) <= L.const_hi) mk |= 1u << t; \
+                cur = sum_parent & mk; \
+            } } break;
+        TADV_V8(TADV_USLOOP, P_USLOOP)
+#define TADV_USEND(OP, V) case TADV_H(OP, V): { \
+            const int k = m.var[V] + UB; const int hi = P.loops[a].const_hi; \
+            if (k <= hi) { \
+                m.var[V] = k; \
+                unsigned mk = 0; \
+                _Pragma("unroll") for (int t = 0; t < T; ++t) if (k + (t % UB) <= hi) mk |= 1u << t; \
+                cur = sum_parent & mk; pc = imm; \
+            } else cur = sum_parent; } break;
+        TADV_V8(TADV_USEND, P_USEND)
 
 #define TADV_ZLOOP_BODY { \
             const TadpLoop &L = P.loops[a]; const int V = L.var; \
@@ -255,14 +323,16 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                 for (int r = 0; r < L.n_lower; ++r) { \
                     const TadpRow &R = P.rows[L.lower0 + r]; \
                     const int nmr = row_num(R, m.var); const int step = R.coef[lane_var] * 32; \
+                    const int ustep = (UB > 1 && unroll_var >= 0) ? R.coef[unroll_var] : 0; \
                     const int rstep = rel_var >= 0 ? R.coef[rel_var] : 0; \
-                    _Pragma("unroll") for (int t = 0; t < T; ++t) { int v = nmr + t * step + (REL && rstep ? rstep * zrel(t) : 0); v = R.den == 1 ? v : ceil_div_i(v, R.den); elo[lvl - 1][t] = max(elo[lvl - 1][t], v); } \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) { int v = nmr + (t / UB) * step + (t % UB) * ustep + (REL && rstep ? rstep * zrel(t) : 0); v = R.den == 1 ? v : ceil_div_i(v, R.den); elo[lvl - 1][t] = max(elo[lvl - 1][t], v); } \
                 } \
                 for (int r = 0; r < L.n_upper; ++r) { \
                     const TadpRow &R = P.rows[L.upper0 + r]; \
                     const int nmr = row_num(R, m.var); const int step = R.coef[lane_var] * 32; \
+                    const int ustep = (UB > 1 && unroll_var >= 0) ? R.coef[unroll_var] : 0; \
                     const int rstep = rel_var >= 0 ? R.coef[rel_var] : 0; \
-                    _Pragma("unroll") for (int t = 0; t < T; ++t) { int v = nmr + t * step + (REL && rstep ? rstep * zrel(t) : 0); v = R.den == 1 ? v : floor_div_i(v, R.den); ehi[lvl - 1][t] = min(ehi[lvl - 1][t], v); } \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) { int v = nmr + (t / UB) * step + (t % UB) * ustep + (REL && rstep ? rstep * zrel(t) : 0); v = R.den == 1 ? v : floor_div_i(v, R.den); ehi[lvl - 1][t] = min(ehi[lvl - 1][t], v); } \
                 } \
                 if (L.is_split) { \
                     /* every element's own range is divided into zsplit contiguous shares */ \
@@ -296,7 +366,7 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                     const int z = wlo + (int)(threadIdx.x & 31u); \
                     set_var(m.var, V, z); \
                     mk = 0; \
-                    _Pragma("unroll") for (int t = 0; t < T; ++t) if (z + 32 * t <= whi) mk |= 1u << t; \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) if (z + 32 * (t / UB) <= whi) mk |= 1u << t; \
                     mk &= parent; \
                 } else { \
                     set_var(m.var, V, wlo); \
@@ -316,14 +386,14 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
             const int lvl = L.mask_level; \
             const unsigned parent = mstack[lvl - 1]; \
             const int whi = loop_hi[a]; \
-            const int z = get_var(m.var, V) + (L.is_lane ? 32 * T : 1); \
+            const int z = get_var(m.var, V) + (L.is_lane ? 32 * TA : 1); \
             const int zbase = L.is_lane ? z - (int)(threadIdx.x & 31u) : z; \
             if (zbase <= whi) { \
                 set_var(m.var, V, z); \
                 unsigned mk; \
                 if (L.is_lane) { \
                     mk = 0; \
-                    _Pragma("unroll") for (int t = 0; t < T; ++t) if (z + 32 * t <= whi) mk |= 1u << t; \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) if (z + 32 * (t / UB) <= whi) mk |= 1u << t; \
                     mk &= parent; \
                 } else if (L.depends_on_lane) { \
                     mk = 0; \
