@@ -771,14 +771,17 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     if (g.kappa >= 1) {
         // a summation that can be split: take the widest shape and split to fill the GPU
         pick = shapes.front();
-        // splitting costs a pass over zsplit x outputs: only for small gradients that starve the GPU
-        if (items_for(pick) < target_warps / 2 && prog.out_limit <= (1 << 22)) {
+        // compact index of an output inside a plane of partial sums: row-major over the outer box
+        int64_t cells = 1;
+        for (int v = g.n_outer - 1; v >= 0; --v) { prog.part_coef[v] = to_i32(cells); cells = mul_ck(cells, prog.outer_ext[v]); }
+        // splitting costs a pass over zsplit planes: only when the outputs are too few to fill the GPU
+        if (items_for(pick) < target_warps / 2 && cells <= (1 << 22)) {
             TadpLoop &L0 = prog.loops[em.code[zbegin[0]].a];
             const int64_t ext0 = std::max<int64_t>(1, g.vars[L0.var].ext / (L0.is_lane ? 32 * pick.ta : 1));
             int64_t S = (int64_t)std::ceil(target_warps / items_for(pick));
             S = std::min<int64_t>(std::min<int64_t>(S, ext0), 4096);
-            while (S > 1 && S * (int64_t)prog.out_limit > (int64_t(1) << 25)) S /= 2;   // <= 128 MB of partial sums
-            if (S >= 2) { prog.zsplit = (int32_t)S; L0.is_split = 1; }
+            while (S > 1 && (S + 1) * cells > (int64_t(1) << 25)) S /= 2;   // <= 128 MB of partial sums
+            if (S >= 2) { prog.zsplit = (int32_t)S; prog.part_limit = to_i32(cells); L0.is_split = 1; }
         }
     } else {
         // element-wise kernel: the widest shape that still leaves enough warps
@@ -1041,7 +1044,7 @@ void generate_backward(tad_plan &p, int q)
     for (int d = 0; d < n; ++d) terms = mul_ck(terms, ap.box_hi[d] - ap.box_lo[d] + 1);
     finish_stats(g, k, true, p.arg_elems[ap.arg], terms, zero_fill && first_of_arg);
     if (prog.zsplit > 1) {
-        p.partial_bytes = std::max(p.partial_bytes, size_t(prog.zsplit) * size_t(prog.out_limit) * 4);
+        p.partial_bytes = std::max(p.partial_bytes, (size_t(prog.zsplit) + 1) * size_t(prog.part_limit) * 4);
         k.stats.n_launches += 1 + (prog.write_only_live ? 1 : 0);
     }
 }

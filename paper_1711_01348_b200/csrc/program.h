@@ -106,6 +106,8 @@ struct alignas(16) TadpProgram {
     int32_t write_only_live;           // 1: skip elements whose Gamma is empty (output pre-zeroed)
     int32_t zsplit;                    // > 1: that many warps share every output; each writes a partial sum
     int32_t rel_var;                   // variable of the relative loop, or -1
+    int32_t part_coef[TADP_MAX_VARS];  // zsplit > 1: compact index of an output in its plane of partial sums,
+    int32_t part_limit;                //   sum_v part_coef[v] * (var[v] - outer_lo[v]); part_limit entries per plane
     TadpInsn code[TADP_MAX_CODE];
     TadpLoad loads[TADP_MAX_LOADS];
     TadpLoop loops[TADP_MAX_LOOPS];
@@ -115,6 +117,7 @@ struct alignas(16) TadpProgram {
 struct TadpPointers {
     const float *in[TADP_MAX_PTRS];
     float *out;
-    float *part;                       // zsplit > 1: partial sums, zsplit planes of out_limit floats
+    float *part;                       // zsplit > 1: zsplit planes of part_limit partial sums, then one plane of
+                                       // flags (non-zero: some share of that output accumulated a term)
     int32_t *debug;                    // NULL unless the plan was compiled with debug_bounds
 };

@@ -88,9 +88,47 @@ tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ Tad
         for (int k = 0; k < TADP_MAX_VARS; ++k) if (k < P.n_outer) off += (unsigned)P.out_coef[k] * (unsigned)m.var[k];
         const unsigned step_a = lane_outer ? (unsigned)P.out_coef[lane_var] * 32u : 0u;
         const unsigned step_b = unroll_outer ? (unsigned)P.out_coef[unroll_var] : 0u;
-        float *dst = zsplit > 1 ? ptrs.part + (size_t)split * (unsigned)P.out_limit : ptrs.out;
-        const bool accumulate = zsplit > 1 ? false : P.accumulate != 0;
-        const bool only_live = zsplit > 1 ? false : P.write_only_live != 0;
+        if (zsplit > 1) {
+            // this warp's share of the sums goes to its plane of partial sums, indexed compactly
+            // by the outer variables; a second launch adds the planes up in order
+            unsigned cidx = 0;
+#pragma unroll
+            for (int k = 0; k < TADP_MAX_VARS; ++k) if (k < P.n_outer) cidx += (unsigned)P.part_coef[k] * (unsigned)(m.var[k] - P.outer_lo[k]);
+            const unsigned cstep_a = lane_outer ? (unsigned)P.part_coef[lane_var] * 32u : 0u;
+            const unsigned cstep_b = unroll_outer ? (unsigned)P.part_coef[unroll_var] : 0u;
+            float *plane = ptrs.part + (size_t)split * (unsigned)P.part_limit;
+            float *flags = ptrs.part + (size_t)zsplit * (unsigned)P.part_limit;
+            if (lane_outer) {
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    if ((e % UB) >= n_u || !((in_range >> e) & 1u)) continue;
+                    const unsigned c = cidx + (unsigned)(e / UB) * cstep_a + (unsigned)(e % UB) * cstep_b;
+                    plane[c] = m.acc[e];
+                    if ((live >> e) & 1u) flags[c] = 1.f;
+                }
+            } else {
+#pragma unroll
+                for (int u = 0; u < UB; ++u) {
+                    if (u >= n_u) continue;
+                    float total = 0.f;
+                    unsigned lv = 0;
+#pragma unroll
+                    for (int t = 0; t < TA; ++t) { total += m.acc[t * UB + u]; lv |= (live >> (t * UB + u)) & 1u; }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+                    const unsigned any_live = __ballot_sync(0xffffffffu, lv != 0);
+                    if (lane == 0 && first_b + (unsigned)u < ext_b) {
+                        const unsigned c = cidx + (unsigned)u * cstep_b;
+                        plane[c] = total;
+                        if (any_live) flags[c] = 1.f;
+                    }
+                }
+            }
+            continue;
+        }
+        float *dst = ptrs.out;
+        const bool accumulate = P.accumulate != 0;
+        const bool only_live = P.write_only_live != 0;
         if (lane_outer) {
 #pragma unroll
             for (int e = 0; e < E; ++e) {
@@ -124,14 +162,26 @@ tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ Tad
     }
 }
 
-// out[i] (+)= part[0][i] + part[1][i] + ... in that order
-__global__ void tad_reduce_partials(float *out, const float *part, unsigned n, int planes, int accumulate)
+// Adds the zsplit planes of partial sums up in plane order and writes the gradient elements:
+// compact index c -> outer variables -> output offset.  Masked gradients write only outputs
+// whose flag says that some term was accumulated.
+__global__ void tad_reduce_partials(const __grid_constant__ TadpProgram P, float *out, const float *part)
 {
+    const unsigned n = (unsigned)P.part_limit;
     const unsigned stride = gridDim.x * blockDim.x;
-    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
-        float sum = accumulate ? out[i] : 0.f;
-        for (int s = 0; s < planes; ++s) sum += part[(size_t)s * n + i];
-        out[i] = sum;
+    const int planes = P.zsplit;
+    for (unsigned c = blockIdx.x * blockDim.x + threadIdx.x; c < n; c += stride) {
+        if (P.write_only_live && part[(size_t)planes * n + c] == 0.f) continue;
+        unsigned rem = c, off = (unsigned)P.out_base;
+        for (int v = P.n_outer - 1; v >= 0; --v) {
+            const unsigned ext = (unsigned)P.outer_ext[v];
+            const unsigned digit = rem % ext; rem /= ext;
+            off += (unsigned)P.out_coef[v] * (unsigned)(P.outer_lo[v] + (int)digit);
+        }
+        if (off >= (unsigned)P.out_limit) continue;
+        float sum = P.accumulate ? out[off] : 0.f;
+        for (int s = 0; s < planes; ++s) sum += part[(size_t)s * n + c];
+        out[off] = sum;
     }
 }
 
@@ -179,8 +229,8 @@ tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStrea
     if (zsplit > 1) {
         if (!ptrs.part) { tad::set_error("internal: partial-sum buffer missing"); return TAD_ERR_WORKSPACE; }
         if (k.prog.write_only_live) {
-            // masked gradients leave elements unvisited: their partial sums must read as zero
-            tad_status st = zero_fill(ptrs.part, (int64_t)zsplit * k.prog.out_limit, stream);
+            // masked gradients: the flag plane must start at zero
+            tad_status st = zero_fill(ptrs.part + (size_t)zsplit * k.prog.part_limit, k.prog.part_limit, stream);
             if (st != TAD_OK) return st;
         }
     }
@@ -206,9 +256,9 @@ tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStrea
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { tad::set_error(std::string("kernel launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
     if (zsplit > 1) {
-        const unsigned n = (unsigned)k.prog.out_limit;
+        const unsigned n = (unsigned)k.prog.part_limit;
         const unsigned rblocks = std::min((n + 255u) / 256u, (unsigned)sm_count() * 16u);
-        tad_reduce_partials<<<rblocks, 256, 0, stream>>>(ptrs.out, ptrs.part, n, zsplit, k.prog.accumulate);
+        tad_reduce_partials<<<rblocks, 256, 0, stream>>>(k.prog, ptrs.out, ptrs.part);
         e = cudaGetLastError();
         if (e != cudaSuccess) { tad::set_error(std::string("reduce launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
     }

@@ -244,5 +244,6 @@ def test_kernel_stats_and_listing():
     assert fwd.alg_bytes == pytest.approx(4 * nij + 4 * (2 * 8192 * 32 + 8223) + 32 * 8192, rel=1e-6)
     q = {e.arg_names[a.arg]: i for i, a in enumerate(e.accesses)}
     st = plan.kernel_stats(q["c"])
-    assert st.terms == 8192 * 8192 * 32 and st.n_launches == 2     # zero fill + gather
+    # zero fill of dc, clearing the flags of the split summation, gather, fixed-order reduction
+    assert st.terms == 8192 * 8192 * 32 and st.n_launches == 4
     assert "ZLOOP" in plan.disassemble(q["c"]) and "SLOOP" in plan.disassemble(-1)
