@@ -88,6 +88,29 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def source_digest() -> str:
+    """Digest of the kernel sources: ncu counters recorded for another digest are stale."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_1711_01348_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(workload: str, part: str):
+    """DRAM bytes per launch of one part from the committed ncu capture, or None if absent or stale."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as fh:
+        rec = json.load(fh)
+    if rec.get("source_digest") != source_digest():
+        return None
+    return rec.get(workload, {}).get(part)
+
+
 def elements_per_step(expr) -> int:
     n = 1
     for s in expr.out_shape:
@@ -148,17 +171,11 @@ def run_ours(opts):
     from paper_1711_01348_b200 import Plan
     from workloads import configs as W
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    distributed = world > 1
-    if distributed:
-        import torch.distributed as dist
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        torch.cuda.set_device(local_rank)
-        dist.init_process_group("nccl")
+    from paper_1711_01348_b200 import replicas
+    rank, local_rank, world = replicas.rank_info()
     dev = torch.device(f"cuda:{local_rank}")
     torch.cuda.set_device(dev)
+    distributed = replicas.init("nccl")
 
     expr, args, df = W.workload(opts.config, full=True)
     if opts.rows:
@@ -199,9 +216,7 @@ def run_ours(opts):
             events[e].record()
 
     def barrier():
-        if distributed:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(distributed)
 
     for _ in range(opts.warmup):
         step()
@@ -218,11 +233,7 @@ def run_ours(opts):
     t_end.record()
     barrier()
     clocks = sampler.stop() if rank == 0 else None
-    total_ms = t_begin.elapsed_time(t_end)
-    if distributed:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = replicas.max_over_ranks(t_begin.elapsed_time(t_end), distributed, dev)
     part_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in all_events) / opts.steps for i in range(n_parts)]
 
     # end to end: pinned host buffers in, results back, through tad_step_host
@@ -247,10 +258,7 @@ def run_ours(opts):
             host_step()
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0) / e2e_steps
-        if distributed:
-            t = torch.tensor([e2e_s], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = replicas.max_over_ranks(e2e_s, distributed, dev)
         h2d = sum(a.numel() * 4 for a in args) + df.numel() * 4
         d2h = h_f.numel() * 4 + sum(d.numel() * 4 for d in h_dargs)
         e2e = {"value": world * elements_per_step(expr) / e2e_s, "unit": UNIT,
@@ -298,6 +306,7 @@ def run_ours(opts):
             roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
         roof["kernel"] = d["part"]
+        roof["traffic"] = recorded_traffic(expr.name, d["part"])
         cpu = None
         if not distributed and not opts.no_cpu_baseline and not opts.rows:
             from oracle.oracle import build as build_oracle, max_threads
@@ -317,9 +326,7 @@ def run_ours(opts):
                 "roofline": roof, "parts": per_part, "cpu_baseline": cpu, "e2e": e2e,
                 "gpu_launches": launches * opts.steps, "clocks": clocks}
         print(json.dumps(line), flush=True)
-    if distributed:
-        dist.barrier()
-        dist.destroy_process_group()
+    replicas.finish(distributed)
 
 
 def main():
