@@ -315,8 +315,8 @@ struct Gen {
 const char *op_name(int op)
 {
     static const char *names[] = {"END", "CONST", "ZERO", "LOAD", "LDT", "NEG", "SQR", "CUBE", "HSUM", "MULC", "ADDC",
-                                  "LDADD", "LDMUL", "FN", "STT", "ACC", "ADD", "SUB", "MUL", "DIV", "SUMADD",
-                                  "MACC", "FMA", "SLOOP", "SEND", "USLOOP", "USEND", "ZLOOP", "ZEND"};
+                                  "LDADD", "LDMUL", "LDADDSQ", "SCALE", "FN", "STT", "ACC", "ADD", "SUB", "MUL", "DIV",
+                                  "SUMADD", "SUMEND", "FMAT", "MACC", "FMA", "SLOOP", "SEND", "USLOOP", "USEND", "ZLOOP", "ZEND"};
     return op < P_NUM_OPS ? names[op] : "?";
 }
 
@@ -373,7 +373,15 @@ struct Emitter {
         case I_TANH: expr(in.a); emit(P_FN, same_for_all_u(in.a), F_TANH); break;
         case I_SINH: expr(in.a); emit(P_FN, same_for_all_u(in.a), F_SINH); break;
         case I_COSH: expr(in.a); emit(P_FN, same_for_all_u(in.a), F_COSH); break;
-        case I_SQR: expr(in.a); emit(P_SQR); break;
+        case I_SQR: {
+            const Inst &ad = g.inst[in.a];
+            if (ad.op == I_ADD && inline_ok(in.a) && (is_inline_load(ad.a) || is_inline_load(ad.b)) &&
+                !(g.inst[ad.a].op == I_MUL && inline_ok(ad.a)) && !(g.inst[ad.b].op == I_MUL && inline_ok(ad.b))) {
+                const int ld = is_inline_load(ad.b) ? ad.b : ad.a, other = is_inline_load(ad.b) ? ad.a : ad.b;
+                expr(other); emit(P_LDADDSQ, g.inst[ld].load);
+            } else { expr(in.a); emit(P_SQR); }
+            break;
+        }
         case I_POWI:
             expr(in.a);
             if (in.ipow == 3) emit(P_CUBE); else emit(P_FN, same_for_all_u(in.a), F_POWI, in.ipow);
@@ -385,7 +393,13 @@ struct Emitter {
             int m = -1, o = -1;
             if (g.inst[in.a].op == I_MUL && inline_ok(in.a)) { m = in.a; o = in.b; }
             else if (g.inst[in.b].op == I_MUL && inline_ok(in.b)) { m = in.b; o = in.a; }
-            if (m >= 0) { expr(g.inst[m].a); expr(g.inst[m].b); expr(o); emit(P_FMA, 0, 0, 0, -2); }
+            if (m >= 0 && (g.inst[g.inst[m].a].temp >= 0 || g.inst[g.inst[m].b].temp >= 0)) {
+                // product with a temporary: the temporary is read by the fused word itself
+                const int tf = g.inst[g.inst[m].b].temp >= 0 ? g.inst[m].b : g.inst[m].a;
+                const int other = tf == g.inst[m].b ? g.inst[m].a : g.inst[m].b;
+                expr(other); expr(o); emit(P_FMAT, g.inst[tf].temp, 0, 0, -1);
+            }
+            else if (m >= 0) { expr(g.inst[m].a); expr(g.inst[m].b); expr(o); emit(P_FMA, 0, 0, 0, -2); }
             else if (is_inline_load(in.b)) { expr(in.a); emit(P_LDADD, g.inst[in.b].load); }
             else if (is_inline_load(in.a)) { expr(in.b); emit(P_LDADD, g.inst[in.a].load); }
             else { expr(in.a); expr(in.b); emit(P_ADD, 0, 0, 0, -1); }
@@ -409,8 +423,11 @@ struct Emitter {
             int begin = emit(over_elements ? P_USLOOP : P_SLOOP, id, 0, 0, 0, in.var);
             temps_of_sum(i);
             expr(in.a);
-            emit(P_SUMADD, 0, 0, 0, -1);
-            int end = emit(over_elements ? P_USEND : P_SEND, id, 0, begin + 1, 0, in.var);
+            int end;
+            if (over_elements) {
+                emit(P_SUMADD, 0, 0, 0, -1);
+                end = emit(P_USEND, id, 0, begin + 1, 0, in.var);
+            } else end = emit(P_SUMEND, id, 0, begin + 1, -1);
             if (over_elements) emit(P_HSUM);
             code[begin].imm = end + 1;
             break;
@@ -452,13 +469,14 @@ double inst_weight(const Inst &in)
 }
 
 // marks use counts of everything reachable from `root`
-void count_uses(Gen &g, int root)
+void count_uses(Gen &g, int root, int root2 = -1)
 {
     for (Inst &in : g.inst) in.uses = 0;
     std::vector<int> stack{root};
     g.inst[root].uses = 1;
     std::vector<bool> seen(g.inst.size(), false);
     seen[root] = true;
+    if (root2 >= 0 && root2 != root) { stack.push_back(root2); g.inst[root2].uses += 1; seen[root2] = true; }
     while (!stack.empty()) {
         int i = stack.back(); stack.pop_back();
         for (int c : {g.inst[i].a, g.inst[i].b}) {
@@ -629,6 +647,40 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
 {
     TadpProgram &prog = k.prog;
     place(g);
+    // Factors of the term that no kernel coordinate touches (and constant factors) multiply the
+    // finished sum once instead of every term:  sum_z (c * X * Y(z)) = c * X * sum_z Y(z).
+    int scale = -1;
+    if (g.kappa >= 1) {
+        std::vector<int> outer_factors, inner_factors;
+        float cfac = 1.f;
+        std::vector<int> todo{root};
+        while (!todo.empty()) {
+            const int i = todo.back(); todo.pop_back();
+            const Inst in = g.inst[i];
+            const bool sole = i == root || in.uses == 1;
+            if (in.op == I_MUL && sole) { todo.push_back(in.a); todo.push_back(in.b); }
+            else if (in.op == I_MULC && sole) { cfac *= in.imm; todo.push_back(in.a); }
+            else if (in.op == I_NEG && sole) { cfac = -cfac; todo.push_back(in.a); }
+            else if (in.op == I_SQR && sole && g.inst[in.a].zlevel == 0 && g.inst[in.a].home_sum < 0) outer_factors.push_back(i);
+            else if (in.zlevel == 0 && in.home_sum < 0 && in.op != I_CONST) outer_factors.push_back(i);
+            else inner_factors.push_back(i);
+        }
+        if (!inner_factors.empty() && (!outer_factors.empty() || cfac != 1.f)) {
+            std::sort(inner_factors.begin(), inner_factors.end());
+            std::sort(outer_factors.begin(), outer_factors.end());
+            int term = inner_factors[0];
+            for (size_t f = 1; f < inner_factors.size(); ++f) term = g.bin(I_MUL, term, inner_factors[f]);
+            if (outer_factors.empty()) scale = g.konst(cfac);
+            else {
+                scale = outer_factors[0];
+                for (size_t f = 1; f < outer_factors.size(); ++f) scale = g.bin(I_MUL, scale, outer_factors[f]);
+                scale = g.mulc(scale, cfac);
+            }
+            root = term;
+            count_uses(g, root, scale);
+            place(g);
+        }
+    }
     choose_element_variable(g);
     // temporaries: shared values and values hoisted out of the loop that consumes them
     std::vector<bool> hoisted(g.inst.size(), false);
@@ -648,7 +700,7 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     for (int i = 0; i < (int)g.inst.size(); ++i) {
         Inst &in = g.inst[i];
         in.temp = -1;
-        if (!in.uses || in.op == I_CONST || i == root) continue;
+        if (!in.uses || in.op == I_CONST || i == root || i == scale) continue;
         if (in.uses > 1 || hoisted[i]) {
             if (n_temps >= TADP_NUM_TEMPS + TADP_MAX_SPILL) throw Unsupported("too many temporaries");
             in.temp = n_temps++;
@@ -678,6 +730,7 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
         int end = em.emit(P_ZEND, loop_id, 0, zbegin[l] + 1, 0, em.loops[loop_id].var);
         em.code[zbegin[l]].imm = end + 1;
     }
+    if (scale >= 0) { em.expr(scale); em.emit(P_SCALE, 0, 0, 0, -1); }
     em.emit(P_END);
     if (em.depth != 0) throw BadExpr("internal: unbalanced operand stack");
     // rows

@@ -33,6 +33,8 @@ enum TadpOp : int {
     P_HSUM,       // top[t][u] <- sum over u' of top[t][u'] (closes a sum loop that runs over the element variable)
     P_MULC, P_ADDC,               // top <- top op imm(float)
     P_LDADD, P_LDMUL,             // top <- top op load(loads[a])
+    P_LDADDSQ,                    // top <- (top + load(loads[a]))^2
+    P_SCALE,      // acc <- acc * top ; pop (factors of the term that no loop variable touches, applied once)
     P_FN,         // top <- function b of top: TadpFn; F_POWI takes its exponent from imm; a != 0: the value is
                   // the same for every u, evaluate it once per lane-variable element
     P_STT,        // temp[a] <- top ; pop
@@ -40,6 +42,8 @@ enum TadpOp : int {
     // two operands (k = 2..7): second <- second op top ; pop
     P_ADD, P_SUB, P_MUL, P_DIV,
     P_SUMADD,     // second += top ; pop
+    P_SUMEND,     // P_SUMADD followed by the P_SEND of loops[a] in one word
+    P_FMAT,       // second <- second * temp[a] + top ; pop
     P_MACC,       // acc += active ? second * top : 0 ; pop 2
     // three operands (k = 3..7)
     P_FMA,        // third <- third * second + top ; pop 2

@@ -206,6 +206,8 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
         TADV_D1(TADV_LDADD, P_LDADD)
 #define TADV_LDMUL(OP, D) TADV_CASE(OP, D, D) TADV_LOAD_BODY(m.s[D - 1][t] = op_mul(m.s[D - 1][t], v)) break;
         TADV_D1(TADV_LDMUL, P_LDMUL)
+#define TADV_LDADDSQ(OP, D) TADV_CASE(OP, D, D) TADV_LOAD_BODY({ const float w2 = op_add(m.s[D - 1][t], v); m.s[D - 1][t] = op_mul(w2, w2); }) break;
+        TADV_D1(TADV_LDADDSQ, P_LDADDSQ)
 
 #define TADV_UNARY(D, EXPR) { _Pragma("unroll") for (int t = 0; t < T; ++t) { const float x = m.s[D - 1][t]; m.s[D - 1][t] = (EXPR); } } break;
 #define TADV_NEG(OP, D) TADV_CASE(OP, D, D) TADV_UNARY(D, op_neg(x))
@@ -236,6 +238,13 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
         // runs over the element variable) leave it unchanged
 #define TADV_SUMADD(OP, D) TADV_CASE(OP, D, D) { _Pragma("unroll") for (int t = 0; t < T; ++t) if (UB == 1 || ((cur >> t) & 1u)) m.s[D - 2][t] = op_add(m.s[D - 2][t], m.s[D - 1][t]); } break;
         TADV_D2(TADV_SUMADD, P_SUMADD)
+        // summand into the accumulator and the end of the (ordinary) sum loop in one word
+#define TADV_SUMEND(OP, D) TADV_CASE(OP, D, D) { \
+            _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 2][t] = op_add(m.s[D - 2][t], m.s[D - 1][t]); \
+            const TadpLoop &L = P.loops[a]; \
+            const int k = get_var(m.var, L.var) + 1; \
+            if (k <= L.const_hi) { set_var(m.var, L.var, k); pc = imm; } } break;
+        TADV_D2(TADV_SUMEND, P_SUMEND)
         // closes a sum over the element variable: add up the UB partial sums, replicate the result
 #define TADV_HSUM(OP, D) TADV_CASE(OP, D, D) { \
             _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { \
@@ -270,8 +279,14 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
             _Pragma("unroll") for (int t = 0; t < T; ++t) spill[K][t] = m.s[D - 1][t];) } break;
         TADV_D1(TADV_STT, P_STT)
 
+#define TADV_FMAT(OP, D) TADV_CASE(OP, D, D) { TADV_TEMP_SWITCH( \
+            _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 2][t] = op_fma(m.s[D - 2][t], m.tmp[K][t], m.s[D - 1][t]);, \
+            _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 2][t] = op_fma(m.s[D - 2][t], spill[K][t], m.s[D - 1][t]);) } break;
+        TADV_D2(TADV_FMAT, P_FMAT)
 #define TADV_ACC(OP, D) TADV_CASE(OP, D, D) { _Pragma("unroll") for (int t = 0; t < T; ++t) if ((cur >> t) & 1u) m.acc[t] = op_add(m.acc[t], m.s[D - 1][t]); live |= cur; } break;
         TADV_D1(TADV_ACC, P_ACC)
+#define TADV_SCALE(OP, D) TADV_CASE(OP, D, D) { _Pragma("unroll") for (int t = 0; t < T; ++t) m.acc[t] = op_mul(m.acc[t], m.s[D - 1][t]); } break;
+        TADV_D1(TADV_SCALE, P_SCALE)
 #define TADV_MACC(OP, D) TADV_CASE(OP, D, D) { _Pragma("unroll") for (int t = 0; t < T; ++t) if ((cur >> t) & 1u) m.acc[t] = op_fma(m.s[D - 2][t], m.s[D - 1][t], m.acc[t]); live |= cur; } break;
         TADV_D2(TADV_MACC, P_MACC)
 
