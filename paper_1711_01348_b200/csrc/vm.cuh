@@ -171,7 +171,8 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                 /* constant along the element variable: one load per lane-variable element */ \
                 _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { \
                     const unsigned mm = (cur >> (ta * UB)) & ((1u << UB) - 1u); \
-                    const float v = mm ? __ldg(base + off + (unsigned)ta * lc) : 0.f; \
+                    const unsigned idx = off + (unsigned)ta * lc;   /* mod 2^32 before it meets the pointer */ \
+                    const float v = mm ? __ldg(base + idx) : 0.f; \
                     _Pragma("unroll") for (int u = 0; u < UB; ++u) { const int t = ta * UB + u; DST_EXPR; } \
                 } \
             } else if (UB % 4 == 0 && uc == 1 && (!REL || L.rel_step == 0) && !DEBUG && (reinterpret_cast<uintptr_t>(base) & 15u) == 0) { \
@@ -182,13 +183,29 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                         const unsigned mm = (cur >> (ta * UB + 4 * g4)) & 0xfu; \
                         float q[4]; \
                         if (mm == 0xfu && ((o + 4u * g4) & 3u) == 0) { \
-                            const float4 f4 = __ldg(reinterpret_cast<const float4 *>(base + o + 4 * g4)); \
+                            const float4 f4 = __ldg(reinterpret_cast<const float4 *>(base + (o + 4u * g4))); \
                             q[0] = f4.x; q[1] = f4.y; q[2] = f4.z; q[3] = f4.w; \
                         } else { \
-                            _Pragma("unroll") for (int i = 0; i < 4; ++i) q[i] = ((mm >> i) & 1u) ? __ldg(base + o + 4 * g4 + i) : 0.f; \
+                            _Pragma("unroll") for (int i = 0; i < 4; ++i) q[i] = ((mm >> i) & 1u) ? __ldg(base + (o + 4u * g4 + i)) : 0.f; \
                         } \
                         _Pragma("unroll") for (int i = 0; i < 4; ++i) { const int t = ta * UB + 4 * g4 + i; const float v = q[i]; DST_EXPR; } \
                     } \
+                } \
+            } else if (UB > 1 && TA > 1 && lc == 0 && (!REL || L.rel_step == 0) && !DEBUG) { \
+                /* the same for every lane and every t: one load per u */ \
+                _Pragma("unroll") for (int u = 0; u < UB; ++u) { \
+                    unsigned mm = 0; \
+                    _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) mm |= (cur >> (ta * UB + u)) & 1u; \
+                    const unsigned idx = off + (unsigned)u * uc; \
+                    const float v = mm ? __ldg(base + idx) : 0.f; \
+                    _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { const int t = ta * UB + u; DST_EXPR; } \
+                } \
+            } else if (!DEBUG && !REL && cur == (T >= 32 ? 0xffffffffu : ((1u << T) - 1u))) { \
+                /* every element live: no per-element predicates */ \
+                _Pragma("unroll") for (int t = 0; t < T; ++t) { \
+                    const unsigned idx = off + (unsigned)(t / UB) * lc + (unsigned)(t % UB) * uc; \
+                    const float v = __ldg(base + idx); \
+                    DST_EXPR; \
                 } \
             } else { \
                 const unsigned rs = REL ? (unsigned)L.rel_step : 0u; \
