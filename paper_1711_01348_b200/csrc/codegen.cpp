@@ -316,7 +316,7 @@ const char *op_name(int op)
 {
     static const char *names[] = {"END", "CONST", "ZERO", "LOAD", "LDT", "NEG", "SQR", "CUBE", "HSUM", "MULC", "ADDC",
                                   "LDADD", "LDMUL", "LDADDSQ", "SCALE", "FN", "STT", "ACC", "ADD", "SUB", "MUL", "DIV",
-                                  "SUMADD", "SUMEND", "FMAT", "MACC", "FMA", "SLOOP", "SEND", "USLOOP", "USEND", "ZLOOP", "ZEND"};
+                                  "SUMADD", "SUMEND", "FMAT", "MACC", "FMA", "SLOOP", "SEND", "USLOOP", "USEND", "ZLOOP", "ZEND", "XLOOP"};
     return op < P_NUM_OPS ? names[op] : "?";
 }
 
@@ -325,7 +325,7 @@ struct Emitter {
     std::vector<TadpInsn> code;
     std::vector<TadpLoop> loops;
     int depth = 0, max_depth = 0;
-    std::string listing;
+    std::vector<int> depth_at;           // operand stack depth before every word
 
     explicit Emitter(Gen &gen) : g(gen) {}
 
@@ -337,16 +337,25 @@ struct Emitter {
         w.handler = (uint16_t)(op * 8 + (k_override >= 0 ? k_override : depth));
         w.a = (uint8_t)a; w.b = (uint8_t)b; w.imm = imm;
         code.push_back(w);
-        char line[160];
-        float f; std::memcpy(&f, &imm, 4);
-        std::snprintf(line, sizeof line, "%3zu  d=%d  %-7s a=%d b=%d imm=%d (%g)\n", code.size() - 1, depth, op_name(op), a, b, imm, (double)f);
-        listing += line;
+        depth_at.push_back(depth);
         depth += delta;
         max_depth = std::max(max_depth, depth);
         if ((int)code.size() >= TADP_MAX_CODE) throw Unsupported("program longer than TADP_MAX_CODE words");
         return (int)code.size() - 1;
     }
     static int32_t fbits(float f) { int32_t b; std::memcpy(&b, &f, 4); return b; }
+    std::string listing() const
+    {
+        std::string out;
+        for (size_t i = 0; i < code.size(); ++i) {
+            char line[160];
+            float f; std::memcpy(&f, &code[i].imm, 4);
+            std::snprintf(line, sizeof line, "%3zu  d=%d  %-7s a=%d b=%d imm=%d (%g)\n", i, depth_at[i], op_name(code[i].handler >> 3),
+                          code[i].a, code[i].b, code[i].imm, (double)f);
+            out += line;
+        }
+        return out;
+    }
 
     bool inline_ok(int i) const { return g.inst[i].temp < 0; }
     // the value does not vary along the element variable (and is not computed inside its sum loop)
@@ -641,6 +650,159 @@ void choose_element_variable(Gen &g)
     }
 }
 
+// ---- fused innermost loops ----------------------------------------------------------------
+// An innermost loop whose body is a short chain of loads and arithmetic on at most two live values
+// (plus two loop-invariant ones) is rewritten as an accumulator program (TadpBody) and the body
+// and loop end are replaced by one P_XLOOP word: the interpreter then runs every trip of the loop
+// without fetching and dispatching a word per operation.  Everything else keeps the general form.
+struct BodyDraft {
+    std::vector<uint8_t> steps;
+    std::vector<int> loads;
+    std::vector<std::pair<int, int32_t>> inv;   // (kind, value)
+    int term = 0;
+    bool uses_y = false;
+};
+
+bool draft_body(const std::vector<TadpInsn> &code, int first, int last, int term_op, BodyDraft &d)
+{
+    int vd = 0;   // live values of the body: 0, 1 (X) or 2 (Y below X)
+    auto inv_slot = [&](int kind, int32_t value) {
+        for (size_t q = 0; q < d.inv.size(); ++q) if (d.inv[q].first == kind && d.inv[q].second == value) return (int)q;
+        if (d.inv.size() >= 2) return -1;
+        d.inv.push_back({kind, value});
+        return (int)d.inv.size() - 1;
+    };
+    auto load_step = [&](int id, int cmb) {
+        int j = -1;
+        for (size_t q = 0; q < d.loads.size(); ++q) if (d.loads[q] == id) j = (int)q;
+        if (j < 0) { if ((int)d.loads.size() >= TADP_BODY_LOADS) return false; d.loads.push_back(id); j = (int)d.loads.size() - 1; }
+        d.steps.push_back((uint8_t)(0x80 | (cmb << 2) | j));
+        return true;
+    };
+    for (int w = first; w <= last; ++w) {
+        const int op = code[w].handler >> 3;
+        switch (op) {
+        case P_LOAD:
+            if (vd == 2) return false;
+            if (vd == 1) { d.steps.push_back(BS_PUSH); d.uses_y = true; }
+            if (!load_step(code[w].a, 0)) return false;
+            ++vd;
+            break;
+        case P_LDT: case P_CONST: {
+            const int q = inv_slot(op == P_LDT ? 2 : 1, op == P_LDT ? (int32_t)code[w].a : code[w].imm);
+            if (q < 0 || vd == 2) return false;
+            if (vd == 0) { d.steps.push_back((uint8_t)(q ? BS_LDI1 : BS_LDI0)); vd = 1; break; }
+            const int next = w + 1 <= last ? code[w + 1].handler >> 3 : -1;
+            if (next == P_MUL) { d.steps.push_back((uint8_t)(q ? BS_MULI1 : BS_MULI0)); ++w; }
+            else if (next == P_ADD) { d.steps.push_back((uint8_t)(q ? BS_ADDI1 : BS_ADDI0)); ++w; }
+            else { d.steps.push_back(BS_PUSH); d.uses_y = true; d.steps.push_back((uint8_t)(q ? BS_LDI1 : BS_LDI0)); vd = 2; }
+            break;
+        }
+        case P_LDADD: case P_LDMUL: case P_LDADDSQ:
+            if (vd < 1 || !load_step(code[w].a, op == P_LDADD ? 1 : op == P_LDMUL ? 2 : 3)) return false;
+            break;
+        case P_NEG: if (vd < 1) return false; d.steps.push_back(BS_NEG); break;
+        case P_SQR: if (vd < 1) return false; d.steps.push_back(BS_SQR); break;
+        case P_CUBE: if (vd < 1) return false; d.steps.push_back(BS_CUBE); break;
+        case P_MULC: case P_ADDC: {
+            const int q = inv_slot(1, code[w].imm);
+            if (q < 0 || vd < 1) return false;
+            d.steps.push_back((uint8_t)(op == P_MULC ? (q ? BS_MULI1 : BS_MULI0) : (q ? BS_ADDI1 : BS_ADDI0)));
+            break;
+        }
+        case P_ADD: case P_SUB: case P_MUL: case P_DIV:
+            if (vd != 2) return false;
+            d.steps.push_back((uint8_t)(op == P_ADD ? BS_ADDY : op == P_SUB ? BS_SUBY : op == P_MUL ? BS_MULY : BS_DIVY));
+            vd = 1;
+            break;
+        case P_FMAT: {
+            const int q = inv_slot(2, code[w].a);
+            if (q < 0 || vd != 2) return false;
+            d.steps.push_back((uint8_t)(q ? BS_FMAYI1 : BS_FMAYI0));
+            vd = 1;
+            break;
+        }
+        default: return false;
+        }
+    }
+    if (term_op == P_MACC) { if (vd != 2) return false; d.term = 1; d.uses_y = true; }
+    else if (vd != 1) return false;
+    return !d.steps.empty() && (int)d.steps.size() <= TADP_BODY_STEPS;
+}
+
+// returns the deepest operand stack the remaining words need
+int fuse_inner_loops(Emitter &em, std::vector<TadpBody> &bodies, int depth_limit)
+{
+    std::vector<TadpInsn> &code = em.code;
+    for (int b = 0; b < (int)code.size(); ++b) {
+        const int bop = code[b].handler >> 3;
+        if (bop != P_SLOOP && bop != P_USLOOP && bop != P_ZLOOP) continue;
+        if ((int)bodies.size() >= TADP_MAX_BODIES) break;
+        const int e = code[b].imm - 1;                       // the loop end word
+        if (e <= b + 1 || e >= (int)code.size()) continue;
+        const int eop = code[e].handler >> 3;
+        bool innermost = true;
+        for (int w = b + 1; w < e; ++w) {
+            const int op = code[w].handler >> 3;
+            if (op >= P_SLOOP && op <= P_XLOOP) innermost = false;
+        }
+        if (!innermost) continue;
+        const TadpLoop &L = em.loops[code[b].a];
+        int last, term_op, kind, xi;
+        if (bop == P_SLOOP && eop == P_SUMEND) { last = e - 1; term_op = P_SUMEND; kind = BL_SUM; xi = 1; }
+        else if (bop == P_USLOOP && eop == P_USEND && (code[e - 1].handler >> 3) == P_SUMADD) { last = e - 2; term_op = P_SUMADD; kind = BL_USUM; xi = 1; }
+        else if (bop == P_ZLOOP && eop == P_ZEND && ((code[e - 1].handler >> 3) == P_ACC || (code[e - 1].handler >> 3) == P_MACC)) {
+            if (L.is_relative) continue;
+            last = e - 2; term_op = code[e - 1].handler >> 3; xi = 0;
+            kind = L.is_lane ? BL_Z_LANE : L.depends_on_lane ? BL_Z_MASKED : BL_Z;
+        } else continue;
+        if (em.depth_at[b + 1] != xi) continue;             // the sum accumulator must be the bottom of the stack
+        BodyDraft d;
+        if (!draft_body(code, b + 1, last, term_op, d)) continue;
+        if (xi + (d.uses_y ? 2 : 1) + (int)d.inv.size() > depth_limit) continue;
+        TadpBody B{};
+        for (size_t i = 0; i < d.steps.size(); ++i) B.steps[i] = d.steps[i];
+        for (size_t i = 0; i < d.loads.size(); ++i) B.load[i] = (uint8_t)d.loads[i];
+        B.n_loads = (int32_t)d.loads.size();
+        B.loop_kind = kind; B.term = d.term;
+        for (size_t q = 0; q < d.inv.size(); ++q) { B.inv_kind[q] = d.inv[q].first; B.inv_value[q] = d.inv[q].second; }
+        bodies.push_back(B);
+        // body and loop end become one word; jump targets behind it move up
+        const int removed = e - (b + 1);
+        TadpInsn x{};
+        x.handler = (uint16_t)(P_XLOOP * 8 + xi); x.a = code[b].a; x.imm = (int32_t)bodies.size() - 1;
+        code[b + 1] = x;
+        code.erase(code.begin() + b + 2, code.begin() + e + 1);
+        em.depth_at.erase(em.depth_at.begin() + b + 2, em.depth_at.begin() + e + 1);
+        for (TadpInsn &w : code) {
+            const int op = w.handler >> 3;
+            const bool jumps = op == P_SLOOP || op == P_SEND || op == P_USLOOP || op == P_USEND || op == P_ZLOOP || op == P_ZEND || op == P_SUMEND;
+            if (jumps && w.imm > e) w.imm -= removed;
+        }
+    }
+    int deepest = 0;
+    for (size_t i = 0; i < code.size(); ++i) {
+        const int op = code[i].handler >> 3;
+        if (op >= P_SLOOP && op <= P_ZEND) continue;
+        int after = em.depth_at[i];
+        if (op == P_XLOOP) continue;                      // checked against depth_limit when it was made
+        if (op == P_CONST || op == P_ZERO || op == P_LOAD || op == P_LDT) after += 1;
+        deepest = std::max(deepest, after);
+    }
+    return deepest;
+}
+
+// how a fused body fetches a load, given the vector shape
+int body_fetch_kind(const TadpLoad &L, int ta, int ub)
+{
+    const bool lane_fixed = L.lane_step == 0, u_fixed = ub == 1 || L.unroll_step == 0;
+    if (lane_fixed && u_fixed) return BF_ONE;
+    if (ub > 1 && u_fixed) return BF_PER_T;
+    if (ub > 1 && ta > 1 && lane_fixed) return BF_PER_U;
+    if (ub > 1 && ub % 4 == 0 && L.unroll_step == 1) return BF_ROW;
+    return BF_EACH;
+}
+
 // shared tail: choose temps, emit, fill the program
 void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<TadpRow>> &lower,
                  const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards)
@@ -749,8 +911,6 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     prog.guard0 = (int32_t)rows.size(); prog.n_guards = (int32_t)guards.size();
     for (const TadpRow &r : guards) rows.push_back(r);
     if ((int)rows.size() > TADP_MAX_ROWS) throw Unsupported("too many bound rows in one kernel");
-    prog.n_code = (int32_t)em.code.size();
-    std::copy(em.code.begin(), em.code.end(), prog.code);
     prog.n_loads = (int32_t)g.loads.size();
     std::copy(g.loads.begin(), g.loads.end(), prog.loads);
     // relative loop: a kernel-coordinate loop whose range is short but starts at a different value
@@ -791,8 +951,14 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     const int64_t lane_ext = g.vars[g.lane_var].ext;
     const double target_warps = 148.0 * 16.0 * 2.0;
     const int64_t uext = g.unroll_var >= 0 ? g.vars[g.unroll_var].ext : 1;
-    const bool shallow = em.max_depth <= TADP_WIDE_DEPTH;
     const bool debug = g.p.opt.debug_bounds != 0;
+    // fused inner loops leave the operand stack to the rest of the program: try them with the
+    // 4-deep stack of the 16-value variants first
+    const bool can_fuse = !debug && prog.rel_var < 0;
+    Emitter trial(em);
+    std::vector<TadpBody> bodies_wide;
+    const int deepest_wide = can_fuse ? fuse_inner_loops(trial, bodies_wide, TADP_WIDE_DEPTH) : em.max_depth;
+    const bool shallow = deepest_wide <= TADP_WIDE_DEPTH;
     // candidate shapes (TA, UB), widest first; 16 values per thread need the shallow stack
     struct Shape { int ta, ub; };
     std::vector<Shape> shapes;
@@ -841,10 +1007,60 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
         for (const Shape &sh : shapes) if (items_for(sh) >= target_warps) { pick = sh; break; }
     }
     k.vec = pick.ta; k.vec_u = pick.ub;
+    std::vector<TadpBody> bodies;
+    if (can_fuse) {
+        if (pick.ta * pick.ub >= 16) { em.code = trial.code; em.depth_at = trial.depth_at; bodies = bodies_wide; }
+        else fuse_inner_loops(em, bodies, TADP_MAX_DEPTH - 1);
+    }
+    for (TadpBody &B : bodies)
+        for (int i = 0; i < TADP_BODY_STEPS; ++i)
+            if (B.steps[i] & 0x80) B.steps[i] |= (uint8_t)(body_fetch_kind(prog.loads[B.load[B.steps[i] & 3]], pick.ta, pick.ub) << 4);
+    prog.n_bodies = (int32_t)bodies.size();
+    std::copy(bodies.begin(), bodies.end(), prog.bodies);
+    prog.n_code = (int32_t)em.code.size();
+    std::copy(em.code.begin(), em.code.end(), prog.code);
     char head[256];
     std::snprintf(head, sizeof head, "; vars=%zu outer=%d kappa=%d lane_var=%d unroll_var=%d vec=%dx%d zsplit=%d temps=%d max_depth=%d loads=%d rows=%d guards=%d\n",
                   g.vars.size(), g.n_outer, g.kappa, g.lane_var, g.unroll_var, k.vec, k.vec_u, prog.zsplit, n_temps, em.max_depth, prog.n_loads, prog.n_rows, prog.n_guards);
-    k.listing = head + em.listing;
+    k.listing = head + em.listing();
+    // tables the code refers to: variables, loads, loops, bound rows
+    auto coefs = [&](const int32_t *c) {
+        std::string t;
+        for (int v = 0; v < (int)g.vars.size() && v < TADP_MAX_VARS; ++v) { char b2[24]; std::snprintf(b2, sizeof b2, " %d", c[v]); t += b2; }
+        return t;
+    };
+    char line[256];
+    for (int v = 0; v < (int)g.vars.size(); ++v) {
+        std::snprintf(line, sizeof line, "; var %d kind=%d ext=%lld\n", v, g.vars[v].kind, (long long)g.vars[v].ext);
+        k.listing += line;
+    }
+    for (int i = 0; i < prog.n_loads; ++i) {
+        std::snprintf(line, sizeof line, "; load %d ptr=%d base=%d coef=[%s ]\n", i, prog.loads[i].ptr, prog.loads[i].base, coefs(prog.loads[i].coef).c_str());
+        k.listing += line;
+    }
+    for (int i = 0; i < prog.n_loops; ++i) {
+        const TadpLoop &L = prog.loops[i];
+        std::snprintf(line, sizeof line, "; loop %d var=%d lane=%d split=%d relative=%d lane_dependent=%d const=[%d,%d] lower=%d+%d upper=%d+%d\n", i, L.var, L.is_lane,
+                      L.is_split, L.is_relative, L.depends_on_lane, L.const_lo, L.const_hi, L.lower0, L.n_lower, L.upper0, L.n_upper);
+        k.listing += line;
+    }
+    for (int i = 0; i < prog.n_bodies; ++i) {
+        const TadpBody &B = prog.bodies[i];
+        std::string t;
+        for (int q = 0; q < TADP_BODY_STEPS && B.steps[q]; ++q) {
+            char b2[40];
+            if (B.steps[q] & 0x80) std::snprintf(b2, sizeof b2, " ld%d(load %d fetch %d op %d)", B.steps[q] & 3, B.load[B.steps[q] & 3], (B.steps[q] >> 4) & 7, (B.steps[q] >> 2) & 3);
+            else std::snprintf(b2, sizeof b2, " s%d", B.steps[q]);
+            t += b2;
+        }
+        std::snprintf(line, sizeof line, "; body %d loop_kind=%d term=%d inv=(%d:%d,%d:%d) steps:%s\n", i, B.loop_kind, B.term, B.inv_kind[0], B.inv_value[0],
+                      B.inv_kind[1], B.inv_value[1], t.c_str());
+        k.listing += line;
+    }
+    for (int i = 0; i < prog.n_rows; ++i) {
+        std::snprintf(line, sizeof line, "; row %d (%d +%s ) / %d\n", i, prog.rows[i].c0, coefs(prog.rows[i].coef).c_str(), prog.rows[i].den);
+        k.listing += line;
+    }
 }
 
 }  // namespace

@@ -54,6 +54,9 @@ enum TadpOp : int {
     P_USEND,
     P_ZLOOP,      // kernel-coordinate loop begin: loops[a]; computes the range from its bound rows
     P_ZEND,       // kernel-coordinate loop end
+    P_XLOOP,      // every trip of an innermost loop in one word: runs bodies[imm] (a short accumulator program) and the
+                  // loop end of loops[a]; follows the loop begin word; k = 1: the loop is a value sum whose accumulator
+                  // is the bottom of the operand stack, k = 0: its terms go to the gradient accumulator
     P_NUM_OPS
 };
 
@@ -94,6 +97,35 @@ struct TadpLoop {
     int32_t is_relative;               // 1: every element walks its own short range, trip r visits lo_e + r
 };
 
+// Body of a fused innermost loop: an accumulator program over two value registers X and Y and up
+// to two loop-invariant values I0, I1.  One byte per step, at most TADP_BODY_STEPS steps, 0 ends.
+//   load step   1 kkk cc jj : v = load through slot jj fetched in manner kkk (TadpBodyFetch);
+//                             cc = 0: X <- v, 1: X <- X + v, 2: X <- X * v, 3: X <- (X + v)^2
+//   other steps 0 xxxxxxx   : TadpBodyStep
+// After the steps the term goes to the sum:  TERM_X: S += X,  TERM_XY: S += Y * X.
+#define TADP_BODY_STEPS 8
+#define TADP_BODY_LOADS 4
+#define TADP_MAX_BODIES 4
+enum TadpBodyFetch : int { BF_EACH = 0, BF_ONE, BF_PER_T, BF_PER_U, BF_ROW };
+enum TadpBodyStep : int {
+    BS_END = 0, BS_PUSH,            // Y <- X
+    BS_NEG, BS_SQR, BS_CUBE,        // X <- op X
+    BS_ADDY, BS_SUBY, BS_MULY, BS_DIVY,   // X <- Y op X
+    BS_LDI0, BS_LDI1,               // X <- I
+    BS_MULI0, BS_MULI1, BS_ADDI0, BS_ADDI1,   // X <- X op I
+    BS_FMAYI0, BS_FMAYI1            // X <- Y * I + X
+};
+enum TadpBodyLoopKind : int { BL_SUM = 0, BL_USUM, BL_Z, BL_Z_MASKED, BL_Z_LANE };
+struct alignas(8) TadpBody {
+    uint8_t steps[TADP_BODY_STEPS];
+    uint8_t load[TADP_BODY_LOADS];     // load descriptor of every slot
+    int32_t n_loads;
+    int32_t loop_kind;                 // TadpBodyLoopKind
+    int32_t term;                      // 0: S += X, 1: S += Y * X
+    int32_t inv_kind[2];               // 0 unused, 1 constant (inv_value), 2 temporary (inv_value = its number)
+    int32_t inv_value[2];
+};
+
 struct alignas(16) TadpProgram {
     int32_t n_code, n_loads, n_loops, n_rows;
     int32_t n_outer;                   // outer variables 0 .. n_outer-1 (decoded from the work item)
@@ -116,6 +148,8 @@ struct alignas(16) TadpProgram {
     TadpLoad loads[TADP_MAX_LOADS];
     TadpLoop loops[TADP_MAX_LOOPS];
     TadpRow rows[TADP_MAX_ROWS];
+    int32_t n_bodies;
+    TadpBody bodies[TADP_MAX_BODIES];
 };
 
 struct TadpPointers {

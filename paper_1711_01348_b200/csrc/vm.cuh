@@ -280,13 +280,14 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
         TADV_D3(TADV_FMA, P_FMA)
 
 #define TADV_TEMP_CASE(KK, STMT_REG, STMT_SPILL) case KK: if constexpr (KK < NTR) { constexpr int K = KK; STMT_REG } else { const int K = KK - NTR; STMT_SPILL } break;
-#define TADV_TEMP_SWITCH(STMT_REG, STMT_SPILL) \
-            switch (a) { \
+#define TADV_TEMP_SWITCH(STMT_REG, STMT_SPILL) TADV_TEMP_SWITCH_ON(a, STMT_REG, STMT_SPILL)
+#define TADV_TEMP_SWITCH_ON(SEL, STMT_REG, STMT_SPILL) \
+            switch (SEL) { \
             TADV_TEMP_CASE(0, STMT_REG, STMT_SPILL) TADV_TEMP_CASE(1, STMT_REG, STMT_SPILL) \
             TADV_TEMP_CASE(2, STMT_REG, STMT_SPILL) TADV_TEMP_CASE(3, STMT_REG, STMT_SPILL) \
             TADV_TEMP_CASE(4, STMT_REG, STMT_SPILL) TADV_TEMP_CASE(5, STMT_REG, STMT_SPILL) \
             TADV_TEMP_CASE(6, STMT_REG, STMT_SPILL) TADV_TEMP_CASE(7, STMT_REG, STMT_SPILL) \
-            default: { const int K = a - NTR; STMT_SPILL } break; }
+            default: { const int K = (SEL) - NTR; STMT_SPILL } break; }
 #define TADV_LDT(OP, D) TADV_CASE(OP, D, D + 1) { TADV_TEMP_SWITCH( \
             _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D][t] = op_mov(m.tmp[K][t]);, \
             _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D][t] = spill[K][t];) } break;
@@ -439,6 +440,163 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                 cur = parent; \
                 if (REL && L.is_relative) { _Pragma("unroll") for (int t = 0; t < T; ++t) zrel(t) = 0; set_var(m.var, V, 0); } \
             } }
+        // ---- fused innermost loop: all trips of the loop run here, without a dispatch per word ----
+        // X = s[SUMMODE], Y = s[SUMMODE + 1], invariants in the two topmost stack registers; a value sum
+        // accumulates into s[0], a gradient loop into acc.  Load offsets advance by a fixed step per trip.
+#define TADV_XSTEP(CODE, EXPR) case CODE: { _Pragma("unroll") for (int t = 0; t < T; ++t) { const float x = m.s[XI][t]; const float y = m.s[YI][t]; (void)y; m.s[XI][t] = (EXPR); } } break;
+#define TADV_XC_SET(t, x) m.s[XI][t] = (x);
+#define TADV_XC_ADD(t, x) m.s[XI][t] += (x);
+#define TADV_XC_MUL(t, x) m.s[XI][t] *= (x);
+#define TADV_XC_ADDSQ(t, x) { const float w2 = m.s[XI][t] + (x); m.s[XI][t] = w2 * w2; }
+        // fetches one load of the body in the manner the host chose and hands every element's value to COMBINE;
+        // ALL: every element of the thread is live (no predicates, signed 64-bit addressing from element 0)
+#define TADV_XFETCH(COMBINE, ALL) \
+                            switch (fk) { \
+                            case BF_ONE: { \
+                                const float x = (ALL || cur) ? __ldg(base + off) : 0.f; \
+                                _Pragma("unroll") for (int t = 0; t < T; ++t) { COMBINE(t, x) } \
+                            } break; \
+                            case BF_PER_T: if constexpr (UB > 1) { \
+                                _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { \
+                                    const unsigned mm = ALL ? 1u : (cur >> (ta * UB)) & ((1u << UB) - 1u); \
+                                    const unsigned idx = off + (unsigned)ta * lc; \
+                                    const float x = mm ? __ldg(base + idx) : 0.f; \
+                                    _Pragma("unroll") for (int u = 0; u < UB; ++u) { COMBINE(ta * UB + u, x) } \
+                                } \
+                            } break; \
+                            case BF_PER_U: if constexpr (UB > 1) { \
+                                _Pragma("unroll") for (int u = 0; u < UB; ++u) { \
+                                    unsigned mm = ALL ? 1u : 0u; \
+                                    if (!ALL) { _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) mm |= (cur >> (ta * UB + u)) & 1u; } \
+                                    const unsigned idx = off + (unsigned)u * uc; \
+                                    const float x = mm ? __ldg(base + idx) : 0.f; \
+                                    _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { COMBINE(ta * UB + u, x) } \
+                                } \
+                            } break; \
+                            case BF_ROW: if constexpr (UB > 1 && UB % 4 == 0) { \
+                                if ((reinterpret_cast<uintptr_t>(base) & 15u) == 0) { \
+                                    _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { \
+                                        const unsigned ob = off + (unsigned)ta * lc; \
+                                        _Pragma("unroll") for (int g4 = 0; g4 < UB / 4; ++g4) { \
+                                            const unsigned mm = ALL ? 0xfu : (cur >> (ta * UB + 4 * g4)) & 0xfu; \
+                                            float q[4]; \
+                                            if (mm == 0xfu && ((ob + 4u * g4) & 3u) == 0) { \
+                                                const float4 f4 = __ldg(reinterpret_cast<const float4 *>(base + (ob + 4u * g4))); \
+                                                q[0] = f4.x; q[1] = f4.y; q[2] = f4.z; q[3] = f4.w; \
+                                            } else { \
+                                                _Pragma("unroll") for (int i = 0; i < 4; ++i) q[i] = ((mm >> i) & 1u) ? __ldg(base + (ob + 4u * g4 + i)) : 0.f; \
+                                            } \
+                                            _Pragma("unroll") for (int i = 0; i < 4; ++i) { COMBINE(ta * UB + 4 * g4 + i, q[i]) } \
+                                        } \
+                                    } \
+                                    break; \
+                                } \
+                            } \
+                            [[fallthrough]]; \
+                            default: \
+                                if (ALL) { \
+                                    const float *p0 = base + off; \
+                                    _Pragma("unroll") for (int t = 0; t < T; ++t) { const float x = __ldg(p0 + ((t / UB) * (int)lc + (t % UB) * (int)uc)); COMBINE(t, x) } \
+                                } else { \
+                                    _Pragma("unroll") for (int t = 0; t < T; ++t) { const unsigned idx = off + (unsigned)(t / UB) * lc + (unsigned)(t % UB) * uc; const float x = ((cur >> t) & 1u) ? __ldg(base + idx) : 0.f; COMBINE(t, x) } \
+                                } \
+                                break; \
+                            }
+        // the steps of one trip and the term that closes it
+#define TADV_XTRIP(SUMMODE, ALL) { \
+                unsigned w0 = steps.x, w1 = steps.y; \
+                for (;;) { \
+                    const unsigned c = w0 & 0xffu; \
+                    if (c == 0) break; \
+                    w0 = __funnelshift_r(w0, w1, 8); w1 >>= 8; \
+                    if (c & 0x80u) { \
+                        const unsigned j = c & 3u, cmb = (c >> 2) & 3u, fk = (c >> 4) & 7u; \
+                        const unsigned off = TADV_XSEL(j, xo); \
+                        const unsigned lc = TADV_XSEL(j, xlc); \
+                        const unsigned uc = TADV_XSEL(j, xuc); \
+                        const float *base = TADV_XSEL(j, xbase); \
+                        switch (cmb) { \
+                        case 0: TADV_XFETCH(TADV_XC_SET, ALL) break; \
+                        case 1: TADV_XFETCH(TADV_XC_ADD, ALL) break; \
+                        case 2: TADV_XFETCH(TADV_XC_MUL, ALL) break; \
+                        default: TADV_XFETCH(TADV_XC_ADDSQ, ALL) break; \
+                        } \
+                    } else { \
+                        switch (c) { \
+                        case BS_PUSH: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[YI][t] = m.s[XI][t]; } break; \
+                        TADV_XSTEP(BS_NEG, -x) TADV_XSTEP(BS_SQR, x * x) TADV_XSTEP(BS_CUBE, x * x * x) \
+                        TADV_XSTEP(BS_ADDY, y + x) TADV_XSTEP(BS_SUBY, y - x) TADV_XSTEP(BS_MULY, y * x) TADV_XSTEP(BS_DIVY, y / x) \
+                        TADV_XSTEP(BS_LDI0, m.s[I0][t]) TADV_XSTEP(BS_LDI1, m.s[I1][t]) \
+                        TADV_XSTEP(BS_MULI0, x * m.s[I0][t]) TADV_XSTEP(BS_MULI1, x * m.s[I1][t]) \
+                        TADV_XSTEP(BS_ADDI0, x + m.s[I0][t]) TADV_XSTEP(BS_ADDI1, x + m.s[I1][t]) \
+                        TADV_XSTEP(BS_FMAYI0, fmaf(y, m.s[I0][t], x)) \
+                        default: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[XI][t] = fmaf(m.s[YI][t], m.s[I1][t], m.s[XI][t]); } break; \
+                        } \
+                    } \
+                } \
+                if (SUMMODE) { \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) if (ALL || UB == 1 || ((cur >> t) & 1u)) \
+                        m.s[0][t] = term ? fmaf(m.s[YI][t], m.s[XI][t], m.s[0][t]) : m.s[0][t] + m.s[XI][t]; \
+                } else { \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) if (ALL || ((cur >> t) & 1u)) \
+                        m.acc[t] = term ? fmaf(m.s[YI][t], m.s[XI][t], m.acc[t]) : m.acc[t] + m.s[XI][t]; \
+                    live |= cur; \
+                } }
+#define TADV_XSEL(j, A) ((j) == 0 ? A[0] : (j) == 1 ? A[1] : (j) == 2 ? A[2] : A[3])
+#define TADV_XLOOP(SUMMODE) case TADV_H(P_XLOOP, SUMMODE): if constexpr (!DEBUG && !REL && (SUMMODE) + 2 <= VmCfg<TA, UB>::DEPTH) { \
+            constexpr int DEPTH = VmCfg<TA, UB>::DEPTH; \
+            constexpr int XI = (SUMMODE), YI = XI + 1, I0 = DEPTH - 1, I1 = DEPTH >= 2 ? DEPTH - 2 : 0; \
+            const TadpBody &B = P.bodies[imm]; \
+            const TadpLoop &L = P.loops[a]; \
+            const int V = L.var; \
+            const int kind = B.loop_kind; \
+            _Pragma("unroll") for (int q = 0; q < 2; ++q) { \
+                const int ik = B.inv_kind[q]; \
+                if (ik == 1) { const float c = __int_as_float(B.inv_value[q]); _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[q ? I1 : I0][t] = c; } \
+                else if (ik == 2) { const int tsel = B.inv_value[q]; TADV_TEMP_SWITCH_ON(tsel, \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[q ? I1 : I0][t] = m.tmp[K][t];, \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[q ? I1 : I0][t] = spill[K][t];) } \
+            } \
+            int z = get_var(m.var, V); \
+            const int lane = (int)(threadIdx.x & 31u); \
+            const int dz = kind == BL_USUM ? UB : kind == BL_Z_LANE ? 32 * TA : 1; \
+            const int hi = kind <= BL_USUM ? L.const_hi : loop_hi[a]; \
+            const int lvl = L.mask_level; \
+            const unsigned parent = kind == BL_SUM ? cur : kind == BL_USUM ? sum_parent : mstack[lvl - 1]; \
+            /* per load slot: offset of this thread's element 0, its step per trip, pointer and element strides */ \
+            unsigned xo[TADP_BODY_LOADS], xst[TADP_BODY_LOADS], xlc[TADP_BODY_LOADS], xuc[TADP_BODY_LOADS]; \
+            const float *xbase[TADP_BODY_LOADS]; \
+            _Pragma("unroll") for (int j = 0; j < TADP_BODY_LOADS; ++j) { \
+                const TadpLoad &Ld = P.loads[B.load[j < B.n_loads ? j : 0]]; \
+                xo[j] = load_offset(Ld, m.var); xst[j] = (unsigned)Ld.coef[V] * (unsigned)dz; \
+                xlc[j] = (unsigned)Ld.lane_step; xuc[j] = UB > 1 ? (unsigned)Ld.unroll_step : 0u; \
+                xbase[j] = ptrs.in[Ld.ptr]; \
+            } \
+            const uint2 steps = *reinterpret_cast<const uint2 *>(B.steps); \
+            const int term = B.term; \
+            constexpr unsigned FULL = T >= 32 ? 0xffffffffu : ((1u << T) - 1u); \
+            for (;;) { \
+                if (cur == FULL) TADV_XTRIP(SUMMODE, true) else TADV_XTRIP(SUMMODE, false) \
+                z += dz; \
+                const int zb = kind == BL_Z_LANE ? z - lane : z; \
+                if (zb > hi) break; \
+                _Pragma("unroll") for (int j = 0; j < TADP_BODY_LOADS; ++j) xo[j] += xst[j]; \
+                if (kind == BL_Z_MASKED) { \
+                    unsigned mk = 0; \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) if (elo[lvl - 1][t] <= z && z <= ehi[lvl - 1][t]) mk |= 1u << t; \
+                    cur = parent & mk; \
+                } else if (zb + dz - 1 > hi) {   /* last trip of a loop that advances by more than one */ \
+                    unsigned mk = 0; \
+                    if (kind == BL_USUM) { _Pragma("unroll") for (int t = 0; t < T; ++t) if (z + (t % UB) <= hi) mk |= 1u << t; } \
+                    else { _Pragma("unroll") for (int t = 0; t < T; ++t) if (z + 32 * (t / UB) <= hi) mk |= 1u << t; } \
+                    cur = parent & mk; \
+                } \
+            } \
+            cur = parent; \
+        } break;
+        TADV_XLOOP(0)
+        TADV_XLOOP(1)
+
         default: {
             const int op = (raw.x & 0xffffu) >> 3;
             if (op == P_ZLOOP) TADV_ZLOOP_BODY

@@ -40,6 +40,27 @@ def test_small_expressions(name):
     check_against_oracle(e, args, df)
 
 
+# Sizes at which the compiler picks its wide vector shapes (2x8, 1x8, 1x4, 16x1 values per thread),
+# split summations and fused inner loops, with extents that leave a ragged tail in every direction.
+MID = {
+    "intro_mid": (lambda: W.intro(300, 333, 11), ("uniform", -0.5, 0.5)),
+    "intro_wide": (lambda: W.intro(130, 1000, 21), ("uniform", -0.5, 0.5)),
+    "matmul_t": (lambda: W.ex_matmul_t(70, 100, 37), ("normal", 0, 1)),
+    "rowsum_sq": (lambda: W.ex_rowsum_sq(1000, 37), ("normal", 0, 1)),
+    "rowsum_sq_short": (lambda: W.ex_rowsum_sq(333, 9), ("normal", 0, 1)),
+    "conv_mid": (lambda: W.conv1d(3, 20, 24, 300, 5), ("normal", 0, 0.1)),
+    "matmul_mid": (lambda: W.ex_matmul(150, 67, 1100), ("normal", 0, 1)),
+}
+
+
+@pytest.mark.parametrize("name", sorted(MID))
+def test_mid_size_expressions(name):
+    make, dist = MID[name]
+    e = make()
+    args, df = W.make_inputs(e, dist, seed=1)
+    check_against_oracle(e, args, df, nthreads=max_threads())
+
+
 @pytest.mark.parametrize("key", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
 def test_reduced_workloads(key):
     """Same structure as the full workloads, several tiles and ragged tails, full oracle run."""

@@ -194,6 +194,25 @@ def ex_matmul(ni: int, nk: int, nj: int) -> Expr:
     return b.done()
 
 
+def ex_matmul_t(ni: int, nj: int, nk: int) -> Expr:
+    """f_ij = sum_k x_ik y_jk: the matrix product of Sec. 5 with the second factor stored transposed,
+    so that its rows are read along the summation index."""
+    b = Builder("ex_matmul_t", [ni, nj], 1, ["x", "y"], [[ni, nk], [nj, nk]])
+    x = b.load("x", [unit(3, (0, 1)), unit(3, (2, 1))])
+    y = b.load("y", [unit(3, (1, 1)), unit(3, (2, 1))])
+    b.sum(2, 0, nk - 1, b.bin("mul", x, y))
+    return b.done()
+
+
+def ex_rowsum_sq(n: int, nk: int) -> Expr:
+    """f_j = sum_k (y_jk)^2 + w_k: every output sums along a row of y."""
+    b = Builder("ex_rowsum_sq", [n], 1, ["y", "w"], [[n, nk], [nk]])
+    y = b.load("y", [unit(2, (0, 1)), unit(2, (1, 1))])
+    w = b.load("w", [unit(2, (1, 1))])
+    b.sum(1, 0, nk - 1, b.bin("add", b.powi(y, 2), w))
+    return b.done()
+
+
 def ex_exp_flat(n: int, m: int) -> Expr:
     """f^5_ij = exp x_{M i + j}, i in [0, n), j in [0, m)  (Sec. 5)."""
     b = Builder("ex_exp_flat", [n, m], 0, ["x"], [[n * m]])
