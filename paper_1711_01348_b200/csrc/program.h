@@ -5,6 +5,7 @@
 #pragma once
 #include <stdint.h>
 
+#define TADP_WARPS_PER_BLOCK 8
 #define TADP_MAX_VARS 8       // loop variables of one kernel: outer + kernel coordinates + bound sums
 #define TADP_MAX_CODE 320     // 8-byte instruction words
 #define TADP_MAX_LOADS 20

@@ -8,159 +8,20 @@
 #include <string>
 
 #include "plan.h"
-#include "vm.cuh"
+#include "program.h"
+#include "vm_shapes.h"
 
 namespace tad {
 void set_error(const std::string &m);
 }
 
+// One build of the interpreter per vector shape, each in an object file of its own (vm_inst.cu).
+#define TAD_DECLARE_VM(TA, UB) void tad_launch_vm_##TA##_##UB(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned blocks, cudaStream_t stream);
+TAD_VM_SHAPES(TAD_DECLARE_VM)
+
 namespace {
 
-using namespace tadvm;
-
-// One warp per work item, grid-stride over the items.  A work item fixes every outer variable
-// except the lane variable A, which the warp covers 32 * TA values at a time, and the element
-// variable B when that is an outer variable, which it covers UB values at a time.
-template <int TA, int UB, bool DEBUG, bool REL>
-__global__ void __launch_bounds__(WARPS_PER_BLOCK * 32, 2)
-tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ TadpPointers ptrs, unsigned n_items)
-{
-    constexpr int E = TA * UB;
-    const unsigned lane = threadIdx.x & 31u;
-    const unsigned warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const unsigned n_warps = (gridDim.x * blockDim.x) >> 5;
-    const int lane_var = P.lane_var;
-    const int unroll_var = P.unroll_var;
-    const bool lane_outer = lane_var < P.n_outer;
-    const bool unroll_outer = UB > 1 && P.unroll_kind == 1;
-    Vm<TA, UB> m;
-    const unsigned zsplit = P.zsplit > 1 ? (unsigned)P.zsplit : 1u;
-    for (unsigned witem = warp; witem < n_items; witem += n_warps) {
-        // warps witem = item * zsplit + s share the outputs of `item`
-        const unsigned item = witem / zsplit;
-        const int split = (int)(witem % zsplit);
-        // decode the outer variables (last one fastest)
-        unsigned rem = item;
-#pragma unroll
-        for (int k = 0; k < TADP_MAX_VARS; ++k) m.var[k] = 0;
-        unsigned first_a = 0, ext_a = 0xffffffffu, first_b = 0, ext_b = 0xffffffffu;
-#pragma unroll
-        for (int v = TADP_MAX_VARS - 1; v >= 0; --v) {
-            if (v < P.n_outer) {
-                const unsigned ext = (unsigned)P.outer_ext[v];
-                if (v == lane_var) {
-                    const unsigned chunks = (ext + 32u * TA - 1u) / (32u * TA);
-                    const unsigned c = rem % chunks; rem /= chunks;
-                    first_a = c * 32u * TA + lane; ext_a = ext;
-                    m.var[v] = P.outer_lo[v] + (int)first_a;
-                } else if (unroll_outer && v == unroll_var) {
-                    const unsigned chunks = (ext + UB - 1u) / UB;
-                    const unsigned c = rem % chunks; rem /= chunks;
-                    first_b = c * UB; ext_b = ext;
-                    m.var[v] = P.outer_lo[v] + (int)first_b;
-                } else {
-                    const unsigned c = rem % ext; rem /= ext;
-                    m.var[v] = P.outer_lo[v] + (int)c;
-                }
-            }
-        }
-        unsigned mask0 = 0;
-#pragma unroll
-        for (int e = 0; e < E; ++e)
-            if (first_a + 32u * (e / UB) < ext_a && first_b + (unsigned)(e % UB) < ext_b) mask0 |= 1u << e;
-        const unsigned in_range = mask0;
-        // guards: rows over the outer variables that must be <= 0 for Gamma to be non-empty
-        for (int r = 0; r < P.n_guards; ++r) {
-            const TadpRow &R = P.rows[P.guard0 + r];
-            const int nmr = row_num(R, m.var);
-            const int sa = lane_outer ? R.coef[lane_var] * 32 : 0;
-            const int sb = unroll_outer ? R.coef[unroll_var] : 0;
-#pragma unroll
-            for (int e = 0; e < E; ++e) if (nmr + (e / UB) * sa + (e % UB) * sb > 0) mask0 &= ~(1u << e);
-        }
-        unsigned live = 0;
-        run_item<TA, UB, DEBUG, REL>(P, ptrs, m, mask0, split, live);
-
-        // ---- output: distinct elements along t when A is an outer variable, along u when B is ----
-        const int n_u = unroll_outer ? UB : 1;
-        unsigned off = (unsigned)P.out_base;
-#pragma unroll
-        for (int k = 0; k < TADP_MAX_VARS; ++k) if (k < P.n_outer) off += (unsigned)P.out_coef[k] * (unsigned)m.var[k];
-        const unsigned step_a = lane_outer ? (unsigned)P.out_coef[lane_var] * 32u : 0u;
-        const unsigned step_b = unroll_outer ? (unsigned)P.out_coef[unroll_var] : 0u;
-        if (zsplit > 1) {
-            // this warp's share of the sums goes to its plane of partial sums, indexed compactly
-            // by the outer variables; a second launch adds the planes up in order
-            unsigned cidx = 0;
-#pragma unroll
-            for (int k = 0; k < TADP_MAX_VARS; ++k) if (k < P.n_outer) cidx += (unsigned)P.part_coef[k] * (unsigned)(m.var[k] - P.outer_lo[k]);
-            const unsigned cstep_a = lane_outer ? (unsigned)P.part_coef[lane_var] * 32u : 0u;
-            const unsigned cstep_b = unroll_outer ? (unsigned)P.part_coef[unroll_var] : 0u;
-            float *plane = ptrs.part + (size_t)split * (unsigned)P.part_limit;
-            float *flags = ptrs.part + (size_t)zsplit * (unsigned)P.part_limit;
-            if (lane_outer) {
-#pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    if ((e % UB) >= n_u || !((in_range >> e) & 1u)) continue;
-                    const unsigned c = cidx + (unsigned)(e / UB) * cstep_a + (unsigned)(e % UB) * cstep_b;
-                    plane[c] = m.acc[e];
-                    if ((live >> e) & 1u) flags[c] = 1.f;
-                }
-            } else {
-#pragma unroll
-                for (int u = 0; u < UB; ++u) {
-                    if (u >= n_u) continue;
-                    float total = 0.f;
-                    unsigned lv = 0;
-#pragma unroll
-                    for (int t = 0; t < TA; ++t) { total += m.acc[t * UB + u]; lv |= (live >> (t * UB + u)) & 1u; }
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
-                    const unsigned any_live = __ballot_sync(0xffffffffu, lv != 0);
-                    if (lane == 0 && first_b + (unsigned)u < ext_b) {
-                        const unsigned c = cidx + (unsigned)u * cstep_b;
-                        plane[c] = total;
-                        if (any_live) flags[c] = 1.f;
-                    }
-                }
-            }
-            continue;
-        }
-        float *dst = ptrs.out;
-        const bool accumulate = P.accumulate != 0;
-        const bool only_live = P.write_only_live != 0;
-        if (lane_outer) {
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-                if ((e % UB) >= n_u) continue;
-                if (!((in_range >> e) & 1u)) continue;
-                if (only_live && !((live >> e) & 1u)) continue;
-                const unsigned idx = off + (unsigned)(e / UB) * step_a + (unsigned)(e % UB) * step_b;
-                if (DEBUG && idx >= (unsigned)P.out_limit) { if (ptrs.debug) atomicCAS(ptrs.debug, 0, 0x20000); continue; }
-                dst[idx] = accumulate ? dst[idx] + m.acc[e] : m.acc[e];
-            }
-        } else {
-            // the lane variable is a kernel coordinate: fixed-order tree reduction over t and the lanes
-#pragma unroll
-            for (int u = 0; u < UB; ++u) {
-                if (u >= n_u) continue;
-                float total = 0.f;
-                unsigned lv = 0;
-#pragma unroll
-                for (int t = 0; t < TA; ++t) { total += m.acc[t * UB + u]; lv |= (live >> (t * UB + u)) & 1u; }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
-                const unsigned any_live = __ballot_sync(0xffffffffu, lv != 0);
-                const bool inside = first_b + (unsigned)u < ext_b;
-                if (lane == 0 && inside && !(only_live && !any_live)) {
-                    const unsigned idx = off + (unsigned)u * step_b;
-                    if (DEBUG && idx >= (unsigned)P.out_limit) { if (ptrs.debug) atomicCAS(ptrs.debug, 0, 0x20000); }
-                    else dst[idx] = accumulate ? dst[idx] + total : total;
-                }
-            }
-        }
-    }
-}
+constexpr int WARPS_PER_BLOCK = TADP_WARPS_PER_BLOCK;
 
 // Adds the zsplit planes of partial sums up in plane order and writes the gradient elements:
 // compact index c -> outer variables -> output offset.  Masked gradients write only outputs
@@ -211,16 +72,6 @@ unsigned long long item_count(const TadpProgram &P, int ta, int ub)
     return n;
 }
 
-// Builds of the interpreter per vector shape: plain, with the relative-loop support and (narrow
-// shapes only) with bounds checks.
-template <int TA, int UB>
-void launch_t(const tad::Kernel &k, const TadpPointers &ptrs, bool debug, unsigned items, unsigned blocks, cudaStream_t stream)
-{
-    if (debug) { if constexpr (TA <= 4 && UB == 1) tad_vm_kernel<TA, UB, true, true><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items); }
-    else if (k.prog.rel_var >= 0) { if constexpr (UB == 1) tad_vm_kernel<TA, UB, false, true><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items); }
-    else tad_vm_kernel<TA, UB, false, false><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(k.prog, ptrs, items);
-}
-
 tad_status zero_fill(float *out, int64_t n, cudaStream_t stream);
 
 tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStream_t stream)
@@ -242,15 +93,8 @@ tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStrea
     const unsigned max_blocks = (unsigned)sm_count() * 16u;
     const unsigned blocks = std::min(blocks_needed, max_blocks);
     switch (k.vec * 100 + k.vec_u) {
-    case 101: launch_t<1, 1>(k, ptrs, debug, items, blocks, stream); break;
-    case 201: launch_t<2, 1>(k, ptrs, debug, items, blocks, stream); break;
-    case 401: launch_t<4, 1>(k, ptrs, debug, items, blocks, stream); break;
-    case 801: launch_t<8, 1>(k, ptrs, debug, items, blocks, stream); break;
-    case 1601: launch_t<16, 1>(k, ptrs, debug, items, blocks, stream); break;
-    case 104: launch_t<1, 4>(k, ptrs, debug, items, blocks, stream); break;
-    case 108: launch_t<1, 8>(k, ptrs, debug, items, blocks, stream); break;
-    case 208: launch_t<2, 8>(k, ptrs, debug, items, blocks, stream); break;
-    case 116: launch_t<1, 16>(k, ptrs, debug, items, blocks, stream); break;
+#define TAD_CASE_VM(TA, UB) case TA * 100 + UB: tad_launch_vm_##TA##_##UB(k.prog, ptrs, debug, items, blocks, stream); break;
+    TAD_VM_SHAPES(TAD_CASE_VM)
     default: tad::set_error("internal: no kernel for this vector shape"); return TAD_ERR_UNSUPPORTED;
     }
     cudaError_t e = cudaGetLastError();

@@ -20,7 +20,7 @@
 
 namespace tadvm {
 
-constexpr int WARPS_PER_BLOCK = 8;
+constexpr int WARPS_PER_BLOCK = TADP_WARPS_PER_BLOCK;
 constexpr int STACK = TADP_MAX_DEPTH - 1;   // usable depth (handlers are encoded for depth 0..7)
 
 __device__ __forceinline__ int floor_div_i(int a, int b) { int q = a / b; return (a % b != 0 && a < 0) ? q - 1 : q; }
@@ -37,7 +37,7 @@ __device__ __forceinline__ float op_neg(float x) { float r; asm volatile("neg.f3
 __device__ __forceinline__ float op_mov(float x) { float r; asm volatile("mov.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
 
 // One copy of every slow elementary function in the kernel image.
-__device__ __noinline__ float apply_fn(int fn, float x, int n)
+static __device__ __noinline__ float apply_fn(int fn, float x, int n)
 {
     switch (fn) {
     case F_EXP: return expf(x);
@@ -444,10 +444,10 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
         // X = s[SUMMODE], Y = s[SUMMODE + 1], invariants in the two topmost stack registers; a value sum
         // accumulates into s[0], a gradient loop into acc.  Load offsets advance by a fixed step per trip.
 #define TADV_XSTEP(CODE, EXPR) case CODE: { _Pragma("unroll") for (int t = 0; t < T; ++t) { const float x = m.s[XI][t]; const float y = m.s[YI][t]; (void)y; m.s[XI][t] = (EXPR); } } break;
-#define TADV_XC_SET(t, x) m.s[XI][t] = (x);
-#define TADV_XC_ADD(t, x) m.s[XI][t] += (x);
-#define TADV_XC_MUL(t, x) m.s[XI][t] *= (x);
-#define TADV_XC_ADDSQ(t, x) { const float w2 = m.s[XI][t] + (x); m.s[XI][t] = w2 * w2; }
+#define TADV_XC_SET(t, x) m.s[XI][t] = op_mov(x);
+#define TADV_XC_ADD(t, x) m.s[XI][t] = op_add(m.s[XI][t], (x));
+#define TADV_XC_MUL(t, x) m.s[XI][t] = op_mul(m.s[XI][t], (x));
+#define TADV_XC_ADDSQ(t, x) { const float w2 = op_add(m.s[XI][t], (x)); m.s[XI][t] = op_mul(w2, w2); }
         // fetches one load of the body in the manner the host chose and hands every element's value to COMBINE;
         // ALL: every element of the thread is live (no predicates, signed 64-bit addressing from element 0)
 #define TADV_XFETCH(COMBINE, ALL) \
@@ -523,23 +523,23 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                         } \
                     } else { \
                         switch (c) { \
-                        case BS_PUSH: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[YI][t] = m.s[XI][t]; } break; \
-                        TADV_XSTEP(BS_NEG, -x) TADV_XSTEP(BS_SQR, x * x) TADV_XSTEP(BS_CUBE, x * x * x) \
-                        TADV_XSTEP(BS_ADDY, y + x) TADV_XSTEP(BS_SUBY, y - x) TADV_XSTEP(BS_MULY, y * x) TADV_XSTEP(BS_DIVY, y / x) \
-                        TADV_XSTEP(BS_LDI0, m.s[I0][t]) TADV_XSTEP(BS_LDI1, m.s[I1][t]) \
-                        TADV_XSTEP(BS_MULI0, x * m.s[I0][t]) TADV_XSTEP(BS_MULI1, x * m.s[I1][t]) \
-                        TADV_XSTEP(BS_ADDI0, x + m.s[I0][t]) TADV_XSTEP(BS_ADDI1, x + m.s[I1][t]) \
-                        TADV_XSTEP(BS_FMAYI0, fmaf(y, m.s[I0][t], x)) \
-                        default: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[XI][t] = fmaf(m.s[YI][t], m.s[I1][t], m.s[XI][t]); } break; \
+                        case BS_PUSH: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[YI][t] = op_mov(m.s[XI][t]); } break; \
+                        TADV_XSTEP(BS_NEG, op_neg(x)) TADV_XSTEP(BS_SQR, op_mul(x, x)) TADV_XSTEP(BS_CUBE, op_mul(op_mul(x, x), x)) \
+                        TADV_XSTEP(BS_ADDY, op_add(y, x)) TADV_XSTEP(BS_SUBY, op_sub(y, x)) TADV_XSTEP(BS_MULY, op_mul(y, x)) TADV_XSTEP(BS_DIVY, y / x) \
+                        TADV_XSTEP(BS_LDI0, op_mov(m.s[I0][t])) TADV_XSTEP(BS_LDI1, op_mov(m.s[I1][t])) \
+                        TADV_XSTEP(BS_MULI0, op_mul(x, m.s[I0][t])) TADV_XSTEP(BS_MULI1, op_mul(x, m.s[I1][t])) \
+                        TADV_XSTEP(BS_ADDI0, op_add(x, m.s[I0][t])) TADV_XSTEP(BS_ADDI1, op_add(x, m.s[I1][t])) \
+                        TADV_XSTEP(BS_FMAYI0, op_fma(y, m.s[I0][t], x)) \
+                        default: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[XI][t] = op_fma(m.s[YI][t], m.s[I1][t], m.s[XI][t]); } break; \
                         } \
                     } \
                 } \
                 if (SUMMODE) { \
                     _Pragma("unroll") for (int t = 0; t < T; ++t) if (ALL || UB == 1 || ((cur >> t) & 1u)) \
-                        m.s[0][t] = term ? fmaf(m.s[YI][t], m.s[XI][t], m.s[0][t]) : m.s[0][t] + m.s[XI][t]; \
+                        m.s[0][t] = term ? op_fma(m.s[YI][t], m.s[XI][t], m.s[0][t]) : op_add(m.s[0][t], m.s[XI][t]); \
                 } else { \
                     _Pragma("unroll") for (int t = 0; t < T; ++t) if (ALL || ((cur >> t) & 1u)) \
-                        m.acc[t] = term ? fmaf(m.s[YI][t], m.s[XI][t], m.acc[t]) : m.acc[t] + m.s[XI][t]; \
+                        m.acc[t] = term ? op_fma(m.s[YI][t], m.s[XI][t], m.acc[t]) : op_add(m.acc[t], m.s[XI][t]); \
                     live |= cur; \
                 } }
 #define TADV_XSEL(j, A) ((j) == 0 ? A[0] : (j) == 1 ? A[1] : (j) == 2 ? A[2] : A[3])
