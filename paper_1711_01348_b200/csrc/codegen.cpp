@@ -996,10 +996,19 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
         // splitting costs a pass over zsplit planes: only when the outputs are too few to fill the GPU
         if (items_for(pick) < target_warps / 2 && cells <= (1 << 22)) {
             TadpLoop &L0 = prog.loops[em.code[zbegin[0]].a];
-            const int64_t ext0 = std::max<int64_t>(1, g.vars[L0.var].ext / (L0.is_lane ? 32 * pick.ta : 1));
-            int64_t S = (int64_t)std::ceil(target_warps / items_for(pick));
-            S = std::min<int64_t>(std::min<int64_t>(S, ext0), 4096);
-            while (S > 1 && (S + 1) * cells > (int64_t(1) << 25)) S /= 2;   // <= 128 MB of partial sums
+            auto splits_for = [&](const Shape &sh) {
+                const int64_t ext0 = std::max<int64_t>(1, g.vars[L0.var].ext / (L0.is_lane ? 32 * sh.ta : 1));
+                int64_t S = (int64_t)std::ceil(target_warps / items_for(sh));
+                S = std::min<int64_t>(std::min<int64_t>(S, ext0), 4096);
+                while (S > 1 && (S + 1) * cells > (int64_t(1) << 25)) S /= 2;   // <= 128 MB of partial sums
+                return S;
+            };
+            // when the loop is too short to give the widest shape enough shares, narrower shapes bring more warps
+            for (const Shape &sh : shapes) {
+                pick = sh;
+                if (items_for(sh) * (double)splits_for(sh) >= target_warps / 2) break;
+            }
+            const int64_t S = splits_for(pick);
             if (S >= 2) { prog.zsplit = (int32_t)S; prog.part_limit = to_i32(cells); L0.is_split = 1; }
         }
     } else {

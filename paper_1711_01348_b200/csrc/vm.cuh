@@ -367,15 +367,22 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                     const int rstep = rel_var >= 0 ? R.coef[rel_var] : 0; \
                     _Pragma("unroll") for (int t = 0; t < T; ++t) { int v = nmr + (t / UB) * step + (t % UB) * ustep + (REL && rstep ? rstep * zrel(t) : 0); v = R.den == 1 ? v : floor_div_i(v, R.den); ehi[lvl - 1][t] = min(ehi[lvl - 1][t], v); } \
                 } \
-                if (L.is_split) { \
-                    /* every element's own range is divided into zsplit contiguous shares */ \
-                    _Pragma("unroll") for (int t = 0; t < T; ++t) if (elo[lvl - 1][t] <= ehi[lvl - 1][t]) { \
-                        const int chunk = (ehi[lvl - 1][t] - elo[lvl - 1][t] + P.zsplit) / P.zsplit; \
-                        elo[lvl - 1][t] += split * chunk; ehi[lvl - 1][t] = min(ehi[lvl - 1][t], elo[lvl - 1][t] + chunk - 1); \
-                    } \
-                } \
                 _Pragma("unroll") for (int t = 0; t < T; ++t) \
                     if (((parent >> t) & 1u) && elo[lvl - 1][t] <= ehi[lvl - 1][t]) { lo_w = min(lo_w, elo[lvl - 1][t]); hi_w = max(hi_w, ehi[lvl - 1][t]); } \
+                if (L.is_split) { \
+                    /* the union of the warp's element ranges is divided into zsplit contiguous shares, the same for \
+                       every element, so that the elements of a share walk it together (fixed chunking: repeatable sums) */ \
+                    _Pragma("unroll") for (int o = 16; o > 0; o >>= 1) { lo_w = min(lo_w, __shfl_xor_sync(0xffffffffu, lo_w, o)); hi_w = max(hi_w, __shfl_xor_sync(0xffffffffu, hi_w, o)); } \
+                    if (lo_w <= hi_w) { \
+                        const int chunk = (hi_w - lo_w + P.zsplit) / P.zsplit; \
+                        const int slo = lo_w + split * chunk, shi = min(hi_w, slo + chunk - 1); \
+                        lo_w = INT_MAX; hi_w = INT_MIN; \
+                        _Pragma("unroll") for (int t = 0; t < T; ++t) { \
+                            elo[lvl - 1][t] = max(elo[lvl - 1][t], slo); ehi[lvl - 1][t] = min(ehi[lvl - 1][t], shi); \
+                            if (((parent >> t) & 1u) && elo[lvl - 1][t] <= ehi[lvl - 1][t]) { lo_w = min(lo_w, elo[lvl - 1][t]); hi_w = max(hi_w, ehi[lvl - 1][t]); } \
+                        } \
+                    } \
+                } \
                 if (REL && L.is_relative) { \
                     /* trip r visits lo_e + r: the warp runs as many trips as its longest element range */ \
                     int len = 0; \
