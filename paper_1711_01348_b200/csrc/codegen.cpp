@@ -431,6 +431,23 @@ struct Emitter {
             emit(P_ZERO, 0, 0, 0, +1);
             int begin = emit(over_elements ? P_USLOOP : P_SLOOP, id, 0, 0, 0, in.var);
             temps_of_sum(i);
+            const Inst inner = g.inst[in.a];
+            if (!over_elements && inner.op == I_SUM && inline_ok(in.a) && inner.var != g.unroll_var) {
+                // a sum whose summand is a sum: the inner loop adds its summands to the same accumulator
+                TadpLoop L2{};
+                L2.var = inner.var; L2.const_lo = (int32_t)inner.lo; L2.const_hi = (int32_t)inner.hi;
+                if ((int)loops.size() >= TADP_MAX_LOOPS) throw Unsupported("too many loops in one kernel");
+                loops.push_back(L2);
+                const int id2 = (int)loops.size() - 1;
+                const int ib = emit(P_SLOOP, id2, 0, 0, 0, inner.var);
+                temps_of_sum(in.a);
+                expr(inner.a);
+                const int ie = emit(P_SUMEND, id2, 0, ib + 1, -1);
+                code[ib].imm = ie + 1;
+                const int oe = emit(P_SEND, id, 0, begin + 1, 0, in.var);
+                code[begin].imm = oe + 1;
+                break;
+            }
             expr(in.a);
             int end;
             if (over_elements) {
@@ -954,7 +971,7 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     const bool debug = g.p.opt.debug_bounds != 0;
     // fused inner loops leave the operand stack to the rest of the program: try them with the
     // 4-deep stack of the 16-value variants first
-    const bool can_fuse = !debug && prog.rel_var < 0;
+    const bool can_fuse = !debug;
     Emitter trial(em);
     std::vector<TadpBody> bodies_wide;
     const int deepest_wide = can_fuse ? fuse_inner_loops(trial, bodies_wide, TADP_WIDE_DEPTH) : em.max_depth;
@@ -996,20 +1013,32 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
         // splitting costs a pass over zsplit planes: only when the outputs are too few to fill the GPU
         if (items_for(pick) < target_warps / 2 && cells <= (1 << 22)) {
             TadpLoop &L0 = prog.loops[em.code[zbegin[0]].a];
-            auto splits_for = [&](const Shape &sh) {
-                const int64_t ext0 = std::max<int64_t>(1, g.vars[L0.var].ext / (L0.is_lane ? 32 * sh.ta : 1));
-                int64_t S = (int64_t)std::ceil(target_warps / items_for(sh));
-                S = std::min<int64_t>(std::min<int64_t>(S, ext0), 4096);
-                while (S > 1 && (S + 1) * cells > (int64_t(1) << 25)) S /= 2;   // <= 128 MB of partial sums
-                return S;
+            // shares of the outermost loop first; when that loop is too short, the next one is divided too
+            // (share number s = s0 * S1 + s1)
+            TadpLoop *L1 = g.kappa >= 2 ? &prog.loops[em.code[zbegin[1]].a] : nullptr;
+            auto loop_trips = [&](const TadpLoop &L, const Shape &sh) {
+                return std::max<int64_t>(1, g.vars[L.var].ext / (L.is_lane ? 32 * sh.ta : 1));
             };
-            // when the loop is too short to give the widest shape enough shares, narrower shapes bring more warps
+            auto splits_for = [&](const Shape &sh, int64_t &S0, int64_t &S1) {
+                const int64_t want = (int64_t)std::ceil(target_warps / items_for(sh));
+                S0 = std::min<int64_t>(std::min<int64_t>(want, loop_trips(L0, sh)), 4096);
+                S1 = 1;
+                if (L1 && S0 < want) S1 = std::min<int64_t>(std::min<int64_t>((want + S0 - 1) / S0, loop_trips(*L1, sh)), std::max<int64_t>(1, 4096 / S0));
+                while (S0 * S1 > 1 && (S0 * S1 + 1) * cells > (int64_t(1) << 25)) { if (S1 > 1) S1 /= 2; else S0 /= 2; }   // <= 128 MB of partial sums
+                return S0 * S1;
+            };
+            // when the loops are too short to give the widest shape enough shares, narrower shapes bring more warps
+            int64_t S0 = 1, S1 = 1;
             for (const Shape &sh : shapes) {
                 pick = sh;
-                if (items_for(sh) * (double)splits_for(sh) >= target_warps / 2) break;
+                if (items_for(sh) * (double)splits_for(sh, S0, S1) >= target_warps / 2) break;
             }
-            const int64_t S = splits_for(pick);
-            if (S >= 2) { prog.zsplit = (int32_t)S; prog.part_limit = to_i32(cells); L0.is_split = 1; }
+            const int64_t S = splits_for(pick, S0, S1);
+            if (S >= 2) {
+                prog.zsplit = (int32_t)S; prog.part_limit = to_i32(cells);
+                if (S0 > 1) { L0.is_split = 1; L0.split_n = (int32_t)S0; L0.split_div = (int32_t)S1; }
+                if (S1 > 1) { L1->is_split = 1; L1->split_n = (int32_t)S1; L1->split_div = 1; }
+            }
         }
     } else {
         // element-wise kernel: the widest shape that still leaves enough warps
@@ -1233,10 +1262,33 @@ void generate_backward(tad_plan &p, int q)
     do {
         g.zorder = perm; g.zpos.assign(kap, 0);
         for (int l = 0; l < kap; ++l) g.zpos[perm[l]] = l;
+        ap.zorder = perm;
+        if (kap >= 2) compute_bounds(ap);
         for (int v = 0; v < g.n_outer + kap; ++v) {
             if (forced_lane >= 0 && v != forced_lane) continue;
             if (g.vars[v].ext < 2 && g.n_outer + kap > 1) continue;
             double c = schedule_cost(g, root, v);
+            if (kap >= 2) {
+                // A loop whose bounds differ from lane to lane pays for a range per element every time it is
+                // entered: such a loop belongs outside the loops whose ranges the whole warp shares.
+                double entries = 1;
+                for (int u = 0; u < g.n_outer; ++u) entries *= u == v ? std::ceil((double)g.vars[u].ext / 32.0) : (double)g.vars[u].ext;
+                for (int l = 0; l < kap; ++l) {
+                    bool dep = false;
+                    auto reads_lane = [&](const BoundRowH &h) {
+                        if (v >= g.n_outer) { for (int m = 0; m < l; ++m) if (perm[m] == v - g.n_outer && h.cz[m]) return true; return false; }
+                        if (!by_beta) return h.cx[v] != 0;
+                        int64_t sum = 0;
+                        for (int j = 0; j < R; ++j) sum += h.cx[j] * ap.U(j, v);
+                        return sum != 0;
+                    };
+                    for (const BoundRowH &h : ap.lower[l]) dep = dep || reads_lane(h);
+                    for (const BoundRowH &h : ap.upper[l]) dep = dep || reads_lane(h);
+                    if (dep) c += entries * 600.0;
+                    const int lv = g.n_outer + perm[l];
+                    entries *= lv == v ? std::ceil((double)g.vars[lv].ext / 32.0) : (double)g.vars[lv].ext;
+                }
+            }
             c /= std::min(1.0, (double)g.vars[v].ext / 32.0);
             if (std::abs(dfL.coef[v]) == 1) c *= 0.999;
             if (g.vars[v].kind == 1) c *= 0.9999;

@@ -94,7 +94,8 @@ struct TadpLoop {
     int16_t lower0, n_lower;           // rows[lower0 .. lower0 + n_lower)
     int16_t upper0, n_upper;
     int32_t mask_level;                // position of its activity mask in the mask stack (1..)
-    int32_t is_split;                  // 1: its range is divided among the zsplit warps that share an output
+    int32_t is_split;                  // 1: its range is divided into split_n contiguous shares; the warp with share
+    int32_t split_n, split_div;        //    number s of an output takes share (s / split_div) % split_n
     int32_t is_relative;               // 1: every element walks its own short range, trip r visits lo_e + r
 };
 

@@ -346,8 +346,8 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                 wlo = lo; whi = hi; \
                 if (L.is_split && lo <= hi) { \
                     /* this warp's contiguous share of the range (fixed chunking: repeatable sums) */ \
-                    const int chunk = (hi - lo + P.zsplit) / P.zsplit; \
-                    wlo = lo + split * chunk; whi = min(hi, wlo + chunk - 1); \
+                    const int chunk = (hi - lo + L.split_n) / L.split_n; \
+                    wlo = lo + ((split / L.split_div) % L.split_n) * chunk; whi = min(hi, wlo + chunk - 1); \
                 } \
                 if (__ballot_sync(0xffffffffu, parent != 0) == 0) { wlo = 1; whi = 0; } \
             } else { \
@@ -374,8 +374,8 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                        every element, so that the elements of a share walk it together (fixed chunking: repeatable sums) */ \
                     _Pragma("unroll") for (int o = 16; o > 0; o >>= 1) { lo_w = min(lo_w, __shfl_xor_sync(0xffffffffu, lo_w, o)); hi_w = max(hi_w, __shfl_xor_sync(0xffffffffu, hi_w, o)); } \
                     if (lo_w <= hi_w) { \
-                        const int chunk = (hi_w - lo_w + P.zsplit) / P.zsplit; \
-                        const int slo = lo_w + split * chunk, shi = min(hi_w, slo + chunk - 1); \
+                        const int chunk = (hi_w - lo_w + L.split_n) / L.split_n; \
+                        const int slo = lo_w + ((split / L.split_div) % L.split_n) * chunk, shi = min(hi_w, slo + chunk - 1); \
                         lo_w = INT_MAX; hi_w = INT_MIN; \
                         _Pragma("unroll") for (int t = 0; t < T; ++t) { \
                             elo[lvl - 1][t] = max(elo[lvl - 1][t], slo); ehi[lvl - 1][t] = min(ehi[lvl - 1][t], shi); \
@@ -458,7 +458,12 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
         // fetches one load of the body in the manner the host chose and hands every element's value to COMBINE;
         // ALL: every element of the thread is live (no predicates, signed 64-bit addressing from element 0)
 #define TADV_XFETCH(COMBINE, ALL) \
-                            switch (fk) { \
+                            if (REL && rs != 0) { \
+                                /* inside a relative loop: every element reads at its own position of that loop */ \
+                                _Pragma("unroll") for (int t = 0; t < T; ++t) { \
+                                    const unsigned idx = off + (unsigned)(t / UB) * lc + (unsigned)(t % UB) * uc + rs * (unsigned)zrel(t); \
+                                    const float x = (ALL || ((cur >> t) & 1u)) ? __ldg(base + idx) : 0.f; COMBINE(t, x) } \
+                            } else switch (fk) { \
                             case BF_ONE: { \
                                 const float x = (ALL || cur) ? __ldg(base + off) : 0.f; \
                                 _Pragma("unroll") for (int t = 0; t < T; ++t) { COMBINE(t, x) } \
@@ -521,6 +526,7 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                         const unsigned off = TADV_XSEL(j, xo); \
                         const unsigned lc = TADV_XSEL(j, xlc); \
                         const unsigned uc = TADV_XSEL(j, xuc); \
+                        const unsigned rs = REL ? TADV_XSEL(j, xrs) : 0u; (void)rs; \
                         const float *base = TADV_XSEL(j, xbase); \
                         switch (cmb) { \
                         case 0: TADV_XFETCH(TADV_XC_SET, ALL) break; \
@@ -550,7 +556,7 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                     live |= cur; \
                 } }
 #define TADV_XSEL(j, A) ((j) == 0 ? A[0] : (j) == 1 ? A[1] : (j) == 2 ? A[2] : A[3])
-#define TADV_XLOOP(SUMMODE) case TADV_H(P_XLOOP, SUMMODE): if constexpr (!DEBUG && !REL && (SUMMODE) + 2 <= VmCfg<TA, UB>::DEPTH) { \
+#define TADV_XLOOP(SUMMODE) case TADV_H(P_XLOOP, SUMMODE): if constexpr (!DEBUG && (SUMMODE) + 2 <= VmCfg<TA, UB>::DEPTH) { \
             constexpr int DEPTH = VmCfg<TA, UB>::DEPTH; \
             constexpr int XI = (SUMMODE), YI = XI + 1, I0 = DEPTH - 1, I1 = DEPTH >= 2 ? DEPTH - 2 : 0; \
             const TadpBody &B = P.bodies[imm]; \
@@ -571,12 +577,13 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
             const int lvl = L.mask_level; \
             const unsigned parent = kind == BL_SUM ? cur : kind == BL_USUM ? sum_parent : mstack[lvl - 1]; \
             /* per load slot: offset of this thread's element 0, its step per trip, pointer and element strides */ \
-            unsigned xo[TADP_BODY_LOADS], xst[TADP_BODY_LOADS], xlc[TADP_BODY_LOADS], xuc[TADP_BODY_LOADS]; \
+            unsigned xo[TADP_BODY_LOADS], xst[TADP_BODY_LOADS], xlc[TADP_BODY_LOADS], xuc[TADP_BODY_LOADS], xrs[REL ? TADP_BODY_LOADS : 1]; \
             const float *xbase[TADP_BODY_LOADS]; \
             _Pragma("unroll") for (int j = 0; j < TADP_BODY_LOADS; ++j) { \
                 const TadpLoad &Ld = P.loads[B.load[j < B.n_loads ? j : 0]]; \
                 xo[j] = load_offset(Ld, m.var); xst[j] = (unsigned)Ld.coef[V] * (unsigned)dz; \
                 xlc[j] = (unsigned)Ld.lane_step; xuc[j] = UB > 1 ? (unsigned)Ld.unroll_step : 0u; \
+                if (REL) xrs[j] = (unsigned)Ld.rel_step; \
                 xbase[j] = ptrs.in[Ld.ptr]; \
             } \
             const uint2 steps = *reinterpret_cast<const uint2 *>(B.steps); \
