@@ -23,26 +23,43 @@ namespace {
 
 constexpr int WARPS_PER_BLOCK = TADP_WARPS_PER_BLOCK;
 
-// Adds the zsplit planes of partial sums up in plane order and writes the gradient elements:
-// compact index c -> outer variables -> output offset.  Masked gradients write only outputs
-// whose flag says that some term was accumulated.
-__global__ void tad_reduce_partials(const __grid_constant__ TadpProgram P, float *out, const float *part)
+// Adds the zsplit planes of partial sums up and writes the gradient elements: compact index
+// c -> outer variables -> output offset.  A block takes 32 consecutive cells (one per lane,
+// so that every plane is read in full sectors); its warp w adds planes w, w + 32, ... in that
+// order and the warps' subtotals are added in warp order: the same association every run.
+// Masked gradients write only outputs whose flag says that some term was accumulated.
+constexpr int REDUCE_WARPS = 32;
+__global__ void __launch_bounds__(REDUCE_WARPS * 32)
+tad_reduce_partials(const __grid_constant__ TadpProgram P, float *out, const float *part)
 {
+    __shared__ float sub[REDUCE_WARPS][32];
     const unsigned n = (unsigned)P.part_limit;
-    const unsigned stride = gridDim.x * blockDim.x;
     const int planes = P.zsplit;
-    for (unsigned c = blockIdx.x * blockDim.x + threadIdx.x; c < n; c += stride) {
-        if (P.write_only_live && part[(size_t)planes * n + c] == 0.f) continue;
-        unsigned rem = c, off = (unsigned)P.out_base;
-        for (int v = P.n_outer - 1; v >= 0; --v) {
-            const unsigned ext = (unsigned)P.outer_ext[v];
-            const unsigned digit = rem % ext; rem /= ext;
-            off += (unsigned)P.out_coef[v] * (unsigned)(P.outer_lo[v] + (int)digit);
+    const unsigned lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    for (unsigned c0 = blockIdx.x * 32u; c0 < n; c0 += gridDim.x * 32u) {
+        const unsigned c = c0 + lane;
+        float sum = 0.f;
+        if (c < n) {
+#pragma unroll 4
+            for (int s = (int)warp; s < planes; s += REDUCE_WARPS) sum += part[(size_t)s * n + c];
         }
-        if (off >= (unsigned)P.out_limit) continue;
-        float sum = P.accumulate ? out[off] : 0.f;
-        for (int s = 0; s < planes; ++s) sum += part[(size_t)s * n + c];
-        out[off] = sum;
+        sub[warp][lane] = sum;
+        __syncthreads();
+        if (warp == 0 && c < n && !(P.write_only_live && part[(size_t)planes * n + c] == 0.f)) {
+            unsigned rem = c, off = (unsigned)P.out_base;
+            for (int v = P.n_outer - 1; v >= 0; --v) {
+                const unsigned ext = (unsigned)P.outer_ext[v];
+                const unsigned digit = rem % ext; rem /= ext;
+                off += (unsigned)P.out_coef[v] * (unsigned)(P.outer_lo[v] + (int)digit);
+            }
+            if (off < (unsigned)P.out_limit) {
+                float total = P.accumulate ? out[off] : 0.f;
+                const int used = planes < REDUCE_WARPS ? planes : REDUCE_WARPS;
+                for (int w = 0; w < used; ++w) total += sub[w][lane];
+                out[off] = total;
+            }
+        }
+        __syncthreads();
     }
 }
 
@@ -101,8 +118,8 @@ tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStrea
     if (e != cudaSuccess) { tad::set_error(std::string("kernel launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
     if (zsplit > 1) {
         const unsigned n = (unsigned)k.prog.part_limit;
-        const unsigned rblocks = std::min((n + 255u) / 256u, (unsigned)sm_count() * 16u);
-        tad_reduce_partials<<<rblocks, 256, 0, stream>>>(k.prog, ptrs.out, ptrs.part);
+        const unsigned rblocks = std::min((n + 31u) / 32u, (unsigned)sm_count() * 8u);
+        tad_reduce_partials<<<rblocks, REDUCE_WARPS * 32, 0, stream>>>(k.prog, ptrs.out, ptrs.part);
         e = cudaGetLastError();
         if (e != cudaSuccess) { tad::set_error(std::string("reduce launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
     }

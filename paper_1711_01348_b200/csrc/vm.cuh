@@ -56,6 +56,37 @@ static __device__ __noinline__ float apply_fn(int fn, float x, int n)
     }
 }
 
+// Inline versions of the functions that dominate element-wise kernels; everything else goes
+// through apply_fn.  Sine and cosine: Cody-Waite reduction by multiples of pi/2 (three-part
+// constant, exact first step) and the degree-7 / degree-8 polynomials of the remainder on
+// [-pi/4, pi/4]; arguments of 8192 and beyond, infinities and NaN take the library routine.
+__device__ __forceinline__ float fast_sincos(float x, int quarter)
+{
+    if (!(fabsf(x) < 8192.f)) return quarter ? cosf(x) : sinf(x);
+    const float k = rintf(x * 0.636619772367581f);
+    float r = fmaf(k, -1.5703125f, x);
+    r = fmaf(k, -4.837512969970703125e-4f, r);
+    r = fmaf(k, -7.54978995489188216e-8f, r);
+    const int q = (int)k + quarter;
+    const float r2 = r * r;
+    const float sn = fmaf(r * r2, fmaf(r2, fmaf(r2, -1.9515295891e-4f, 8.3321608736e-3f), -1.6666654611e-1f), r);
+    const float cs = fmaf(r2 * r2, fmaf(r2, fmaf(r2, 2.443315711809948e-5f, -1.388731625493765e-3f), 4.166664568298827e-2f),
+                          fmaf(r2, -0.5f, 1.f));
+    const float v = (q & 1) ? cs : sn;
+    return (q & 2) ? -v : v;
+}
+// tanh: odd series below 1/4 (truncation 3e-7 relative), 1 - 2 / (exp(2|x|) + 1) above
+__device__ __forceinline__ float fast_tanh(float x)
+{
+    const float ax = fabsf(x);
+    if (ax < 0.25f) {
+        const float x2 = x * x;
+        return x * fmaf(x2, fmaf(x2, fmaf(x2, -17.f / 315.f, 2.f / 15.f), -1.f / 3.f), 1.f);
+    }
+    const float e = __expf(2.f * ax);
+    return copysignf(1.f - __fdividef(2.f, e + 1.f), x);
+}
+
 // Per vector width: NTR temporaries kept in registers (the rest spill to local memory) and the
 // usable operand stack depth.  Wide vectors amortise the dispatch cost over more elements and
 // pay for it with a shallower stack; the host picks the widest variant a program fits.
@@ -245,7 +276,13 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                 } \
                 break; \
             } \
-            TADV_UNARY(D, apply_fn(fn_code, x, imm)) }
+            switch (fn_code) { \
+            case F_EXP: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 1][t] = __expf(m.s[D - 1][t]); } break; \
+            case F_SIN: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 1][t] = fast_sincos(m.s[D - 1][t], 0); } break; \
+            case F_COS: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 1][t] = fast_sincos(m.s[D - 1][t], 1); } break; \
+            case F_TANH: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 1][t] = fast_tanh(m.s[D - 1][t]); } break; \
+            default: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 1][t] = apply_fn(fn_code, m.s[D - 1][t], imm); } break; \
+            } } break;
         TADV_D1(TADV_FN, P_FN)
 
 #define TADV_BINARY(D, EXPR) { _Pragma("unroll") for (int t = 0; t < T; ++t) { const float x = m.s[D - 2][t], y = m.s[D - 1][t]; m.s[D - 2][t] = (EXPR); } } break;
