@@ -433,18 +433,25 @@ struct Emitter {
             temps_of_sum(i);
             const Inst inner = g.inst[in.a];
             if (!over_elements && inner.op == I_SUM && inline_ok(in.a) && inner.var != g.unroll_var) {
-                // a sum whose summand is a sum: the inner loop adds its summands to the same accumulator
+                // a sum whose summand is a sum: the inner loop adds its summands to the same accumulator;
+                // the longer of the two ranges runs innermost (the order of a sum of sums is free)
                 TadpLoop L2{};
                 L2.var = inner.var; L2.const_lo = (int32_t)inner.lo; L2.const_hi = (int32_t)inner.hi;
                 if ((int)loops.size() >= TADP_MAX_LOOPS) throw Unsupported("too many loops in one kernel");
+                int outer_var = in.var;
+                if (inner.hi - inner.lo < in.hi - in.lo && swap_ok(i, in.a)) {
+                    std::swap(loops[id], L2);
+                    outer_var = inner.var;
+                    code[begin].handler = (uint16_t)(P_SLOOP * 8 + outer_var);
+                }
                 loops.push_back(L2);
                 const int id2 = (int)loops.size() - 1;
-                const int ib = emit(P_SLOOP, id2, 0, 0, 0, inner.var);
+                const int ib = emit(P_SLOOP, id2, 0, 0, 0, loops[id2].var);
                 temps_of_sum(in.a);
                 expr(inner.a);
                 const int ie = emit(P_SUMEND, id2, 0, ib + 1, -1);
                 code[ib].imm = ie + 1;
-                const int oe = emit(P_SEND, id, 0, begin + 1, 0, in.var);
+                const int oe = emit(P_SEND, id, 0, begin + 1, 0, outer_var);
                 code[begin].imm = oe + 1;
                 break;
             }
@@ -459,6 +466,14 @@ struct Emitter {
             break;
         }
         }
+    }
+    // nested sums that share an accumulator may trade places when no temporary belongs to either of
+    // them (a temporary is evaluated at the head of its own loop)
+    bool swap_ok(int outer_sum, int inner_sum) const
+    {
+        for (const Inst &in : g.inst)
+            if (in.temp >= 0 && in.uses > 0 && (in.home_sum == inner_sum || in.home_sum == outer_sum)) return false;
+        return true;
     }
     void temps_of_sum(int sum_inst)
     {
@@ -639,7 +654,7 @@ void finish_stats(Gen &g, Kernel &k, bool backward, int64_t outputs, int64_t ter
 // uses the sector in full; a strided load that does not depend on B is fetched once for all its
 // elements.  Candidates: outer variables (a tile of gradient elements per thread) and bound
 // sums (several summands per trip).
-void choose_element_variable(Gen &g)
+void choose_element_variable(Gen &g, bool allow_outer_product)
 {
     g.unroll_var = -1;
     if (g.p.opt.debug_bounds) return;            // debug plans use the narrow kernels
@@ -650,6 +665,7 @@ void choose_element_variable(Gen &g)
         if (g.vars[v].kind == 2 && (g.vars[v].sum_inst < 0 || !g.inst[g.vars[v].sum_inst].uses)) continue;
         double score = 0;
         bool fixes_strided = false;
+        bool lane_free_load = false, u_free_load = false;   // a load that varies with v only, one that varies with A only
         for (const Inst &in : g.inst) {
             if (!in.uses || in.op != I_LOAD) continue;
             const TadpLoad &L = g.loads[in.load];
@@ -658,12 +674,16 @@ void choose_element_variable(Gen &g)
             double w = 1;
             for (int x = g.n_outer; x < (int)g.vars.size(); ++x)
                 if (x != v && (in.deps & (1u << x))) w *= (double)g.vars[x].ext;
+            if (cb != 0 && ca == 0) lane_free_load = true;
+            if (cb == 0 && ca != 0) u_free_load = true;
             if (cb == 1 && ca >= 8) { score += 4 * w; fixes_strided = true; }          // strided load becomes row reads
             else if (cb == 0 && ca >= 8) { score += 3 * w; fixes_strided = true; }     // strided load shared by all u
             else if (cb == 0) score += w;
             else if (cb == 1 && ca == 0) score += 0.5 * w;
         }
-        if (fixes_strided && score > best) { best = score; g.unroll_var = v; }
+        // outer-product structure: one load per value of v and one per value of A serve UB x TA elements
+        const bool outer_product = allow_outer_product && lane_free_load && u_free_load && g.vars[v].ext >= 8;
+        if ((fixes_strided || outer_product) && score > best) { best = score; g.unroll_var = v; }
     }
 }
 
@@ -860,7 +880,16 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
             place(g);
         }
     }
-    choose_element_variable(g);
+    // a short loop whose range shifts from lane to lane will be walked relative to every element's own
+    // start, which needs the elements of a thread to lie along the lane variable only
+    bool relative_candidate = false;
+    for (int l = 0; l < g.kappa; ++l) {
+        const int v = g.n_outer + g.zorder[l];
+        if (v == g.lane_var || g.vars[v].ext > 16) continue;
+        for (const TadpRow &r : lower[l]) if (r.coef[g.lane_var]) relative_candidate = true;
+        for (const TadpRow &r : upper[l]) if (r.coef[g.lane_var]) relative_candidate = true;
+    }
+    choose_element_variable(g, !relative_candidate);
     // temporaries: shared values and values hoisted out of the loop that consumes them
     std::vector<bool> hoisted(g.inst.size(), false);
     auto effective_level = [&](int i) { return i == root ? g.kappa : g.inst[i].zlevel; };

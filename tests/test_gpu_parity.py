@@ -69,6 +69,14 @@ def test_reduced_workloads(key):
     check_against_oracle(e, args, df, nthreads=max_threads())
 
 
+@pytest.mark.parametrize("fn", ["exp", "log", "sin", "cos", "tanh", "sinh", "cosh"])
+def test_function_argument_sweeps(fn):
+    """The inline evaluations (own range reduction, polynomials, fast exponential) and the library
+    fall-backs, over large, tiny and awkward arguments, value and derivative."""
+    e, args, df = W.function_sweep(fn)
+    check_against_oracle(e, args, df)
+
+
 def test_gradient_subset_and_repeat_calls():
     e, args, df = W.workload("cfg2", full=False)
     run = GpuRun(e, args, df)

@@ -171,6 +171,40 @@ def ex_sin(n: int) -> Expr:
     return b.done()
 
 
+def ex_unary(fn: str, n: int) -> Expr:
+    """f_i = fn(x_i) for one elementary function (argument sweeps of the function tests)."""
+    b = Builder("ex_" + fn, [n], 0, ["x"], [[n]])
+    b.un(fn, b.load("x", [unit(1, (0, 1))]))
+    return b.done()
+
+
+def function_sweep(fn: str, n: int = 8192, seed: int = 0):
+    """Arguments that exercise an elementary function over its whole useful range: moderate and
+    large magnitudes, values next to multiples of pi / 2 and around the switch points of
+    piecewise evaluations, tiny values, zeros.  Returns (expr, [x], df)."""
+    import math
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed)
+    q = n // 8
+    parts = [
+        (torch.rand(q, generator=g) * 2 - 1) * 10.0,
+        torch.randn(q, generator=g) * (30.0 if fn in ("exp", "sinh", "cosh") else 3000.0),
+        torch.round(torch.randn(q, generator=g) * 40) * (math.pi / 2) + (torch.rand(q, generator=g) - 0.5) * 1e-3,
+        (torch.rand(q, generator=g) * 2 - 1) * 0.5,
+        0.25 + (torch.rand(q, generator=g) - 0.5) * 1e-4,
+        (torch.rand(q, generator=g) * 2 - 1) * 1e-5,
+        torch.randn(q, generator=g) * (80.0 if fn in ("exp", "sinh", "cosh") else 3.0e5),
+    ]
+    x = torch.cat(parts)
+    x = torch.cat([x, torch.zeros(n - x.numel())]).to(torch.float32)
+    if fn == "log":
+        x = x.abs() + 1e-3
+    if fn in ("exp", "sinh", "cosh"):
+        x = x.clamp(-85.0, 85.0)
+    df = torch.randn(n, generator=g, dtype=torch.float32)
+    return ex_unary(fn, n), [x.contiguous()], df.contiguous()
+
+
 def ex_xy(n: int) -> Expr:
     """f^2_ij = x_i y_ij  (Sec. 5)."""
     b = Builder("ex_xy", [n, n], 0, ["x", "y"], [[n], [n, n]])
