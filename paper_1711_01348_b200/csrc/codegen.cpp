@@ -1049,7 +1049,11 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
                 return std::max<int64_t>(1, g.vars[L.var].ext / (L.is_lane ? 32 * sh.ta : 1));
             };
             auto splits_for = [&](const Shape &sh, int64_t &S0, int64_t &S1) {
-                const int64_t want = (int64_t)std::ceil(target_warps / items_for(sh));
+                // whole waves of resident warps (148 SMs x 16): a last wave that is mostly empty costs a full one
+                const double resident = 148.0 * 16.0;
+                int64_t want = (int64_t)std::ceil(2.0 * target_warps / items_for(sh));
+                const double waves = std::max(1.0, std::round(items_for(sh) * (double)want / resident));
+                want = std::max<int64_t>(1, (int64_t)std::floor(waves * resident / items_for(sh)));
                 S0 = std::min<int64_t>(std::min<int64_t>(want, loop_trips(L0, sh)), 4096);
                 S1 = 1;
                 if (L1 && S0 < want) S1 = std::min<int64_t>(std::min<int64_t>((want + S0 - 1) / S0, loop_trips(*L1, sh)), std::max<int64_t>(1, 4096 / S0));
