@@ -666,6 +666,7 @@ void choose_element_variable(Gen &g, bool allow_outer_product)
         double score = 0;
         bool fixes_strided = false;
         bool lane_free_load = false, u_free_load = false;   // a load that varies with v only, one that varies with A only
+        bool shared_stream = false, own_stream = false;     // loads inside the summation loops: the same for every u, one per u
         for (const Inst &in : g.inst) {
             if (!in.uses || in.op != I_LOAD) continue;
             const TadpLoad &L = g.loads[in.load];
@@ -676,6 +677,8 @@ void choose_element_variable(Gen &g, bool allow_outer_product)
                 if (x != v && (in.deps & (1u << x))) w *= (double)g.vars[x].ext;
             if (cb != 0 && ca == 0) lane_free_load = true;
             if (cb == 0 && ca != 0) u_free_load = true;
+            if (w > 1 && cb == 0) shared_stream = true;
+            if (w > 1 && cb != 0) own_stream = true;
             if (cb == 1 && ca >= 8) { score += 4 * w; fixes_strided = true; }          // strided load becomes row reads
             else if (cb == 0 && ca >= 8) { score += 3 * w; fixes_strided = true; }     // strided load shared by all u
             else if (cb == 0) score += w;
@@ -683,7 +686,11 @@ void choose_element_variable(Gen &g, bool allow_outer_product)
         }
         // outer-product structure: one load per value of v and one per value of A serve UB x TA elements
         const bool outer_product = allow_outer_product && lane_free_load && u_free_load && g.vars[v].ext >= 8;
-        if ((fixes_strided || outer_product) && score > best) { best = score; g.unroll_var = v; }
+        // a summation that streams one tensor for every output and another that UB outputs can share: a tile of
+        // outputs per thread reads the shared one once (less traffic from L2 and HBM per term)
+        const bool shared_reads = allow_outer_product && g.kappa >= 1 && g.vars[v].kind == 0 && shared_stream && own_stream &&
+                                  g.vars[v].ext >= 8;
+        if ((fixes_strided || outer_product || shared_reads) && score > best) { best = score; g.unroll_var = v; }
     }
 }
 
