@@ -1296,9 +1296,11 @@ void generate_backward(tad_plan &p, int q)
             (forced_lane < 0 || g.vars[v].ext > g.vars[forced_lane].ext ||
              (g.vars[v].ext == g.vars[forced_lane].ext && g.vars[v].kind == 1)))
             forced_lane = v;
+    double best = -1; std::vector<int> best_order(kap); int best_lane = -1;
+    auto search = [&](int forced_lane) {
     std::vector<int> perm(kap);
     for (int l = 0; l < kap; ++l) perm[l] = l;
-    double best = -1; std::vector<int> best_order = perm; int best_lane = -1;
+    best = -1; best_order = perm; best_lane = -1;
     do {
         g.zorder = perm; g.zpos.assign(kap, 0);
         for (int l = 0; l < kap; ++l) g.zpos[perm[l]] = l;
@@ -1335,6 +1337,15 @@ void generate_backward(tad_plan &p, int q)
             if (best < 0 || c < best) { best = c; best_order = perm; best_lane = v; }
         }
     } while (std::next_permutation(perm.begin(), perm.end()));
+    };
+    search(forced_lane);
+    if (forced_lane >= 0) {
+        // ... unless another variable is estimated to be far cheaper (the strided loads of the forced
+        // choice cost a transaction per lane: cfg2 da reads b[j, k] with one lane per j)
+        const double forced_cost = best; const std::vector<int> forced_order = best_order; const int forced = best_lane;
+        search(-1);
+        if (!(best >= 0 && best * 2.5 < forced_cost)) { best = forced_cost; best_order = forced_order; best_lane = forced; }
+    }
     if (best_lane < 0) best_lane = 0;
     g.zorder = best_order; g.zpos.assign(kap, 0);
     for (int l = 0; l < kap; ++l) g.zpos[best_order[l]] = l;
