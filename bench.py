@@ -24,7 +24,9 @@ METRIC = "fwd+bwd tensor elements/s"
 UNIT = "elements/s"
 
 # rows of the output the oracle sample covers, per workload (about 10-30 s of CPU work on 16 cores)
-ORACLE_SAMPLE_ROWS = {"cfg1": 64, "cfg2": 256, "cfg3": 4096, "cfg4": 96, "cfg5": 1}
+ORACLE_SAMPLE_ROWS = {"cfg1": 64, "cfg2": 2048, "cfg3": 4096, "cfg4": 96, "cfg5": 1}
+# ... and per step of the reference arm, which repeats it steps + warmup times (a second or two each)
+REFERENCE_STEP_ROWS = {"cfg1": 64, "cfg2": 256, "cfg3": 4096, "cfg4": 16, "cfg5": 1}
 
 
 # how every workload keeps the timed iterations from running out of L2 (126 MB)
@@ -133,10 +135,10 @@ def elements_per_step(expr) -> int:
     return n
 
 
-def oracle_sample(key, expr, args, df, nthreads):
+def oracle_sample(key, expr, args, df, nthreads, table=None):
     """Runs the oracle, as it stands, on the first rows of the output; returns (seconds, elements)."""
     from oracle.oracle import Oracle
-    rows = min(ORACLE_SAMPLE_ROWS[key], expr.out_shape[0])
+    rows = min((table or ORACLE_SAMPLE_ROWS)[key], expr.out_shape[0])
     lo = [0] * len(expr.out_shape)
     hi = [rows] + list(expr.out_shape[1:])
     orc = Oracle(expr)
@@ -161,7 +163,7 @@ def run_reference(opts):
     sample = ""
     elems = 0.0
     for i in range(opts.warmup + opts.steps):
-        dt, elems, sample = oracle_sample(opts.config, expr, args, df, cores)
+        dt, elems, sample = oracle_sample(opts.config, expr, args, df, cores, REFERENCE_STEP_ROWS)
         if i >= opts.warmup:
             times.append(dt)
     total = sum(times)
@@ -342,7 +344,7 @@ def run_ours(opts):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
