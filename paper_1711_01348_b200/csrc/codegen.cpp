@@ -1314,6 +1314,7 @@ void generate_backward(tad_plan &p, int q)
                 // A loop whose bounds differ from lane to lane pays for a range per element every time it is
                 // entered: such a loop belongs outside the loops whose ranges the whole warp shares.
                 double entries = 1;
+                bool any_dep = false;
                 for (int u = 0; u < g.n_outer; ++u) entries *= u == v ? std::ceil((double)g.vars[u].ext / 32.0) : (double)g.vars[u].ext;
                 for (int l = 0; l < kap; ++l) {
                     bool dep = false;
@@ -1326,10 +1327,16 @@ void generate_backward(tad_plan &p, int q)
                     };
                     for (const BoundRowH &h : ap.lower[l]) dep = dep || reads_lane(h);
                     for (const BoundRowH &h : ap.upper[l]) dep = dep || reads_lane(h);
-                    if (dep) c += entries * 600.0;
+                    // every entry of a loop costs its set-up, so the loop with the most trips belongs innermost
+                    // (a loop over the lane variable makes one trip per 512 values at the widest shape)
+                    c += entries * 50.0;
+                    if (dep) { c += entries * 600.0; any_dep = true; }
                     const int lv = g.n_outer + perm[l];
-                    entries *= lv == v ? std::ceil((double)g.vars[lv].ext / 32.0) : (double)g.vars[lv].ext;
+                    entries *= lv == v ? std::ceil((double)g.vars[lv].ext / 512.0) : (double)g.vars[lv].ext;
                 }
+                // ... and everything inside it runs under per-element masks and start offsets, with the lanes
+                // whose range is shorter idle: measured about three times the cost per term (cfg5 dx)
+                if (any_dep) c *= 3.0;
             }
             c /= std::min(1.0, (double)g.vars[v].ext / 32.0);
             if (std::abs(dfL.coef[v]) == 1) c *= 0.999;
