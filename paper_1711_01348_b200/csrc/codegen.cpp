@@ -810,6 +810,11 @@ int fuse_inner_loops(Emitter &em, std::vector<TadpBody> &bodies, int depth_limit
         B.n_loads = (int32_t)d.loads.size();
         B.loop_kind = kind; B.term = d.term;
         for (size_t q = 0; q < d.inv.size(); ++q) { B.inv_kind[q] = d.inv[q].first; B.inv_value[q] = d.inv[q].second; }
+        // the term is the product of two loads and nothing else
+        if (d.inv.empty() && d.loads.size() == 2 &&
+            ((d.term == 0 && d.steps == std::vector<uint8_t>{0x80 | 0, 0x80 | (2 << 2) | 1}) ||
+             (d.term == 1 && d.steps == std::vector<uint8_t>{0x80 | 0, BS_PUSH, 0x80 | 1})))
+            B.dot = 1;
         bodies.push_back(B);
         // body and loop end become one word; jump targets behind it move up
         const int removed = e - (b + 1);
@@ -1012,10 +1017,36 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     std::vector<TadpBody> bodies_wide;
     const int deepest_wide = can_fuse ? fuse_inner_loops(trial, bodies_wide, TADP_WIDE_DEPTH) : em.max_depth;
     const bool shallow = deepest_wide <= TADP_WIDE_DEPTH;
+    // Product kernels: when every fused loop is a product of two loads, one of which has a value per u or
+    // per t only, and the rest of the program needs a single operand slot, the thread can hold 4 x 8
+    // sums (nothing but the sums has 32 entries: an outer-product or streamed multiply-add per trip).
+    auto load_class = [&](const TadpLoad &L, int ta, int ub) {
+        const int fk = body_fetch_kind(L, ta, ub);
+        return fk == BF_ONE || fk == BF_PER_U ? 0 : fk == BF_PER_T ? 1 : 2;
+    };
+    bool product_only = can_fuse && g.unroll_var >= 0 && !bodies_wide.empty() && prog.rel_var < 0;
+    if (product_only) {
+        int deepest32 = 0;
+        for (size_t i = 0; i < trial.code.size(); ++i) {
+            const int op = trial.code[i].handler >> 3;
+            if (op == P_XLOOP) {
+                const TadpBody &B = bodies_wide[trial.code[i].imm];
+                if (!B.dot || std::min(load_class(prog.loads[B.load[0]], 4, 8), load_class(prog.loads[B.load[1]], 4, 8)) > 1) product_only = false;
+                deepest32 = std::max(deepest32, trial.depth_at[i]);
+                continue;
+            }
+            if (op >= P_SLOOP && op <= P_ZEND) continue;
+            int after = trial.depth_at[i];
+            if (op == P_CONST || op == P_ZERO || op == P_LOAD || op == P_LDT) after += 1;
+            deepest32 = std::max(deepest32, after);
+        }
+        if (deepest32 > 1) product_only = false;
+    }
     // candidate shapes (TA, UB), widest first; 16 values per thread need the shallow stack
     struct Shape { int ta, ub; };
     std::vector<Shape> shapes;
     if (g.unroll_var >= 0 && !debug) {
+        if (product_only && uext >= 8 && lane_ext >= 128) shapes.push_back({4, 8});
         if (uext >= 8 && shallow && lane_ext >= 64) shapes.push_back({2, 8});     // measured best on the intro expression
         if (uext >= 16 && shallow) shapes.push_back({1, 16});
         if (uext >= 8) shapes.push_back({1, 8});
@@ -1093,6 +1124,13 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     for (TadpBody &B : bodies)
         for (int i = 0; i < TADP_BODY_STEPS; ++i)
             if (B.steps[i] & 0x80) B.steps[i] |= (uint8_t)(body_fetch_kind(prog.loads[B.load[B.steps[i] & 3]], pick.ta, pick.ub) << 4);
+    if (pick.ta * pick.ub >= 32)
+        for (TadpBody &B : bodies) {
+            // P is the operand of the smaller class: its buffer is small and the other one is never stored
+            if (load_class(prog.loads[B.load[1]], pick.ta, pick.ub) < load_class(prog.loads[B.load[0]], pick.ta, pick.ub)) std::swap(B.load[0], B.load[1]);
+            B.dot_pclass = load_class(prog.loads[B.load[0]], pick.ta, pick.ub);
+            for (int j = 0; j < 2; ++j) B.dot_fk[j] = body_fetch_kind(prog.loads[B.load[j]], pick.ta, pick.ub);
+        }
     prog.n_bodies = (int32_t)bodies.size();
     std::copy(bodies.begin(), bodies.end(), prog.bodies);
     prog.n_code = (int32_t)em.code.size();

@@ -126,6 +126,12 @@ struct alignas(8) TadpBody {
     int32_t term;                      // 0: S += X, 1: S += Y * X
     int32_t inv_kind[2];               // 0 unused, 1 constant (inv_value), 2 temporary (inv_value = its number)
     int32_t inv_value[2];
+    // Product body: the term is the product of two loads and nothing else, S += P * Q with P = slot 0 and
+    // Q = slot 1.  The 32-value shapes run only such bodies: P is fetched into a buffer of its shape
+    // class (0: one value per u, 1: one per t), Q is multiplied in and accumulated as it arrives.
+    int32_t dot;
+    int32_t dot_pclass;
+    int32_t dot_fk[2];                 // TadpBodyFetch of P and Q
 };
 
 struct alignas(16) TadpProgram {

@@ -16,12 +16,11 @@ void set_error(const std::string &m);
 }
 
 // One build of the interpreter per vector shape, each in an object file of its own (vm_inst.cu).
-#define TAD_DECLARE_VM(TA, UB) void tad_launch_vm_##TA##_##UB(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned blocks, cudaStream_t stream);
+#define TAD_DECLARE_VM(TA, UB) void tad_launch_vm_##TA##_##UB(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream);
 TAD_VM_SHAPES(TAD_DECLARE_VM)
 
 namespace {
 
-constexpr int WARPS_PER_BLOCK = TADP_WARPS_PER_BLOCK;
 
 // Adds the zsplit planes of partial sums up and writes the gradient elements: compact index
 // c -> outer variables -> output offset.  A block takes 32 consecutive cells (one per lane,
@@ -106,11 +105,8 @@ tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStrea
     if (items64 == 0) return TAD_OK;
     if (items64 >= (1ull << 32)) { tad::set_error("too many work items"); return TAD_ERR_UNSUPPORTED; }
     const unsigned items = (unsigned)items64;
-    const unsigned blocks_needed = (items + WARPS_PER_BLOCK - 1) / WARPS_PER_BLOCK;
-    const unsigned max_blocks = (unsigned)sm_count() * 16u;
-    const unsigned blocks = std::min(blocks_needed, max_blocks);
     switch (k.vec * 100 + k.vec_u) {
-#define TAD_CASE_VM(TA, UB) case TA * 100 + UB: tad_launch_vm_##TA##_##UB(k.prog, ptrs, debug, items, blocks, stream); break;
+#define TAD_CASE_VM(TA, UB) case TA * 100 + UB: tad_launch_vm_##TA##_##UB(k.prog, ptrs, debug, items, (unsigned)sm_count(), stream); break;
     TAD_VM_SHAPES(TAD_CASE_VM)
     default: tad::set_error("internal: no kernel for this vector shape"); return TAD_ERR_UNSUPPORTED;
     }

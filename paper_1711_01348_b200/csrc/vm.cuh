@@ -20,7 +20,6 @@
 
 namespace tadvm {
 
-constexpr int WARPS_PER_BLOCK = TADP_WARPS_PER_BLOCK;
 constexpr int STACK = TADP_MAX_DEPTH - 1;   // usable depth (handlers are encoded for depth 0..7)
 
 __device__ __forceinline__ int floor_div_i(int a, int b) { int q = a / b; return (a % b != 0 && a < 0) ? q - 1 : q; }
@@ -94,7 +93,9 @@ template <int TA, int UB>
 struct VmCfg {
     static constexpr int E = TA * UB;           // values per thread and operand
     static constexpr int NTR = E >= 16 ? 0 : E >= 8 ? 2 : TADP_NUM_TEMPS;
-    static constexpr int DEPTH = E >= 16 ? TADP_WIDE_DEPTH : STACK;
+    // 32 values per thread: the shapes of the product kernels; one operand slot, blocks of 4 warps
+    static constexpr int DEPTH = E >= 32 ? 1 : E >= 16 ? TADP_WIDE_DEPTH : STACK;
+    static constexpr int WARPS = E >= 32 ? 4 : TADP_WARPS_PER_BLOCK;
 };
 
 template <int TA, int UB>
@@ -163,7 +164,7 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
     int elo[TADP_MAX_ZLOOPS][T], ehi[TADP_MAX_ZLOOPS][T];
     // per-element start of the relative loop; in shared memory (one column per thread) because it is
     // rarely touched and would otherwise cost T registers in every kernel
-    __shared__ int zrel_s[REL ? T : 1][WARPS_PER_BLOCK * 32];
+    __shared__ int zrel_s[REL ? T : 1][VmCfg<TA, UB>::WARPS * 32];
 #define zrel(t) zrel_s[t][threadIdx.x]
     const int rel_var = REL ? P.rel_var : -1;
     constexpr int NTR = VmCfg<TA, UB>::NTR;
@@ -593,7 +594,71 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                     live |= cur; \
                 } }
 #define TADV_XSEL(j, A) ((j) == 0 ? A[0] : (j) == 1 ? A[1] : (j) == 2 ? A[2] : A[3])
-#define TADV_XLOOP(SUMMODE) case TADV_H(P_XLOOP, SUMMODE): if constexpr (!DEBUG && (SUMMODE) + 2 <= VmCfg<TA, UB>::DEPTH) { \
+        // ---- product loops of the 32-value shapes: S += P * Q, P (one value per u, or one per t) into a small
+        // buffer, Q multiplied in and accumulated value by value as it arrives; nothing but S has 32 entries ----
+#define TADV_DC_PU(t, x) pu[(t) % UB] = (x);
+#define TADV_DC_PT(t, x) pt[(t) / UB] = (x);
+#define TADV_DC_ACC(t, p, x, ALL) if (ALL || (SM && UB == 1) || ((cur >> (t)) & 1u)) SS[t] = op_fma((p), (x), SS[t]);
+#define TADV_DC_QU_T(t, x) TADV_DC_ACC(t, pu[(t) % UB], x, true)
+#define TADV_DC_QT_T(t, x) TADV_DC_ACC(t, pt[(t) / UB], x, true)
+#define TADV_DC_QU_F(t, x) TADV_DC_ACC(t, pu[(t) % UB], x, false)
+#define TADV_DC_QT_F(t, x) TADV_DC_ACC(t, pt[(t) / UB], x, false)
+#define TADV_DOT_SLOT(J) \
+                const unsigned fk = (unsigned)B.dot_fk[J]; const unsigned off = xo[J], lc = xlc[J], uc = xuc[J]; \
+                const unsigned rs = 0u; (void)rs; const float *base = xbase[J];
+#define TADV_DOTTRIP(ALL, SUF) { \
+                float pu[UB], pt[TA]; \
+                if (pcls == 0) { \
+                    { TADV_DOT_SLOT(0) TADV_XFETCH(TADV_DC_PU, ALL) } \
+                    { TADV_DOT_SLOT(1) TADV_XFETCH(TADV_DC_QU_##SUF, ALL) } \
+                } else { \
+                    { TADV_DOT_SLOT(0) TADV_XFETCH(TADV_DC_PT, ALL) } \
+                    { TADV_DOT_SLOT(1) TADV_XFETCH(TADV_DC_QT_##SUF, ALL) } \
+                } \
+                if (!SM) live |= cur; }
+#define TADV_XLOOP_WIDE(SUMMODE) if constexpr (!DEBUG && !REL && T >= 32) { \
+            constexpr bool SM = (SUMMODE) != 0; \
+            float (&SS)[T] = SM ? m.s[0] : m.acc; \
+            const TadpBody &B = P.bodies[imm]; \
+            const TadpLoop &L = P.loops[a]; \
+            const int V = L.var; \
+            const int kind = B.loop_kind; \
+            const int pcls = B.dot_pclass; \
+            int z = get_var(m.var, V); \
+            const int lane = (int)(threadIdx.x & 31u); \
+            const int dz = kind == BL_USUM ? UB : kind == BL_Z_LANE ? 32 * TA : 1; \
+            const int hi = kind <= BL_USUM ? L.const_hi : loop_hi[a]; \
+            const int lvl = L.mask_level; \
+            const unsigned parent = kind == BL_SUM ? cur : kind == BL_USUM ? sum_parent : mstack[lvl - 1]; \
+            unsigned xo[2], xst[2], xlc[2], xuc[2]; \
+            const float *xbase[2]; \
+            _Pragma("unroll") for (int j = 0; j < 2; ++j) { \
+                const TadpLoad &Ld = P.loads[B.load[j]]; \
+                xo[j] = load_offset(Ld, m.var); xst[j] = (unsigned)Ld.coef[V] * (unsigned)dz; \
+                xlc[j] = (unsigned)Ld.lane_step; xuc[j] = UB > 1 ? (unsigned)Ld.unroll_step : 0u; \
+                xbase[j] = ptrs.in[Ld.ptr]; \
+            } \
+            constexpr unsigned FULL = 0xffffffffu; \
+            for (;;) { \
+                if (cur == FULL) TADV_DOTTRIP(true, T) else TADV_DOTTRIP(false, F) \
+                z += dz; \
+                const int zb = kind == BL_Z_LANE ? z - lane : z; \
+                if (zb > hi) break; \
+                xo[0] += xst[0]; xo[1] += xst[1]; \
+                if (kind == BL_Z_MASKED) { \
+                    unsigned mk = 0; \
+                    _Pragma("unroll") for (int t = 0; t < T; ++t) if (elo[lvl - 1][t] <= z && z <= ehi[lvl - 1][t]) mk |= 1u << t; \
+                    cur = parent & mk; \
+                } else if (zb + dz - 1 > hi) { \
+                    unsigned mk = 0; \
+                    if (kind == BL_USUM) { _Pragma("unroll") for (int t = 0; t < T; ++t) if (z + (t % UB) <= hi) mk |= 1u << t; } \
+                    else { _Pragma("unroll") for (int t = 0; t < T; ++t) if (z + 32 * (t / UB) <= hi) mk |= 1u << t; } \
+                    cur = parent & mk; \
+                } \
+            } \
+            cur = parent; \
+        } else
+#define TADV_XLOOP(SUMMODE) case TADV_H(P_XLOOP, SUMMODE): TADV_XLOOP_WIDE(SUMMODE) if constexpr (!DEBUG && (SUMMODE) + 2 <= VmCfg<TA, UB>::DEPTH) { \
             constexpr int DEPTH = VmCfg<TA, UB>::DEPTH; \
             constexpr int XI = (SUMMODE), YI = XI + 1, I0 = DEPTH - 1, I1 = DEPTH >= 2 ? DEPTH - 2 : 0; \
             const TadpBody &B = P.bodies[imm]; \

@@ -1,6 +1,8 @@
 // The interpreter kernel for one vector shape (TAD_TA x TAD_UB, given on the command line) and its launcher.
 #include <cuda_runtime.h>
 
+#include <algorithm>
+
 #include "vm.cuh"
 
 #ifndef TAD_TA
@@ -15,7 +17,7 @@ using namespace tadvm;
 // except the lane variable A, which the warp covers 32 * TA values at a time, and the element
 // variable B when that is an outer variable, which it covers UB values at a time.
 template <int TA, int UB, bool DEBUG, bool REL>
-__global__ void __launch_bounds__(WARPS_PER_BLOCK * 32, (TA * UB >= 32 ? 1 : 2))
+__global__ void __launch_bounds__(VmCfg<TA, UB>::WARPS * 32, (TA * UB >= 32 ? 3 : 2))
 tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ TadpPointers ptrs, unsigned n_items)
 {
     constexpr int E = TA * UB;
@@ -162,10 +164,13 @@ tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ Tad
 
 // Builds per shape: plain, with the relative-loop support (no element variable) and, for narrow
 // shapes, with bounds checks.
-void TAD_LAUNCH_NAME(TAD_TA, TAD_UB)(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned blocks, cudaStream_t stream)
+void TAD_LAUNCH_NAME(TAD_TA, TAD_UB)(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream)
 {
     constexpr int TA = TAD_TA, UB = TAD_UB;
-    if (debug) { if constexpr (TA <= 4 && UB == 1) tad_vm_kernel<TA, UB, true, true><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(prog, ptrs, items); }
-    else if (prog.rel_var >= 0) { if constexpr (UB == 1) tad_vm_kernel<TA, UB, false, true><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(prog, ptrs, items); }
-    else tad_vm_kernel<TA, UB, false, false><<<blocks, WARPS_PER_BLOCK * 32, 0, stream>>>(prog, ptrs, items);
+    constexpr unsigned WPB = VmCfg<TA, UB>::WARPS;
+    // one warp per work item, grid-stride; at most 128 warps' worth of blocks per SM
+    const unsigned blocks = std::min((items + WPB - 1) / WPB, sms * (128u / WPB));
+    if (debug) { if constexpr (TA <= 4 && UB == 1) tad_vm_kernel<TA, UB, true, true><<<blocks, WPB * 32, 0, stream>>>(prog, ptrs, items); }
+    else if (prog.rel_var >= 0) { if constexpr (UB == 1) tad_vm_kernel<TA, UB, false, true><<<blocks, WPB * 32, 0, stream>>>(prog, ptrs, items); }
+    else tad_vm_kernel<TA, UB, false, false><<<blocks, WPB * 32, 0, stream>>>(prog, ptrs, items);
 }
