@@ -58,10 +58,10 @@ static __device__ __noinline__ float apply_fn(int fn, float x, int n)
 // Inline versions of the functions that dominate element-wise kernels; everything else goes
 // through apply_fn.  Sine and cosine: Cody-Waite reduction by multiples of pi/2 (three-part
 // constant, exact first step) and the degree-7 / degree-8 polynomials of the remainder on
-// [-pi/4, pi/4]; arguments of 8192 and beyond, infinities and NaN take the library routine.
+// [-pi/4, pi/4]; arguments of 8192 and beyond, infinities and NaN take the library routine (the
+// function word tests all values of a thread at once, so that the usual case has no branch per value).
 __device__ __forceinline__ float fast_sincos(float x, int quarter)
 {
-    if (!(fabsf(x) < 8192.f)) return quarter ? cosf(x) : sinf(x);
     const float k = rintf(x * 0.636619772367581f);
     float r = fmaf(k, -1.5703125f, x);
     r = fmaf(k, -4.837512969970703125e-4f, r);
@@ -279,8 +279,13 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
             } \
             switch (fn_code) { \
             case F_EXP: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 1][t] = __expf(m.s[D - 1][t]); } break; \
-            case F_SIN: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 1][t] = fast_sincos(m.s[D - 1][t], 0); } break; \
-            case F_COS: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 1][t] = fast_sincos(m.s[D - 1][t], 1); } break; \
+            case F_SIN: case F_COS: { \
+                const int quarter = fn_code == F_COS ? 1 : 0; \
+                float biggest = 0.f; \
+                _Pragma("unroll") for (int t = 0; t < T; ++t) biggest = fmaxf(biggest, fabsf(m.s[D - 1][t]) < 8192.f ? 0.f : 1.f); \
+                if (biggest == 0.f) { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 1][t] = fast_sincos(m.s[D - 1][t], quarter); } \
+                else { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 1][t] = apply_fn(fn_code, m.s[D - 1][t], imm); } \
+            } break; \
             case F_TANH: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 1][t] = fast_tanh(m.s[D - 1][t]); } break; \
             default: { _Pragma("unroll") for (int t = 0; t < T; ++t) m.s[D - 1][t] = apply_fn(fn_code, m.s[D - 1][t], imm); } break; \
             } } break;

@@ -124,7 +124,23 @@ tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ Tad
         float *dst = ptrs.out;
         const bool accumulate = P.accumulate != 0;
         const bool only_live = P.write_only_live != 0;
-        if (lane_outer) {
+        constexpr unsigned FULL_MASK = E >= 32 ? 0xffffffffu : ((1u << E) - 1u);
+        if (!DEBUG && lane_outer && n_u == UB && in_range == FULL_MASK && !only_live) {
+            // a full tile of outputs: no test per element
+            if (accumulate) {
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const unsigned idx = off + (unsigned)(e / UB) * step_a + (unsigned)(e % UB) * step_b;
+                    dst[idx] += m.acc[e];
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const unsigned idx = off + (unsigned)(e / UB) * step_a + (unsigned)(e % UB) * step_b;
+                    dst[idx] = m.acc[e];
+                }
+            }
+        } else if (lane_outer) {
 #pragma unroll
             for (int e = 0; e < E; ++e) {
                 if ((e % UB) >= n_u) continue;
