@@ -669,17 +669,18 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                 float pt[TA], nt[TA]; \
                 _Pragma("unroll") for (int t = 0; t < TA; ++t) pt[t] = __ldg(xbase[0] + (xo[0] + (unsigned)t * xlc[0])); \
                 for (;;) { \
-                    float q[T]; \
-                    _Pragma("unroll") for (int t = 0; t < TA; ++t) \
-                        _Pragma("unroll") for (int u = 0; u < UB; ++u) q[t * UB + u] = __ldg(xbase[1] + (xo[1] + (unsigned)t * xlc[1] + (unsigned)u * xuc[1])); \
+                    const unsigned qo = xo[1]; \
                     ++z; \
                     const bool more = z <= hi; \
                     if (more) { \
                         xo[0] += xst[0]; xo[1] += xst[1]; \
                         _Pragma("unroll") for (int t = 0; t < TA; ++t) nt[t] = __ldg(xbase[0] + (xo[0] + (unsigned)t * xlc[0])); \
                     } \
-                    _Pragma("unroll") for (int t = 0; t < TA; ++t) \
-                        _Pragma("unroll") for (int u = 0; u < UB; ++u) SS[t * UB + u] = fmaf(pt[t], q[t * UB + u], SS[t * UB + u]); \
+                    _Pragma("unroll") for (int t = 0; t < TA; ++t) { \
+                        float q[UB]; \
+                        _Pragma("unroll") for (int u = 0; u < UB; ++u) q[u] = __ldg(xbase[1] + (qo + (unsigned)t * xlc[1] + (unsigned)u * xuc[1])); \
+                        _Pragma("unroll") for (int u = 0; u < UB; ++u) SS[t * UB + u] = fmaf(pt[t], q[u], SS[t * UB + u]); \
+                    } \
                     if (!more) break; \
                     _Pragma("unroll") for (int t = 0; t < TA; ++t) pt[t] = nt[t]; \
                 } \
