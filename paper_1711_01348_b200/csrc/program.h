@@ -57,7 +57,8 @@ enum TadpOp : int {
     P_ZEND,       // kernel-coordinate loop end
     P_XLOOP,      // every trip of an innermost loop in one word: runs bodies[imm] (a short accumulator program) and the
                   // loop end of loops[a]; follows the loop begin word; k = 1: the loop is a value sum whose accumulator
-                  // is the bottom of the operand stack, k = 0: its terms go to the gradient accumulator
+                  // is the bottom of the operand stack, k = 0: its terms go to the gradient accumulator.  In the
+                  // 32-value shapes the body is a product of two loads (TadpBody::dot) and its steps are not read
     P_NUM_OPS
 };
 

@@ -9,8 +9,10 @@
 // The operand stack is a register array indexed only by compile-time constants: the host
 // encodes the stack depth (or, for loop control, the loop variable) into the handler number
 // of every instruction, so each handler names its registers statically and nothing of the
-// stack spills to local memory.  Transcendental functions are out-of-line calls so that the
-// handler code stays small enough for the instruction cache.
+// stack spills to local memory.  exp, sin, cos and tanh are evaluated inline, a word's values side
+// by side; the other elementary functions are out-of-line calls so that the handler code stays
+// small.  Innermost loops whose body is a short chain of loads and arithmetic run inside one
+// word (P_XLOOP); in the 32-value shapes that word runs products of two loads in loops of their own.
 #pragma once
 #include <cuda_runtime.h>
 #include <limits.h>

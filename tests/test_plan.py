@@ -247,3 +247,44 @@ def test_kernel_stats_and_listing():
     # zero fill of dc, clearing the flags of the split summation, gather, fixed-order reduction
     assert st.terms == 8192 * 8192 * 32 and st.n_launches == 4
     assert "ZLOOP" in plan.disassemble(q["c"]) and "SLOOP" in plan.disassemble(-1)
+
+
+# --------------------------------------------------------------------------- #
+# schedules the compiler is expected to find for the workloads (read from the listings)
+# --------------------------------------------------------------------------- #
+
+def _header(listing: str) -> dict:
+    first = listing.splitlines()[0]
+    return dict(item.split("=") for item in first.lstrip("; ").split())
+
+
+def test_contractions_get_the_product_shape():
+    """Convolution forward and both gradients: every fused loop multiplies two loads, so the 4 x 8
+    product shape applies and dx runs with uniform loops (lanes along the channel index)."""
+    from workloads import configs as W
+    plan = Plan(W.FULL["cfg5"]())
+    for which in (-1, 0, 1):
+        listing = plan.disassemble(which)
+        assert _header(listing)["vec"] == "4x8", listing.splitlines()[0]
+        assert "XLOOP" in listing
+    dx = plan.disassemble(1)
+    assert "lane_dependent=1" not in dx and "relative=1" not in dx
+
+
+def test_split_summations_fill_whole_waves():
+    """Shares of a split summation: work items x shares is close to a multiple of the resident warps."""
+    from workloads import configs as W
+    plan = Plan(W.FULL["cfg2"]())
+    head = _header(plan.disassemble(1))          # db: 512 work items
+    assert int(head["zsplit"]) > 1
+    warps = 512 * int(head["zsplit"])
+    resident = 148 * 16
+    assert abs(warps / resident - round(warps / resident)) < 0.15
+
+
+def test_two_levels_of_shares_when_the_outer_loop_is_short():
+    from workloads import configs as W
+    plan = Plan(W.FULL["cfg4"]())
+    listing = plan.disassemble(1)                # dy: 512 live outputs x 262 144 terms
+    assert listing.count("split=1") == 2
+    assert int(_header(listing)["zsplit"]) > 512
