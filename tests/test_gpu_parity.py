@@ -40,7 +40,7 @@ def test_small_expressions(name):
     check_against_oracle(e, args, df)
 
 
-# Sizes at which the compiler picks its wide vector shapes (2x8, 1x8, 1x4, 16x1 values per thread),
+# Sizes at which the compiler picks its wide vector shapes (4x8, 2x8, 1x8, 1x4, 16x1 values per thread),
 # split summations and fused inner loops, with extents that leave a ragged tail in every direction.
 MID = {
     "intro_mid": (lambda: W.intro(300, 333, 11), ("uniform", -0.5, 0.5)),
@@ -50,6 +50,10 @@ MID = {
     "rowsum_sq_short": (lambda: W.ex_rowsum_sq(333, 9), ("normal", 0, 1)),
     "conv_mid": (lambda: W.conv1d(3, 20, 24, 300, 5), ("normal", 0, 0.1)),
     "matmul_mid": (lambda: W.ex_matmul(150, 67, 1100), ("normal", 0, 1)),
+    # large enough for the 4 x 8 product shape: forward and dw (outer product and per-element operand,
+    # ragged tails along t), then dw and dx with the lanes along c and per-u tap ranges (masked trips)
+    "conv_wide": (lambda: W.conv1d(16, 4, 128, 2400, 5), ("normal", 0, 0.1)),
+    "conv_channels": (lambda: W.conv1d(4, 160, 24, 700, 3), ("normal", 0, 0.1)),
 }
 
 
