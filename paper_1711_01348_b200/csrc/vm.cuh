@@ -648,19 +648,22 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
             constexpr unsigned FULL = 0xffffffffu; \
             if (UB > 1 && pcls == 0 && B.dot_fk[0] == BF_PER_U && B.dot_fk[1] == BF_PER_T && cur == FULL && (kind == BL_SUM || kind == BL_Z)) { \
                 /* outer product, every element live in every trip: one value per u (the same for all lanes) times one \
-                   value per t.  The per-t operand of the next trip is loaded before the multiply-adds of this one. */ \
+                   value per t.  The operands of the next trip are loaded while the multiply-adds of this one run. */ \
                 float pu[UB], pt[TA], nt[TA]; \
+                _Pragma("unroll") for (int u = 0; u < UB; ++u) pu[u] = __ldg(xbase[0] + (xo[0] + (unsigned)u * xuc[0])); \
                 _Pragma("unroll") for (int t = 0; t < TA; ++t) pt[t] = __ldg(xbase[1] + (xo[1] + (unsigned)t * xlc[1])); \
                 for (;;) { \
-                    _Pragma("unroll") for (int u = 0; u < UB; ++u) pu[u] = __ldg(xbase[0] + (xo[0] + (unsigned)u * xuc[0])); \
                     ++z; \
                     const bool more = z <= hi; \
                     if (more) { \
                         xo[0] += xst[0]; xo[1] += xst[1]; \
                         _Pragma("unroll") for (int t = 0; t < TA; ++t) nt[t] = __ldg(xbase[1] + (xo[1] + (unsigned)t * xlc[1])); \
                     } \
-                    _Pragma("unroll") for (int t = 0; t < TA; ++t) \
-                        _Pragma("unroll") for (int u = 0; u < UB; ++u) SS[t * UB + u] = fmaf(pu[u], pt[t], SS[t * UB + u]); \
+                    _Pragma("unroll") for (int u = 0; u < UB; ++u) { \
+                        _Pragma("unroll") for (int t = 0; t < TA; ++t) SS[t * UB + u] = fmaf(pu[u], pt[t], SS[t * UB + u]); \
+                        /* this per-u value is used up: its register takes the value of the next trip */ \
+                        if (more) pu[u] = __ldg(xbase[0] + (xo[0] + (unsigned)u * xuc[0])); \
+                    } \
                     if (!more) break; \
                     _Pragma("unroll") for (int t = 0; t < TA; ++t) pt[t] = nt[t]; \
                 } \
