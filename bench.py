@@ -196,7 +196,7 @@ def run_ours(opts):
             raise SystemExit("--rows is implemented for cfg2 only")
         expr = W.intro(opts.rows, 8192, 32, name=f"cfg2_intro_scaled_rows{opts.rows}")
         args, df = W.make_inputs(expr, W.DIST["cfg2"], seed=0)
-    plan = Plan(expr)
+    plan = Plan(expr, saved_forward=opts.saved_forward)
     d_args = [a.to(dev) for a in args]
     d_df = df.to(dev)
     f = torch.empty(expr.out_shape, dtype=torch.float32, device=dev)
@@ -204,6 +204,8 @@ def run_ours(opts):
     ws = torch.zeros(max(256, plan.workspace_bytes()), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream().cuda_stream
     arg_ptrs = [a.data_ptr() for a in d_args]
+    # a plan compiled with saved_forward reads the forward output of the same step in its backward kernels
+    bwd_ptrs = arg_ptrs + ([f.data_ptr()] if opts.saved_forward else [])
     darg_ptrs = [d.data_ptr() for d in dargs]
     n_args = len(d_args)
     n_stages = plan.num_stages()
@@ -219,11 +221,11 @@ def run_ours(opts):
         if n_stages:
             if events is not None:
                 events[e].record(); e += 1
-            plan.backward_stage(arg_ptrs, d_df.data_ptr(), ws.data_ptr(), ws.numel(), stream)
+            plan.backward_stage(bwd_ptrs, d_df.data_ptr(), ws.data_ptr(), ws.numel(), stream)
         for p in range(n_args):
             if events is not None:
                 events[e].record(); e += 1
-            plan.backward_arg(arg_ptrs, d_df.data_ptr(), p, darg_ptrs[p], ws.data_ptr(), ws.numel(), stream)
+            plan.backward_arg(bwd_ptrs, d_df.data_ptr(), p, darg_ptrs[p], ws.data_ptr(), ws.numel(), stream)
         if events is not None:
             events[e].record()
 
@@ -334,6 +336,7 @@ def run_ours(opts):
                 "data": "synthetic",
                 "config": {"workload": expr.name, "out_shape": expr.out_shape, "arg_shapes": expr.arg_shapes,
                            "l2": L2_NOTE[opts.config],
+                           "saved_forward": bool(opts.saved_forward),
                            "parallelism": "replicas" if world > 1 else "single"},
                 "roofline": roof, "parts": per_part, "cpu_baseline": cpu, "e2e": e2e,
                 "gpu_launches": launches * opts.steps, "clocks": clocks}
@@ -350,6 +353,8 @@ def main():
     ap.add_argument("--config", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--saved-forward", action="store_true",
+                    help="compile the plan with saved_forward: the backward kernels read f of the same step")
     ap.add_argument("--rows", type=int, default=0,
                     help="profiler captures only: shrink the first output extent of cfg2 (not a bench number)")
     opts = ap.parse_args()

@@ -108,7 +108,13 @@ typedef struct {
 typedef struct {
     int32_t debug_bounds;   /* non-zero: kernels range-check every computed address, skip bad
                                accesses and record the first one (tad_debug_status) */
-    int32_t reserved[7];    /* must be zero */
+    int32_t saved_forward;  /* non-zero: the derivative kernels read the forward output f (as tad_forward wrote
+                               it for the same arguments) wherever a derivative expression contains the value
+                               of the whole expression, instead of evaluating it again.  Every backward entry
+                               point then takes n_args + 1 pointers in `args`: the arguments, then f.  The
+                               paper's algorithm keeps no values of the forward pass (Sec. 7); this option
+                               is the usual trade of one |f|-sized read for the recomputation. */
+    int32_t reserved[6];    /* must be zero */
 } tad_options;
 
 /* Limits: n_idx <= 8, argument rank <= 4, kernel dimension kappa <= 4, every tensor
@@ -152,7 +158,9 @@ tad_status tad_forward(const tad_plan *plan, const float *const *args, float *f,
  * equation of Sec. 5.1 (gather form: one owner per output element, no atomics, fp32
  * accumulation); the results of several index expressions of one argument are added
  * (Sec. 5.3: dx <- 0, then accumulate over q).
- *   args   host array of n_args DEVICE pointers
+ *   args   host array of n_args DEVICE pointers; for a plan compiled with saved_forward one more
+ *          entry follows them: the forward output f of the same arguments (read-only), and the
+ *          same holds for tad_backward_stage, tad_backward_arg and tad_backward_noalloc
  *   df     DEVICE pointer, prod(out_shape) floats
  *   dargs  host array of n_args DEVICE pointers; NULL entry = gradient not wanted;
  *          every requested tensor is fully overwritten (zeros where Gamma(beta) is empty)

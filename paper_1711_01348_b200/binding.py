@@ -55,7 +55,7 @@ class _Expr(C.Structure):
 
 
 class _Options(C.Structure):
-    _fields_ = [("debug_bounds", C.c_int32), ("reserved", C.c_int32 * 7)]
+    _fields_ = [("debug_bounds", C.c_int32), ("saved_forward", C.c_int32), ("reserved", C.c_int32 * 6)]
 
 
 class AccessInfo(C.Structure):
@@ -123,7 +123,7 @@ def _i64(values) -> "C.Array":
 class Plan:
     """Owns a tad_plan.  `expr` is any object with the fields of workloads.expr.Expr."""
 
-    def __init__(self, expr, debug_bounds: bool = False):
+    def __init__(self, expr, debug_bounds: bool = False, saved_forward: bool = False):
         keep = []
         e = _Expr()
         e.n_out_dims = len(expr.out_shape)
@@ -161,6 +161,8 @@ class Plan:
         e.nodes = C.cast(nodes, C.POINTER(_Node))
         opt = _Options()
         opt.debug_bounds = 1 if debug_bounds else 0
+        opt.saved_forward = 1 if saved_forward else 0
+        self.saved_forward = bool(saved_forward)
         handle = C.c_void_p()
         _check(lib.tad_compile(C.byref(e), C.byref(opt), C.byref(handle)))
         self._h = handle

@@ -60,6 +60,8 @@ struct Gen {
     int unroll_var = -1;                                      // element variable B (-1: none)
     std::map<int, int> staged;                                // sum node -> pointer slot of its staged adjoint
     std::vector<int> stages_used;                             // pointer slots the derivative reads
+    bool use_f = false;                                       // the value of the root is read from the saved forward output
+    bool reads_f = false;
 
     Gen(tad_plan &pl, int acc) : p(pl), q(acc) {}
 
@@ -185,6 +187,13 @@ struct Gen {
     {
         const NodeH &nd = p.nodes[n];
         if (nd.op == TAD_OP_CONST) return konst((float)nd.imm);
+        if (use_f && n == (int)p.nodes.size() - 1 && free_set == 0) {
+            // f[alpha] as the forward pass wrote it
+            std::vector<int64_t> A(size_t(p.n_out) * n_idx(), 0), off(p.n_out, 0);
+            for (int d = 0; d < p.n_out; ++d) A[size_t(d) * n_idx() + d] = 1;
+            reads_f = true;
+            return make_load(TADP_F_SLOT, A, off, p.n_out, p.out_shape, 0, 0);
+        }
         auto key = std::make_pair(n, free_set);
         auto it = val_memo.find(key);
         if (it != val_memo.end()) return it->second;
@@ -1240,8 +1249,9 @@ void generate_stages(tad_plan &p)
     for (int n = 0; n < root; ++n) {
         const NodeH &nd = p.nodes[n];
         if (!nd.reachable || nd.op != TAD_OP_SUM || nd.scope != 0) continue;
-        if (p.n_args + 1 + (int)p.stages.size() >= TADP_MAX_PTRS) break;
+        if (p.n_args + 1 + (int)p.stages.size() >= TADP_MAX_PTRS - (p.opt.saved_forward ? 1 : 0)) break;
         Gen g(p, -1);
+        g.use_f = p.opt.saved_forward != 0;
         try {
             setup_alpha_gen(p, g);
             std::vector<int64_t> dfA(size_t(p.n_out) * g.n_idx(), 0), dfOff(p.n_out, 0);
@@ -1252,7 +1262,11 @@ void generate_stages(tad_plan &p)
             count_uses(g, adj);
             bool has_sum = false;
             for (const Inst &in : g.inst) if (in.uses && in.op == I_SUM) has_sum = true;
-            if (!has_sum) continue;
+            // with the forward output at hand the adjoint may be a few element-wise operations on df and f:
+            // still evaluated once per alpha, so that the gradient loops read one tensor instead of two
+            bool reads_f = false;
+            for (const Inst &in : g.inst) if (in.uses && in.op == I_LOAD && g.loads[in.load].ptr == TADP_F_SLOT) reads_f = true;
+            if (!has_sum && !reads_f) continue;
             Kernel k;
             std::memset(&k.prog, 0, sizeof k.prog);
             k.out_arg = -1; k.access = -1;
@@ -1281,6 +1295,7 @@ void generate_backward(tad_plan &p, int q)
     const bool zero_fill = p.arg_zero_fill[ap.arg];
 
     Gen g(p, q);
+    g.use_f = p.opt.saved_forward != 0;
     const int R = ap.R, kap = ap.kappa, n = ap.n, rank = ap.rank;
     // outer variables: beta itself when the map is onto the whole argument lattice, else x'
     const bool by_beta = !ap.masked;

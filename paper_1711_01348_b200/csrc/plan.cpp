@@ -25,7 +25,7 @@ void build_expression(tad_plan &p, const tad_expr *e, const tad_options *opt)
     if (!e) throw InvalidArg("expr is NULL");
     if (opt) {
         p.opt = *opt;
-        for (int i = 0; i < 7; ++i) if (opt->reserved[i] != 0) throw InvalidArg("tad_options.reserved must be zero");
+        for (int i = 0; i < 6; ++i) if (opt->reserved[i] != 0) throw InvalidArg("tad_options.reserved must be zero");
     }
     if (e->n_out_dims < 1 || e->n_sum_idx < 0 || e->n_args < 0 || e->n_access < 0 || e->n_nodes < 1)
         throw InvalidArg("negative or zero count in tad_expr");

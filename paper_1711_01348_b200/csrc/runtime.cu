@@ -167,6 +167,10 @@ bool fill_inputs(const tad_plan *plan, const float *const *args, const float *df
         ptrs.in[a] = args[a];
     }
     ptrs.in[plan->n_args] = df;
+    if (plan->opt.saved_forward) {
+        if (!args[plan->n_args]) { tad::set_error("this plan was compiled with saved_forward: args[n_args] must be the forward output f"); return false; }
+        ptrs.in[TADP_F_SLOT] = args[plan->n_args];
+    }
     for (int s = 0; s < (int)plan->stages.size(); ++s)
         ptrs.in[plan->n_args + 1 + s] = reinterpret_cast<const float *>(static_cast<char *>(workspace) + stage_offset(plan, s));
     ptrs.debug = plan->opt.debug_bounds ? static_cast<int32_t *>(workspace) : nullptr;
@@ -298,6 +302,10 @@ tad_status tad_step_host(const tad_plan *plan, const float *const *h_args, const
         st = tad_forward(plan, d_args, d_f, stream);
         if (st != TAD_OK) return st;
         if (!check(cudaMemcpyAsync(h_f, d_f, fbytes, cudaMemcpyDeviceToHost, stream), "copy of f")) return TAD_ERR_CUDA;
+    }
+    if (plan->opt.saved_forward) {
+        if (!h_f) { st = tad_forward(plan, d_args, d_f, stream); if (st != TAD_OK) return st; }   // the backward pass reads f
+        d_args[plan->n_args] = d_f;
     }
     if (plan->opt.debug_bounds && !check(cudaMemsetAsync(ws, 0, 256, stream), "clearing the debug word")) return TAD_ERR_CUDA;
     st = tad_backward(plan, d_args, d_df, d_dargs, ws, tad_workspace_bytes(plan), stream);

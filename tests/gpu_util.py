@@ -13,9 +13,10 @@ ATOL = 1e-6
 
 
 class GpuRun:
-    def __init__(self, expr, args, df, debug_bounds=False):
+    def __init__(self, expr, args, df, debug_bounds=False, saved_forward=False):
         self.expr = expr
-        self.plan = Plan(expr, debug_bounds=debug_bounds)
+        self.saved_forward = saved_forward
+        self.plan = Plan(expr, debug_bounds=debug_bounds, saved_forward=saved_forward)
         dev = torch.device("cuda:0")
         self.args = [a.to(dev).contiguous() for a in args]
         self.df = df.to(dev).contiguous()
@@ -33,7 +34,9 @@ class GpuRun:
     def backward(self, wanted=None):
         stream = torch.cuda.current_stream().cuda_stream
         wanted = [True] * len(self.args) if wanted is None else wanted
-        self.plan.backward([a.data_ptr() for a in self.args], self.df.data_ptr(),
+        # a plan compiled with saved_forward reads the forward output (run forward() first)
+        extra = [self.f.data_ptr()] if self.saved_forward else []
+        self.plan.backward([a.data_ptr() for a in self.args] + extra, self.df.data_ptr(),
                            [d.data_ptr() if w else 0 for d, w in zip(self.dargs, wanted)],
                            self.ws.data_ptr(), self.ws.numel(), stream)
         torch.cuda.synchronize()
@@ -51,8 +54,8 @@ def assert_close(got, want, scale, what=""):
                              f"gpu={got[idx]!r} oracle={want[idx]!r} tol={tol[idx]!r}")
 
 
-def check_against_oracle(expr, args, df, nthreads=1, debug_bounds=False):
-    run = GpuRun(expr, args, df, debug_bounds=debug_bounds)
+def check_against_oracle(expr, args, df, nthreads=1, debug_bounds=False, saved_forward=False):
+    run = GpuRun(expr, args, df, debug_bounds=debug_bounds, saved_forward=saved_forward)
     orc = Oracle(expr)
     f_o, fabs_o = orc.forward(args, nthreads=nthreads)
     assert_close(run.forward(), f_o, fabs_o, f"{expr.name} forward")

@@ -81,6 +81,31 @@ def test_function_argument_sweeps(fn):
     check_against_oracle(e, args, df)
 
 
+@pytest.mark.parametrize("name", ["sec6", "exp_shift", "exp_flat", "all_ops", "one_row"])
+def test_saved_forward_small(name):
+    """Plans that read the forward output instead of evaluating the expression again in the derivative."""
+    make, dist = SMALL[name]
+    e = make()
+    args, df = W.make_inputs(e, dist, seed=2)
+    check_against_oracle(e, args, df, saved_forward=True)
+    check_against_oracle(e, args, df, saved_forward=True, debug_bounds=True)
+
+
+@pytest.mark.parametrize("key", ["cfg1", "cfg2", "cfg3", "cfg5"])
+def test_saved_forward_reduced_workloads(key):
+    e, args, df = W.workload(key, full=False)
+    check_against_oracle(e, args, df, nthreads=max_threads(), saved_forward=True)
+
+
+def test_saved_forward_needs_f():
+    from paper_1711_01348_b200 import TadError
+    e, args, df = W.workload("cfg1", full=False)
+    run = GpuRun(e, args, df, saved_forward=True)
+    with pytest.raises(TadError):
+        run.plan.backward([a.data_ptr() for a in run.args] + [0], run.df.data_ptr(), [d.data_ptr() for d in run.dargs],
+                          run.ws.data_ptr(), run.ws.numel())
+
+
 def test_gradient_subset_and_repeat_calls():
     e, args, df = W.workload("cfg2", full=False)
     run = GpuRun(e, args, df)
