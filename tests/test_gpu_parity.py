@@ -125,3 +125,26 @@ def test_null_pointer_is_rejected():
         run.plan.forward([a.data_ptr() for a in run.args], 0)
     with pytest.raises(TadError):
         run.plan.backward([0] * 4, run.df.data_ptr(), [d.data_ptr() for d in run.dargs])
+
+
+@pytest.mark.parametrize("key,saved", [("cfg2", False), ("cfg2", True), ("cfg4", False), ("cfg5", False)])
+def test_host_buffer_entry_point(key, saved):
+    """tad_step_host: host buffers in, forward and every gradient back, copies inside the call."""
+    from paper_1711_01348_b200 import Plan
+    e, args, df = W.workload(key, full=False)
+    plan = Plan(e, saved_forward=saved)
+    h_args = [a.contiguous().pin_memory() for a in args]
+    h_df = df.contiguous().pin_memory()
+    h_f = torch.full(list(e.out_shape), float("nan"), dtype=torch.float32).pin_memory()
+    h_dargs = [torch.full(list(s), float("nan"), dtype=torch.float32).pin_memory() for s in e.arg_shapes]
+    staging = torch.empty(plan.staging_bytes(), dtype=torch.uint8, device="cuda:0")
+    for _ in range(2):           # the staging area is reused as it stands
+        plan.step_host([a.data_ptr() for a in h_args], h_df.data_ptr(), h_f.data_ptr(),
+                       [d.data_ptr() for d in h_dargs], staging.data_ptr(), staging.numel(),
+                       torch.cuda.current_stream().cuda_stream)
+    orc = Oracle(e)
+    f_o, fabs_o = orc.forward(args, nthreads=max_threads())
+    assert_close(h_f.numpy(), f_o, fabs_o, f"{e.name} forward (host buffers)")
+    dx_o, t_o = orc.backward(args, df, nthreads=max_threads())
+    for p, name in enumerate(e.arg_names):
+        assert_close(h_dargs[p].numpy(), dx_o[p], t_o[p], f"{e.name} d{name} (host buffers)")
