@@ -216,8 +216,10 @@ tad_status tad_backward_noalloc(const tad_plan *plan, const float *const *args, 
 /*
  * tad_step_host: one forward and one backward pass with HOST buffers (same meaning as
  * tad_forward followed by tad_backward).  Inputs are copied to the device staging area,
- * results copied back; all copies and launches are enqueued on the stream and the call
- * returns after the stream has drained.  Host buffers should be pinned for the copies to
+ * results copied back.  The kernels run on the given stream, after whatever it already
+ * holds; the copies run on two streams the call creates and destroys, ordered by events so
+ * that df goes up during the forward pass and f and each gradient come down while the next
+ * kernels run.  The call returns after all of it has drained.  Host buffers should be pinned for the copies to
  * be asynchronous.  staging is a DEVICE buffer of at least tad_staging_bytes() bytes,
  * 256-byte aligned, that the caller allocated; the library allocates nothing.  h_f and
  * entries of h_dargs may be NULL (not wanted).  (The paper has no counterpart; it is the

@@ -285,34 +285,84 @@ tad_status tad_step_host(const tad_plan *plan, const float *const *h_args, const
         if (e != cudaSuccess) { tad::set_error(std::string(what) + ": " + cudaGetErrorString(e)); return false; }
         return true;
     };
+    for (int a = 0; a < plan->n_args; ++a) cur += 2 * pad(size_t(plan->arg_elems[a]) * 4);   // x^p and dx^p, filled below
+    const size_t fbytes = size_t(plan->out_elems) * 4;
+    float *d_f = reinterpret_cast<float *>(cur); cur += pad(fbytes);
+    float *d_df = reinterpret_cast<float *>(cur); cur += pad(fbytes);
+
+    // Copies run on two streams of their own so that they overlap the kernels: df goes up while the
+    // forward pass runs, f and every gradient come down while the next kernels run.
+    struct Side {
+        cudaStream_t in = nullptr, out = nullptr;
+        cudaEvent_t ev[4 + TADP_MAX_PTRS] = {};
+        int n_ev = 0;
+        ~Side()
+        {
+            for (int i = 0; i < n_ev; ++i) if (ev[i]) cudaEventDestroy(ev[i]);
+            if (in) cudaStreamDestroy(in);
+            if (out) cudaStreamDestroy(out);
+        }
+        cudaEvent_t event()
+        {
+            cudaEvent_t e = nullptr;
+            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+            ev[n_ev++] = e;
+            return e;
+        }
+    } side;
+    if (!check(cudaStreamCreateWithFlags(&side.in, cudaStreamNonBlocking), "stream for the copies in") ||
+        !check(cudaStreamCreateWithFlags(&side.out, cudaStreamNonBlocking), "stream for the copies out")) return TAD_ERR_CUDA;
+    cudaEvent_t ev_start = side.event(), ev_args = side.event(), ev_df = side.event(), ev_f = side.event();
+    if (!ev_start || !ev_args || !ev_df || !ev_f) { tad::set_error("event creation failed"); return TAD_ERR_CUDA; }
+    // whatever the caller queued on its stream comes first
+    if (!check(cudaEventRecord(ev_start, stream), "event record") || !check(cudaStreamWaitEvent(side.in, ev_start, 0), "stream wait") ||
+        !check(cudaStreamWaitEvent(side.out, ev_start, 0), "stream wait")) return TAD_ERR_CUDA;
+    cur = static_cast<char *>(staging) + pad(tad_workspace_bytes(plan));
     for (int a = 0; a < plan->n_args; ++a) {
         const size_t bytes = size_t(plan->arg_elems[a]) * 4;
         float *dx = reinterpret_cast<float *>(cur); cur += pad(bytes);
         float *dg = reinterpret_cast<float *>(cur); cur += pad(bytes);
         if (!h_args[a]) { tad::set_error("NULL host argument"); return TAD_ERR_INVALID_ARG; }
-        if (!check(cudaMemcpyAsync(dx, h_args[a], bytes, cudaMemcpyHostToDevice, stream), "copy of an argument")) return TAD_ERR_CUDA;
+        if (!check(cudaMemcpyAsync(dx, h_args[a], bytes, cudaMemcpyHostToDevice, side.in), "copy of an argument")) return TAD_ERR_CUDA;
         d_args[a] = dx; d_dargs[a] = h_dargs[a] ? dg : nullptr;
     }
-    const size_t fbytes = size_t(plan->out_elems) * 4;
-    float *d_f = reinterpret_cast<float *>(cur); cur += pad(fbytes);
-    float *d_df = reinterpret_cast<float *>(cur); cur += pad(fbytes);
-    if (!check(cudaMemcpyAsync(d_df, h_df, fbytes, cudaMemcpyHostToDevice, stream), "copy of df")) return TAD_ERR_CUDA;
+    if (!check(cudaEventRecord(ev_args, side.in), "event record")) return TAD_ERR_CUDA;
+    if (!check(cudaMemcpyAsync(d_df, h_df, fbytes, cudaMemcpyHostToDevice, side.in), "copy of df")) return TAD_ERR_CUDA;
+    if (!check(cudaEventRecord(ev_df, side.in), "event record")) return TAD_ERR_CUDA;
+
     tad_status st = TAD_OK;
-    if (h_f) {
+    if (!check(cudaStreamWaitEvent(stream, ev_args, 0), "stream wait")) return TAD_ERR_CUDA;
+    if (h_f || plan->opt.saved_forward) {
         st = tad_forward(plan, d_args, d_f, stream);
         if (st != TAD_OK) return st;
-        if (!check(cudaMemcpyAsync(h_f, d_f, fbytes, cudaMemcpyDeviceToHost, stream), "copy of f")) return TAD_ERR_CUDA;
+        if (h_f) {
+            if (!check(cudaEventRecord(ev_f, stream), "event record") || !check(cudaStreamWaitEvent(side.out, ev_f, 0), "stream wait") ||
+                !check(cudaMemcpyAsync(h_f, d_f, fbytes, cudaMemcpyDeviceToHost, side.out), "copy of f")) return TAD_ERR_CUDA;
+        }
     }
-    if (plan->opt.saved_forward) {
-        if (!h_f) { st = tad_forward(plan, d_args, d_f, stream); if (st != TAD_OK) return st; }   // the backward pass reads f
-        d_args[plan->n_args] = d_f;
-    }
+    if (plan->opt.saved_forward) d_args[plan->n_args] = d_f;      // the backward pass reads f
+    if (!check(cudaStreamWaitEvent(stream, ev_df, 0), "stream wait")) return TAD_ERR_CUDA;
     if (plan->opt.debug_bounds && !check(cudaMemsetAsync(ws, 0, 256, stream), "clearing the debug word")) return TAD_ERR_CUDA;
-    st = tad_backward(plan, d_args, d_df, d_dargs, ws, tad_workspace_bytes(plan), stream);
-    if (st != TAD_OK) return st;
+    bool need_stage = false;
     for (int a = 0; a < plan->n_args; ++a)
-        if (h_dargs[a] && !check(cudaMemcpyAsync(h_dargs[a], d_dargs[a], size_t(plan->arg_elems[a]) * 4, cudaMemcpyDeviceToHost, stream), "copy of a gradient")) return TAD_ERR_CUDA;
-    if (!check(cudaStreamSynchronize(stream), "stream synchronise")) return TAD_ERR_CUDA;
+        if (d_dargs[a])
+            for (int ki : plan->arg_kernels[a]) if (!plan->backward[ki].stages_used.empty()) need_stage = true;
+    if (need_stage) {
+        st = tad_backward_stage(plan, d_args, d_df, ws, tad_workspace_bytes(plan), stream);
+        if (st != TAD_OK) return st;
+    }
+    for (int a = 0; a < plan->n_args; ++a) {
+        if (!d_dargs[a]) continue;
+        st = tad_backward_arg(plan, d_args, d_df, a, d_dargs[a], ws, tad_workspace_bytes(plan), stream);
+        if (st != TAD_OK) return st;
+        cudaEvent_t ev_g = side.event();
+        if (!ev_g) { tad::set_error("event creation failed"); return TAD_ERR_CUDA; }
+        if (!check(cudaEventRecord(ev_g, stream), "event record") || !check(cudaStreamWaitEvent(side.out, ev_g, 0), "stream wait") ||
+            !check(cudaMemcpyAsync(h_dargs[a], d_dargs[a], size_t(plan->arg_elems[a]) * 4, cudaMemcpyDeviceToHost, side.out), "copy of a gradient"))
+            return TAD_ERR_CUDA;
+    }
+    if (!check(cudaStreamSynchronize(stream), "stream synchronise") || !check(cudaStreamSynchronize(side.out), "stream synchronise") ||
+        !check(cudaStreamSynchronize(side.in), "stream synchronise")) return TAD_ERR_CUDA;
     return TAD_OK;
 }
 
