@@ -663,14 +663,14 @@ void finish_stats(Gen &g, Kernel &k, bool backward, int64_t outputs, int64_t ter
 // uses the sector in full; a strided load that does not depend on B is fetched once for all its
 // elements.  Candidates: outer variables (a tile of gradient elements per thread) and bound
 // sums (several summands per trip).
-void choose_element_variable(Gen &g, bool allow_outer_product)
+void choose_element_variable(Gen &g, bool allow_outer_product, uint32_t excluded = 0)
 {
     g.unroll_var = -1;
     if (g.p.opt.debug_bounds) return;            // debug plans use the narrow kernels
     const int A = g.lane_var;
     double best = 0;
     for (int v = 0; v < (int)g.vars.size(); ++v) {
-        if (v == A || g.vars[v].ext < 4 || g.vars[v].kind == 1) continue;
+        if (v == A || g.vars[v].ext < 4 || g.vars[v].kind == 1 || ((excluded >> v) & 1u)) continue;
         if (g.vars[v].kind == 2 && (g.vars[v].sum_inst < 0 || !g.inst[g.vars[v].sum_inst].uses)) continue;
         double score = 0;
         bool fixes_strided = false;
@@ -910,7 +910,16 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
         for (const TadpRow &r : lower[l]) if (r.coef[g.lane_var]) relative_candidate = true;
         for (const TadpRow &r : upper[l]) if (r.coef[g.lane_var]) relative_candidate = true;
     }
-    choose_element_variable(g, !relative_candidate);
+    // the loop over the lane variable takes one range for the whole thread: a variable that its bounds
+    // depend on cannot give the thread's elements different values
+    uint32_t lane_bound_vars = 0;
+    for (int l = 0; l < g.kappa; ++l) {
+        if (g.n_outer + g.zorder[l] != g.lane_var) continue;
+        for (const std::vector<TadpRow> *rows : {&lower[l], &upper[l]})
+            for (const TadpRow &r : *rows)
+                for (int x = 0; x < (int)g.vars.size(); ++x) if (r.coef[x]) lane_bound_vars |= 1u << x;
+    }
+    choose_element_variable(g, !relative_candidate, lane_bound_vars);
     // temporaries: shared values and values hoisted out of the loop that consumes them
     std::vector<bool> hoisted(g.inst.size(), false);
     auto effective_level = [&](int i) { return i == root ? g.kappa : g.inst[i].zlevel; };

@@ -148,3 +148,49 @@ def test_host_buffer_entry_point(key, saved):
     dx_o, t_o = orc.backward(args, df, nthreads=max_threads())
     for p, name in enumerate(e.arg_names):
         assert_close(h_dargs[p].numpy(), dx_o[p], t_o[p], f"{e.name} d{name} (host buffers)")
+
+
+@pytest.mark.parametrize("seed", range(80))
+def test_random_expressions(seed):
+    """Random index maps (strides, negative and repeated indices, several index expressions of one
+    argument) and random function trees, every gradient against the oracle."""
+    from paper_1711_01348_b200 import TadError
+    from workloads.random_expr import random_expression
+    e = random_expression(seed)
+    args, df = W.make_inputs(e, ("uniform", -1, 1), seed=seed)
+    try:
+        check_against_oracle(e, args, df, debug_bounds=seed % 3 == 0, saved_forward=seed % 4 == 1)
+    except TadError as exc:
+        if "TAD_ERR_UNSUPPORTED" in str(exc) or "TAD_ERR_OVERFLOW" in str(exc):
+            pytest.skip(str(exc))
+        raise
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_expressions_large(seed):
+    """The same at extents where the wide vector shapes, element variables and split summations apply."""
+    from paper_1711_01348_b200 import TadError
+    from workloads.random_expr import random_expression
+    e = random_expression(seed, large=1)
+    args, df = W.make_inputs(e, ("uniform", -1, 1), seed=seed)
+    try:
+        check_against_oracle(e, args, df, nthreads=max_threads(), saved_forward=seed % 4 == 1)
+    except TadError as exc:
+        if "TAD_ERR_UNSUPPORTED" in str(exc) or "TAD_ERR_OVERFLOW" in str(exc):
+            pytest.skip(str(exc))
+        raise
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_expressions_huge(seed):
+    """... and with millions of outputs: 16 values per thread, element variables, fused loops."""
+    from paper_1711_01348_b200 import TadError
+    from workloads.random_expr import random_expression
+    e = random_expression(seed, large=2)
+    args, df = W.make_inputs(e, ("uniform", -1, 1), seed=seed)
+    try:
+        check_against_oracle(e, args, df, nthreads=max_threads(), saved_forward=seed % 4 == 1)
+    except TadError as exc:
+        if "TAD_ERR_UNSUPPORTED" in str(exc) or "TAD_ERR_OVERFLOW" in str(exc):
+            pytest.skip(str(exc))
+        raise

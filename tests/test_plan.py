@@ -288,3 +288,40 @@ def test_two_levels_of_shares_when_the_outer_loop_is_short():
     listing = plan.disassemble(1)                # dy: 512 live outputs x 262 144 terms
     assert listing.count("split=1") == 2
     assert int(_header(listing)["zsplit"]) > 512
+
+
+def _lane_loop_row_variables(listing: str) -> set:
+    """Variables with a non-zero coefficient in a bound row of the loop over the lane variable."""
+    import re
+    rows = {}
+    for line in listing.splitlines():
+        m = re.match(r"; row (\d+) \((-?\d+) \+ ([-\d ]+)\) / (-?\d+)", line)
+        if m:
+            rows[int(m.group(1))] = [int(x) for x in m.group(3).split()]
+    used = set()
+    for line in listing.splitlines():
+        m = re.match(r"; loop \d+ var=\d+ lane=1 .* lower=(\d+)\+(\d+) upper=(\d+)\+(\d+)", line)
+        if not m:
+            continue
+        l0, nl, u0, nu = map(int, m.groups())
+        for r in list(range(l0, l0 + nl)) + list(range(u0, u0 + nu)):
+            used |= {v for v, c in enumerate(rows[r]) if c}
+    return used
+
+
+def test_lane_loop_bounds_do_not_depend_on_the_element_variable():
+    """The loop over the lane variable takes one range per thread, so a variable in its bound rows
+    may not be the element variable (the thread's values would need a range each).  Seed 8 of the
+    largest generator level has a gradient whose summation ranges depend on the gradient index."""
+    from workloads.random_expr import random_expression
+    cases = [(8, 2)] + [(s, 1) for s in range(12)] + [(s, 2) for s in range(12)]
+    for seed, level in cases:
+        try:
+            plan = Plan(random_expression(seed, level))
+        except TadError:
+            continue
+        for which in range(len(plan.expr.accesses)):
+            listing = plan.disassemble(which)
+            u = int(_header(listing)["unroll_var"])
+            if u >= 0:
+                assert u not in _lane_loop_row_variables(listing), (seed, level, which)

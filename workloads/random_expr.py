@@ -1,0 +1,93 @@
+"""Seeded random expressions for the parity tests: random integer affine index maps (strides,
+negative coefficients, repeated and constant indices, several index expressions per argument),
+random trees of elementary functions, optionally one inner sum.  Data only: nothing here
+evaluates an expression."""
+from __future__ import annotations
+
+from typing import List
+
+import numpy as np
+
+from .expr import Builder, Expr
+
+
+def random_expression(seed: int, large: int = 0) -> Expr:
+    """large = 1, 2: extents at which split summations, then the wide vector shapes and element variables apply."""
+    rng = np.random.default_rng(seed + 100003 * large)
+    n_out = int(rng.integers(1, 4))
+    top = [[48, 14, 7], [6000, 400, 48], [3000000, 1800, 150]][large]
+    out_shape = [int(rng.integers(max(2, top[n_out - 1] // 3) if large else 2, top[n_out - 1] + 1)) for _ in range(n_out)]
+    n_sum = int(rng.integers(0, 2))
+    sum_len = int(rng.integers(1, 7)) if n_sum else 0
+    n_idx = n_out + n_sum
+    ext = out_shape + ([sum_len] if n_sum else [])
+    n_args = int(rng.integers(1, 4))
+    names = ["x", "y", "w"][:n_args]
+    ranks = [int(rng.integers(1, 3)) for _ in range(n_args)]
+
+    # leaves: (argument, rows, offset) with every index inside [0, shape)
+    leaves = []
+    shapes = [[1] * r for r in ranks]
+
+    def make_leaf(inside_sum: bool):
+        # arguments stay below 3 M elements: a leaf that would make its argument larger is drawn again
+        for _ in range(50):
+            saved = [list(sh) for sh in shapes]
+            leaf = draw_leaf(inside_sum)
+            if int(np.prod(shapes[leaf[0]], dtype=np.int64)) <= 3_000_000:
+                return leaf
+            for k, sh in enumerate(saved):
+                shapes[k][:] = sh
+        # a constant index always fits
+        p = int(rng.integers(0, n_args))
+        return p, [[0] * n_idx for _ in range(ranks[p])], [0] * ranks[p]
+
+    def draw_leaf(inside_sum: bool):
+        p = int(rng.integers(0, n_args))
+        rows, offs = [], []
+        for r in range(ranks[p]):
+            row = [0] * n_idx
+            for d in range(n_idx):
+                if d >= n_out and not inside_sum:
+                    continue
+                if rng.random() < 0.55:
+                    row[d] = int(rng.choice([1, 1, 1, 2, 3, -1, -2]))
+            lo = sum(min(0, c * (ext[d] - 1)) for d, c in enumerate(row))
+            hi = sum(max(0, c * (ext[d] - 1)) for d, c in enumerate(row))
+            off = -lo + int(rng.integers(0, 3))
+            rows.append(row); offs.append(off)
+            shapes[p][r] = max(shapes[p][r], hi + off + 1 + int(rng.integers(0, 2)))
+        return p, rows, offs
+
+    n_in = int(rng.integers(1, 4)) if n_sum else 0
+    n_outside = int(rng.integers(1 if not n_sum else 0, 4))
+    inside = [make_leaf(True) for _ in range(n_in)]
+    outside = [make_leaf(False) for _ in range(n_outside)]
+
+    b = Builder(f"random_{large}_{seed}", out_shape, n_sum, names, shapes)
+    # the shapes grew while the leaves were drawn
+    b.e.arg_shapes = [list(s) for s in shapes]
+
+    def tree(leaf_ids: List[int]) -> int:
+        nodes = list(leaf_ids)
+        for k in range(len(nodes)):
+            if rng.random() < 0.5:
+                op = str(rng.choice(["sin", "cos", "tanh", "exp", "neg", "sq", "cube"]))
+                nodes[k] = b.powi(nodes[k], 2) if op == "sq" else b.powi(nodes[k], 3) if op == "cube" else b.un(op, nodes[k])
+        while len(nodes) > 1:
+            i = int(rng.integers(0, len(nodes) - 1))
+            op = str(rng.choice(["add", "mul", "mul", "sub"]))
+            nodes[i:i + 2] = [b.bin(op, nodes[i], nodes[i + 1])]
+        root = nodes[0]
+        if rng.random() < 0.3:
+            root = b.bin("mul", root, b.const(float(rng.choice([2.0, -0.5, 3.0]))))
+        return root
+
+    parts = [b.load(names[p], rows, offs) for p, rows, offs in outside]
+    if n_sum:
+        body = tree([b.load(names[p], rows, offs) for p, rows, offs in inside])
+        parts.append(b.sum(n_out, 0, sum_len - 1, body))
+    root = tree(parts)
+    if rng.random() < 0.3:
+        b.un(str(rng.choice(["exp", "tanh", "sin"])), root)
+    return b.done()
