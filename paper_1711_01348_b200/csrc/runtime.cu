@@ -351,7 +351,12 @@ tad_status tad_step_host(const tad_plan *plan, const float *const *h_args, const
         st = tad_backward_stage(plan, d_args, d_df, ws, tad_workspace_bytes(plan), stream);
         if (st != TAD_OK) return st;
     }
-    for (int a = 0; a < plan->n_args; ++a) {
+    // largest gradient first: its copy to the host runs while the kernels of the others do
+    int order[TADP_MAX_PTRS];
+    for (int a = 0; a < plan->n_args; ++a) order[a] = a;
+    std::stable_sort(order, order + plan->n_args, [&](int x, int y) { return plan->arg_elems[x] > plan->arg_elems[y]; });
+    for (int oi = 0; oi < plan->n_args; ++oi) {
+        const int a = order[oi];
         if (!d_dargs[a]) continue;
         st = tad_backward_arg(plan, d_args, d_df, a, d_dargs[a], ws, tad_workspace_bytes(plan), stream);
         if (st != TAD_OK) return st;
