@@ -273,8 +273,12 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
         TADV_D1(TADV_ADDC, P_ADDC)
 #define TADV_FN(OP, D) TADV_CASE(OP, D, D) { \
             if (UB > 1 && a) { \
+                /* the operand is the same for every u: one evaluation per t, taken from the first live u \
+                   (a value sum leaves the elements that are masked off unfinished) */ \
                 _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { \
-                    const float r = apply_fn(fn_code, m.s[D - 1][ta * UB], imm); \
+                    float src = m.s[D - 1][ta * UB + UB - 1]; \
+                    _Pragma("unroll") for (int u = UB - 2; u >= 0; --u) if ((cur >> (ta * UB + u)) & 1u) src = m.s[D - 1][ta * UB + u]; \
+                    const float r = apply_fn(fn_code, src, imm); \
                     _Pragma("unroll") for (int u = 0; u < UB; ++u) m.s[D - 1][ta * UB + u] = r; \
                 } \
                 break; \

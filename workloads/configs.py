@@ -247,6 +247,19 @@ def ex_rowsum_sq(n: int, nk: int) -> Expr:
     return b.done()
 
 
+def ex_guarded_shared_fn(ni: int, nj: int, ns: int, nt: int) -> Expr:
+    """f_ij = sum_s (cos x_{i+1} + w_s) tanh(sum_t 0.1 y_{nj-1-j}^2) with x longer than the image of i + 1: the
+    gradient of x has elements with no term at both ends, and the function of the inner sum is the same
+    for every element of x."""
+    b = Builder("ex_guarded_shared_fn", [ni, nj], 2, ["x", "y", "w"], [[nj], [nj], [ns]])
+    xi = b.load("x", [[1, 0, 0, 0]], [1])
+    ws = b.load("w", [[0, 0, 1, 0]])
+    yj = b.load("y", [[0, -1, 0, 0]], [nj - 1])
+    inner = b.sum(3, 0, nt - 1, b.bin("mul", b.powi(yj, 2), b.const(0.1)))
+    b.sum(2, 0, ns - 1, b.bin("mul", b.bin("add", b.un("cos", xi), ws), b.un("tanh", inner)))
+    return b.done()
+
+
 def ex_exp_flat(n: int, m: int) -> Expr:
     """f^5_ij = exp x_{M i + j}, i in [0, n), j in [0, m)  (Sec. 5)."""
     b = Builder("ex_exp_flat", [n, m], 0, ["x"], [[n * m]])

@@ -1,7 +1,7 @@
 """Seeded random expressions for the parity tests: random integer affine index maps (strides,
 negative coefficients, repeated and constant indices, several index expressions per argument),
-random trees of elementary functions, optionally one inner sum.  Data only: nothing here
-evaluates an expression."""
+random trees of elementary functions, optionally one inner sum (level 3: two sums, one inside
+the other, with leaves at every depth).  Data only: nothing here evaluates an expression."""
 from __future__ import annotations
 
 from typing import List
@@ -12,15 +12,21 @@ from .expr import Builder, Expr
 
 
 def random_expression(seed: int, large: int = 0) -> Expr:
-    """large = 1, 2: extents at which split summations, then the wide vector shapes and element variables apply."""
+    """large = 1, 2: extents at which split summations, then the wide vector shapes and element variables apply;
+    large = 3: a sum of up to 40 terms inside a sum of up to 12, medium extents."""
     rng = np.random.default_rng(seed + 100003 * large)
     n_out = int(rng.integers(1, 4))
-    top = [[48, 14, 7], [6000, 400, 48], [3000000, 1800, 150]][large]
+    top = [[48, 14, 7], [6000, 400, 48], [3000000, 1800, 150], [3000, 160, 28]][large]
     out_shape = [int(rng.integers(max(2, top[n_out - 1] // 3) if large else 2, top[n_out - 1] + 1)) for _ in range(n_out)]
-    n_sum = int(rng.integers(0, 2))
-    sum_len = int(rng.integers(1, 7)) if n_sum else 0
+    if large == 3:
+        n_sum = 2
+        sum_lens = [int(rng.integers(1, 13)), int(rng.integers(1, 41))]
+    else:
+        n_sum = int(rng.integers(0, 2))
+        sum_lens = [int(rng.integers(1, 7))] if n_sum else []
+    sum_len = sum_lens[0] if n_sum else 0
     n_idx = n_out + n_sum
-    ext = out_shape + ([sum_len] if n_sum else [])
+    ext = out_shape + sum_lens
     n_args = int(rng.integers(1, 4))
     names = ["x", "y", "w"][:n_args]
     ranks = [int(rng.integers(1, 3)) for _ in range(n_args)]
@@ -29,7 +35,7 @@ def random_expression(seed: int, large: int = 0) -> Expr:
     leaves = []
     shapes = [[1] * r for r in ranks]
 
-    def make_leaf(inside_sum: bool):
+    def make_leaf(inside_sum):
         # arguments stay below 3 M elements: a leaf that would make its argument larger is drawn again
         for _ in range(50):
             saved = [list(sh) for sh in shapes]
@@ -42,13 +48,15 @@ def random_expression(seed: int, large: int = 0) -> Expr:
         p = int(rng.integers(0, n_args))
         return p, [[0] * n_idx for _ in range(ranks[p])], [0] * ranks[p]
 
-    def draw_leaf(inside_sum: bool):
+    def draw_leaf(inside_sum):
+        # inside_sum: False = output indices only, True = all indices, an int = that many leading indices
+        n_allowed = n_out if inside_sum is False else n_idx if inside_sum is True else int(inside_sum)
         p = int(rng.integers(0, n_args))
         rows, offs = [], []
         for r in range(ranks[p]):
             row = [0] * n_idx
             for d in range(n_idx):
-                if d >= n_out and not inside_sum:
+                if d >= n_allowed:
                     continue
                 if rng.random() < 0.55:
                     row[d] = int(rng.choice([1, 1, 1, 2, 3, -1, -2]))
@@ -63,14 +71,19 @@ def random_expression(seed: int, large: int = 0) -> Expr:
     n_outside = int(rng.integers(1 if not n_sum else 0, 4))
     inside = [make_leaf(True) for _ in range(n_in)]
     outside = [make_leaf(False) for _ in range(n_outside)]
+    middle = [make_leaf(n_out + 1) for _ in range(int(rng.integers(0, 3)))] if large == 3 else []
 
     b = Builder(f"random_{large}_{seed}", out_shape, n_sum, names, shapes)
     # the shapes grew while the leaves were drawn
     b.e.arg_shapes = [list(s) for s in shapes]
 
-    def tree(leaf_ids: List[int]) -> int:
+    def tree(leaf_ids: List[int], n_leaves: int = -1) -> int:
+        # level 3 applies functions to index expressions only (n_leaves of the ids), never to a sum: a function of
+        # a long cancelling sum is ill-conditioned in fp32 and says nothing about the code under test
         nodes = list(leaf_ids)
         for k in range(len(nodes)):
+            if large == 3 and k >= n_leaves:
+                continue
             if rng.random() < 0.5:
                 op = str(rng.choice(["sin", "cos", "tanh", "exp", "neg", "sq", "cube"]))
                 nodes[k] = b.powi(nodes[k], 2) if op == "sq" else b.powi(nodes[k], 3) if op == "cube" else b.un(op, nodes[k])
@@ -84,7 +97,13 @@ def random_expression(seed: int, large: int = 0) -> Expr:
         return root
 
     parts = [b.load(names[p], rows, offs) for p, rows, offs in outside]
-    if n_sum:
+    if n_sum == 2:
+        inner = b.sum(n_out + 1, 0, sum_lens[1] - 1, tree([b.load(names[p], rows, offs) for p, rows, offs in inside], len(inside)))
+        body = tree([b.load(names[p], rows, offs) for p, rows, offs in middle] + [inner], len(middle))
+        parts.append(b.sum(n_out, 0, sum_lens[0] - 1, body))
+        tree(parts, len(outside))
+        return b.done()
+    elif n_sum:
         body = tree([b.load(names[p], rows, offs) for p, rows, offs in inside])
         parts.append(b.sum(n_out, 0, sum_len - 1, body))
     root = tree(parts)
