@@ -232,3 +232,21 @@ def test_random_expressions_nested_sums(seed):
         if "TAD_ERR_UNSUPPORTED" in str(exc) or "TAD_ERR_OVERFLOW" in str(exc):
             pytest.skip(str(exc))
         raise
+
+
+@pytest.mark.parametrize("seed", range(50))
+def test_random_expressions_all_functions(seed):
+    """One or two sums (the inner one up to 64 terms), up to 2e5 outputs, and log, division, sinh and
+    cosh among the functions, their arguments kept inside their domains."""
+    from paper_1711_01348_b200 import TadError
+    from workloads.random_expr import random_expression
+    e = random_expression(seed, large=4)
+    args, df = W.make_inputs(e, ("uniform", -1, 1), seed=seed)
+    if not _well_conditioned(e, args, df, max_threads()):
+        pytest.skip("ill-conditioned in fp32 (decided by the oracle alone)")
+    try:
+        check_against_oracle(e, args, df, nthreads=max_threads(), saved_forward=seed % 4 == 1)
+    except TadError as exc:
+        if "TAD_ERR_UNSUPPORTED" in str(exc) or "TAD_ERR_OVERFLOW" in str(exc):
+            pytest.skip(str(exc))
+        raise

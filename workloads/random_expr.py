@@ -13,14 +13,19 @@ from .expr import Builder, Expr
 
 def random_expression(seed: int, large: int = 0) -> Expr:
     """large = 1, 2: extents at which split summations, then the wide vector shapes and element variables apply;
-    large = 3: a sum of up to 40 terms inside a sum of up to 12, medium extents."""
+    large = 3: a sum of up to 40 terms inside a sum of up to 12, medium extents;
+    large = 4: one or two sums, the inner one up to 64 terms, up to 2e5 outputs, and the remaining elementary
+    functions (log, division, sinh, cosh) with arguments kept inside their domains."""
     rng = np.random.default_rng(seed + 100003 * large)
     n_out = int(rng.integers(1, 4))
-    top = [[48, 14, 7], [6000, 400, 48], [3000000, 1800, 150], [3000, 160, 28]][large]
+    top = [[48, 14, 7], [6000, 400, 48], [3000000, 1800, 150], [3000, 160, 28], [200000, 600, 60]][large]
     out_shape = [int(rng.integers(max(2, top[n_out - 1] // 3) if large else 2, top[n_out - 1] + 1)) for _ in range(n_out)]
     if large == 3:
         n_sum = 2
         sum_lens = [int(rng.integers(1, 13)), int(rng.integers(1, 41))]
+    elif large == 4:
+        n_sum = int(rng.integers(1, 3))
+        sum_lens = [int(rng.integers(1, 9)), int(rng.integers(1, 65))][2 - n_sum:]
     else:
         n_sum = int(rng.integers(0, 2))
         sum_lens = [int(rng.integers(1, 7))] if n_sum else []
@@ -71,7 +76,7 @@ def random_expression(seed: int, large: int = 0) -> Expr:
     n_outside = int(rng.integers(1 if not n_sum else 0, 4))
     inside = [make_leaf(True) for _ in range(n_in)]
     outside = [make_leaf(False) for _ in range(n_outside)]
-    middle = [make_leaf(n_out + 1) for _ in range(int(rng.integers(0, 3)))] if large == 3 else []
+    middle = [make_leaf(n_out + 1) for _ in range(int(rng.integers(0, 3)))] if large >= 3 and n_sum == 2 else []
 
     b = Builder(f"random_{large}_{seed}", out_shape, n_sum, names, shapes)
     # the shapes grew while the leaves were drawn
@@ -82,7 +87,19 @@ def random_expression(seed: int, large: int = 0) -> Expr:
         # a long cancelling sum is ill-conditioned in fp32 and says nothing about the code under test
         nodes = list(leaf_ids)
         for k in range(len(nodes)):
-            if large == 3 and k >= n_leaves:
+            if large >= 3 and k >= n_leaves:
+                continue
+            if large == 4 and rng.random() < 0.35:
+                # arguments are drawn from [-1, 1]: 1.5 + x and 2 + x stay positive
+                op = str(rng.choice(["log", "recip", "sinh", "cosh", "quot"]))
+                if op == "log":
+                    nodes[k] = b.un("log", b.bin("add", nodes[k], b.const(1.5)))
+                elif op == "recip":
+                    nodes[k] = b.bin("div", b.const(1.0), b.bin("add", nodes[k], b.const(2.0)))
+                elif op == "quot":
+                    nodes[k] = b.bin("div", nodes[k], b.bin("add", b.powi(nodes[k], 2), b.const(1.0)))
+                else:
+                    nodes[k] = b.un(op, nodes[k])
                 continue
             if rng.random() < 0.5:
                 op = str(rng.choice(["sin", "cos", "tanh", "exp", "neg", "sq", "cube"]))
@@ -101,6 +118,11 @@ def random_expression(seed: int, large: int = 0) -> Expr:
         inner = b.sum(n_out + 1, 0, sum_lens[1] - 1, tree([b.load(names[p], rows, offs) for p, rows, offs in inside], len(inside)))
         body = tree([b.load(names[p], rows, offs) for p, rows, offs in middle] + [inner], len(middle))
         parts.append(b.sum(n_out, 0, sum_lens[0] - 1, body))
+        tree(parts, len(outside))
+        return b.done()
+    elif large == 4:
+        body = tree([b.load(names[p], rows, offs) for p, rows, offs in inside], len(inside))
+        parts.append(b.sum(n_out, 0, sum_len - 1, body))
         tree(parts, len(outside))
         return b.done()
     elif n_sum:
