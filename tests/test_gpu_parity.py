@@ -250,3 +250,13 @@ def test_random_expressions_all_functions(seed):
         if "TAD_ERR_UNSUPPORTED" in str(exc) or "TAD_ERR_OVERFLOW" in str(exc):
             pytest.skip(str(exc))
         raise
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_contractions(seed):
+    """Products of two index expressions under one or two sums, 4e4 to 4e6 outputs: the product
+    kernels (32 sums per thread) and the shapes next to them, with random strides and offsets."""
+    from workloads.random_expr import random_expression
+    e = random_expression(seed, large=5)
+    args, df = W.make_inputs(e, ("normal", 0, 1), seed=seed)
+    check_against_oracle(e, args, df, nthreads=max_threads(), saved_forward=seed % 4 == 1)

@@ -15,7 +15,10 @@ def random_expression(seed: int, large: int = 0) -> Expr:
     """large = 1, 2: extents at which split summations, then the wide vector shapes and element variables apply;
     large = 3: a sum of up to 40 terms inside a sum of up to 12, medium extents;
     large = 4: one or two sums, the inner one up to 64 terms, up to 2e5 outputs, and the remaining elementary
-    functions (log, division, sinh, cosh) with arguments kept inside their domains."""
+    functions (log, division, sinh, cosh) with arguments kept inside their domains;
+    large = 5: contractions, a product of two index expressions under one or two sums (the product kernels)."""
+    if large == 5:
+        return _random_contraction(seed)
     rng = np.random.default_rng(seed + 100003 * large)
     n_out = int(rng.integers(1, 4))
     top = [[48, 14, 7], [6000, 400, 48], [3000000, 1800, 150], [3000, 160, 28], [200000, 600, 60]][large]
@@ -131,4 +134,48 @@ def random_expression(seed: int, large: int = 0) -> Expr:
     root = tree(parts)
     if rng.random() < 0.3:
         b.un(str(rng.choice(["exp", "tanh", "sin"])), root)
+    return b.done()
+
+
+def _random_contraction(seed: int) -> Expr:
+    """f_alpha = sum_{s0[, s1]} x[...] * y[...] with random index maps: every index appears in at least one
+    factor, coefficients from {1, 1, 1, 2, -1}; 4e4 .. 4e6 outputs, 8 .. 300 terms each."""
+    rng = np.random.default_rng(seed + 100003 * 5)
+    n_out = int(rng.integers(2, 4))
+    sizes = [[int(rng.integers(100, 800)), int(rng.integers(400, 3000))],
+             [int(rng.integers(2, 20)), int(rng.integers(16, 160)), int(rng.integers(200, 1200))]][n_out - 2]
+    out_shape = [int(v) for v in rng.permutation(sizes)]
+    n_sum = int(rng.integers(1, 3))
+    sum_lens = [int(rng.integers(8, 65))] if n_sum == 1 else [int(rng.integers(8, 49)), int(rng.integers(2, 7))]
+    n_idx = n_out + n_sum
+    ext = out_shape + sum_lens
+    ranks = [int(rng.integers(1, 4)), int(rng.integers(1, 4))]
+    while True:
+        maps = []
+        for r in ranks:
+            rows = [[0] * n_idx for _ in range(r)]
+            for d in range(n_idx):
+                if rng.random() < 0.6:
+                    rows[int(rng.integers(0, r))][d] = int(rng.choice([1, 1, 1, 2, -1]))
+            maps.append(rows)
+        used = [any(rows[k][d] for rows in maps for k in range(len(rows))) for d in range(n_idx)]
+        sizes_ok = True
+        shapes, offsets = [], []
+        for rows in maps:
+            shape, offs = [], []
+            for row in rows:
+                lo = sum(min(0, c * (ext[d] - 1)) for d, c in enumerate(row))
+                hi = sum(max(0, c * (ext[d] - 1)) for d, c in enumerate(row))
+                shift = int(rng.integers(0, 2))
+                offs.append(-lo + shift)
+                shape.append(hi - lo + 1 + shift + int(rng.integers(0, 3)))
+            shapes.append(shape); offsets.append(offs)
+            if int(np.prod(shape, dtype=np.int64)) > 3_000_000:
+                sizes_ok = False
+        if all(used) and sizes_ok:
+            break
+    b = Builder(f"random_5_{seed}", out_shape, n_sum, ["x", "y"], shapes)
+    prod = b.bin("mul", b.load("x", maps[0], offsets[0]), b.load("y", maps[1], offsets[1]))
+    for k in range(n_sum - 1, -1, -1):
+        prod = b.sum(n_out + k, 0, sum_lens[k] - 1, prod)
     return b.done()
