@@ -260,3 +260,50 @@ def test_random_contractions(seed):
     e = random_expression(seed, large=5)
     args, df = W.make_inputs(e, ("normal", 0, 1), seed=seed)
     check_against_oracle(e, args, df, nthreads=max_threads(), saved_forward=seed % 4 == 1)
+
+
+@pytest.mark.parametrize("level,seed", [(lv, sd) for lv in (0, 1, 3, 4) for sd in range(12)])
+def test_entry_points_agree(level, seed):
+    """tad_backward with every gradient, with a subset of them (the others untouched), the entry point
+    with its own scratch and the host-buffer step run the same kernels: bit-identical results."""
+    from paper_1711_01348_b200 import TadError
+    from workloads.random_expr import random_expression
+    e = random_expression(seed, large=level)
+    args, df = W.make_inputs(e, ("normal", 0, 0.7), seed=seed)
+    saved = seed % 2 == 1
+    try:
+        run = GpuRun(e, args, df, saved_forward=saved)
+    except TadError as exc:
+        if "TAD_ERR_UNSUPPORTED" in str(exc) or "TAD_ERR_OVERFLOW" in str(exc):
+            pytest.skip(str(exc))
+        raise
+    f = run.forward()
+    d = run.backward()
+    stream = torch.cuda.current_stream().cuda_stream
+    extra = [run.f.data_ptr()] if saved else []
+    if run.plan.workspace_bytes() <= 32 << 20:
+        outs = [torch.full(list(s), float("nan"), dtype=torch.float32, device="cuda:0") for s in e.arg_shapes]
+        run.plan.backward_noalloc([x.data_ptr() for x in run.args] + extra, run.df.data_ptr(),
+                                  [o.data_ptr() for o in outs], stream)
+        torch.cuda.synchronize()
+        for p, o in enumerate(outs):
+            assert np.array_equal(o.cpu().numpy(), d[p], equal_nan=True), f"own scratch, gradient {p}"
+    wanted = [(seed >> p) & 1 == 0 for p in range(len(e.arg_shapes))]
+    other = GpuRun(e, args, df, saved_forward=saved)
+    other.forward()
+    sub = other.backward(wanted)
+    for p, w in enumerate(wanted):
+        if w:
+            assert np.array_equal(sub[p], d[p], equal_nan=True), f"subset, gradient {p}"
+        else:
+            assert np.all(np.isnan(other.dargs[p].cpu().numpy())), f"gradient {p} was not asked for but written"
+    h_args = [x.contiguous().pin_memory() for x in args]
+    h_df = df.contiguous().pin_memory()
+    h_f = torch.full(list(e.out_shape), float("nan"), dtype=torch.float32).pin_memory()
+    h_d = [torch.full(list(s), float("nan"), dtype=torch.float32).pin_memory() for s in e.arg_shapes]
+    staging = torch.empty(run.plan.staging_bytes(), dtype=torch.uint8, device="cuda:0")
+    run.plan.step_host([x.data_ptr() for x in h_args], h_df.data_ptr(), h_f.data_ptr(), [x.data_ptr() for x in h_d],
+                       staging.data_ptr(), staging.numel(), stream)
+    assert np.array_equal(h_f.numpy(), f, equal_nan=True), "host buffers, f"
+    for p in range(len(h_d)):
+        assert np.array_equal(h_d[p].numpy(), d[p], equal_nan=True), f"host buffers, gradient {p}"
