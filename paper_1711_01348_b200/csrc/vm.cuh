@@ -506,36 +506,42 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
 #define TADV_XC_ADDSQ(t, x) { const float w2 = op_add(m.s[XI][t], (x)); m.s[XI][t] = op_mul(w2, w2); }
         // fetches one load of the body in the manner the host chose and hands every element's value to COMBINE;
         // ALL: every element of the thread is live (no predicates, signed 64-bit addressing from element 0)
-#define TADV_XFETCH(COMBINE, ALL) \
-                            if (REL && rs != 0) { \
+#define TADV_XF_REL(COMBINE, ALL) { \
                                 /* inside a relative loop: every element reads at its own position of that loop */ \
                                 _Pragma("unroll") for (int t = 0; t < T; ++t) { \
                                     const unsigned idx = off + (unsigned)(t / UB) * lc + (unsigned)(t % UB) * uc + rs * (unsigned)zrel(t); \
-                                    const float x = (ALL || ((cur >> t) & 1u)) ? __ldg(base + idx) : 0.f; COMBINE(t, x) } \
-                            } else switch (fk) { \
-                            case BF_ONE: { \
+                                    const float x = (ALL || ((cur >> t) & 1u)) ? __ldg(base + idx) : 0.f; COMBINE(t, x) } }
+#define TADV_XF_ONE(COMBINE, ALL) { \
                                 const float x = (ALL || cur) ? __ldg(base + off) : 0.f; \
-                                _Pragma("unroll") for (int t = 0; t < T; ++t) { COMBINE(t, x) } \
-                            } break; \
-                            case BF_PER_T: if constexpr (UB > 1) { \
+                                _Pragma("unroll") for (int t = 0; t < T; ++t) { COMBINE(t, x) } }
+#define TADV_XF_PER_T(COMBINE, ALL) { if constexpr (UB > 1) { \
                                 _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { \
                                     const unsigned mm = ALL ? 1u : (cur >> (ta * UB)) & ((1u << UB) - 1u); \
                                     const unsigned idx = off + (unsigned)ta * lc; \
                                     const float x = mm ? __ldg(base + idx) : 0.f; \
                                     _Pragma("unroll") for (int u = 0; u < UB; ++u) { COMBINE(ta * UB + u, x) } \
-                                } \
-                            } break; \
-                            case BF_PER_U: if constexpr (UB > 1) { \
+                                } } }
+#define TADV_XF_PER_U(COMBINE, ALL) { if constexpr (UB > 1) { \
                                 _Pragma("unroll") for (int u = 0; u < UB; ++u) { \
                                     unsigned mm = ALL ? 1u : 0u; \
                                     if (!ALL) { _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) mm |= (cur >> (ta * UB + u)) & 1u; } \
                                     const unsigned idx = off + (unsigned)u * uc; \
                                     const float x = mm ? __ldg(base + idx) : 0.f; \
                                     _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { COMBINE(ta * UB + u, x) } \
-                                } \
-                            } break; \
-                            case BF_ROW: if constexpr (UB > 1 && UB % 4 == 0) { \
+                                } } }
+#define TADV_XF_EACH(COMBINE, ALL) { \
+                                if (ALL) { \
+                                    const float *p0 = base + off; \
+                                    _Pragma("unroll") for (int t = 0; t < T; ++t) { const float x = __ldg(p0 + ((t / UB) * (int)lc + (t % UB) * (int)uc)); COMBINE(t, x) } \
+                                } else { \
+                                    _Pragma("unroll") for (int t = 0; t < T; ++t) { const unsigned idx = off + (unsigned)(t / UB) * lc + (unsigned)(t % UB) * uc; const float x = ((cur >> t) & 1u) ? __ldg(base + idx) : 0.f; COMBINE(t, x) } \
+                                } }
+        // rows of four along the element variable as 128-bit loads when the pointer allows, else element by element
+#define TADV_XF_ROW(COMBINE, ALL) { \
+                                bool rows_done = false; \
+                                if constexpr (UB > 1 && UB % 4 == 0) { \
                                 if ((reinterpret_cast<uintptr_t>(base) & 15u) == 0) { \
+                                    rows_done = true; \
                                     _Pragma("unroll") for (int ta = 0; ta < TA; ++ta) { \
                                         const unsigned ob = off + (unsigned)ta * lc; \
                                         _Pragma("unroll") for (int g4 = 0; g4 < UB / 4; ++g4) { \
@@ -550,19 +556,23 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                                             _Pragma("unroll") for (int i = 0; i < 4; ++i) { COMBINE(ta * UB + 4 * g4 + i, q[i]) } \
                                         } \
                                     } \
-                                    break; \
-                                } \
-                            } \
-                            [[fallthrough]]; \
-                            default: \
-                                if (ALL) { \
-                                    const float *p0 = base + off; \
-                                    _Pragma("unroll") for (int t = 0; t < T; ++t) { const float x = __ldg(p0 + ((t / UB) * (int)lc + (t % UB) * (int)uc)); COMBINE(t, x) } \
-                                } else { \
-                                    _Pragma("unroll") for (int t = 0; t < T; ++t) { const unsigned idx = off + (unsigned)(t / UB) * lc + (unsigned)(t % UB) * uc; const float x = ((cur >> t) & 1u) ? __ldg(base + idx) : 0.f; COMBINE(t, x) } \
-                                } \
-                                break; \
+                                } } \
+                                if (!rows_done) TADV_XF_EACH(COMBINE, ALL) }
+#define TADV_XFETCH(COMBINE, ALL) \
+                            if (REL && rs != 0) TADV_XF_REL(COMBINE, ALL) \
+                            else switch (fk) { \
+                            case BF_ONE: TADV_XF_ONE(COMBINE, ALL) break; \
+                            case BF_PER_T: TADV_XF_PER_T(COMBINE, ALL) break; \
+                            case BF_PER_U: TADV_XF_PER_U(COMBINE, ALL) break; \
+                            case BF_ROW: TADV_XF_ROW(COMBINE, ALL) break; \
+                            default: TADV_XF_EACH(COMBINE, ALL) break; \
                             }
+        // one dispatch per load step: fetch kind and combine together select the code
+#define TADV_XF_CASES(KIND, FETCH, ALL) \
+                            case (KIND) * 4 + 0: FETCH(TADV_XC_SET, ALL) break; \
+                            case (KIND) * 4 + 1: FETCH(TADV_XC_ADD, ALL) break; \
+                            case (KIND) * 4 + 2: FETCH(TADV_XC_MUL, ALL) break; \
+                            case (KIND) * 4 + 3: FETCH(TADV_XC_ADDSQ, ALL) break;
         // the steps of one trip and the term that closes it
 #define TADV_XTRIP(SUMMODE, ALL) { \
                 unsigned w0 = steps.x, w1 = steps.y; \
@@ -571,17 +581,21 @@ __device__ __forceinline__ void run_item(const TadpProgram &P, const TadpPointer
                     if (c == 0) break; \
                     w0 = __funnelshift_r(w0, w1, 8); w1 >>= 8; \
                     if (c & 0x80u) { \
-                        const unsigned j = c & 3u, cmb = (c >> 2) & 3u, fk = (c >> 4) & 7u; \
+                        const unsigned j = c & 3u; \
                         const unsigned off = TADV_XSEL(j, xo); \
                         const unsigned lc = TADV_XSEL(j, xlc); \
                         const unsigned uc = TADV_XSEL(j, xuc); \
                         const unsigned rs = REL ? TADV_XSEL(j, xrs) : 0u; (void)rs; \
                         const float *base = TADV_XSEL(j, xbase); \
-                        switch (cmb) { \
-                        case 0: TADV_XFETCH(TADV_XC_SET, ALL) break; \
-                        case 1: TADV_XFETCH(TADV_XC_ADD, ALL) break; \
-                        case 2: TADV_XFETCH(TADV_XC_MUL, ALL) break; \
-                        default: TADV_XFETCH(TADV_XC_ADDSQ, ALL) break; \
+                        if (REL && rs != 0) { \
+                            switch ((c >> 2) & 3u) { TADV_XF_CASES(0, TADV_XF_REL, ALL) } \
+                        } else switch ((c >> 2) & 0x1fu) {   /* fetch kind x 4 + combine */ \
+                        TADV_XF_CASES(BF_ONE, TADV_XF_ONE, ALL) \
+                        TADV_XF_CASES(BF_PER_T, TADV_XF_PER_T, ALL) \
+                        TADV_XF_CASES(BF_PER_U, TADV_XF_PER_U, ALL) \
+                        TADV_XF_CASES(BF_ROW, TADV_XF_ROW, ALL) \
+                        TADV_XF_CASES(BF_EACH, TADV_XF_EACH, ALL) \
+                        default: break; \
                         } \
                     } else { \
                         switch (c) { \
