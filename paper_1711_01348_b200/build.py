@@ -48,6 +48,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
         jobs.append((common + [f"-DTAD_TA={ta}", f"-DTAD_UB={ub}", "-c", os.path.join(CSRC, "vm_inst.cu"), "-o", obj],
                      f"vm_inst {ta}x{ub}"))
 
+    # the 16 x 1 shape once more with 168 registers per thread (kernels whose fused loop runs under per-element masks)
+    jobs.append((common + ["-DTAD_TA=16", "-DTAD_UB=1", "-DTAD_RICH_BUILD=1", "-c", os.path.join(CSRC, "vm_inst.cu"),
+                           "-o", os.path.join(OBJ, "vm_16_1_rich.o")], "vm_inst 16x1 rich"))
+
     def run(job):
         cmd, name = job
         res = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)

@@ -1149,13 +1149,18 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
             B.dot_pclass = load_class(prog.loads[B.load[0]], pick.ta, pick.ub);
             for (int j = 0; j < 2; ++j) B.dot_fk[j] = body_fetch_kind(prog.loads[B.load[j]], pick.ta, pick.ub);
         }
+    // a fused loop under per-element masks keeps a range per element besides the values: measured faster with
+    // 168 registers and 12 warps per SM than with 128 and 16 (cfg4 dx 0.90 -> 0.73 ms), unlike everything else
+    k.rich = false;
+    if (pick.ta == 16 && pick.ub == 1 && !debug && prog.rel_var < 0)
+        for (const TadpBody &B : bodies) if (B.loop_kind == BL_Z_MASKED) k.rich = true;
     prog.n_bodies = (int32_t)bodies.size();
     std::copy(bodies.begin(), bodies.end(), prog.bodies);
     prog.n_code = (int32_t)em.code.size();
     std::copy(em.code.begin(), em.code.end(), prog.code);
     char head[256];
-    std::snprintf(head, sizeof head, "; vars=%zu outer=%d kappa=%d lane_var=%d unroll_var=%d vec=%dx%d zsplit=%d temps=%d max_depth=%d loads=%d rows=%d guards=%d\n",
-                  g.vars.size(), g.n_outer, g.kappa, g.lane_var, g.unroll_var, k.vec, k.vec_u, prog.zsplit, n_temps, em.max_depth, prog.n_loads, prog.n_rows, prog.n_guards);
+    std::snprintf(head, sizeof head, "; vars=%zu outer=%d kappa=%d lane_var=%d unroll_var=%d vec=%dx%d%s zsplit=%d temps=%d max_depth=%d loads=%d rows=%d guards=%d\n",
+                  g.vars.size(), g.n_outer, g.kappa, g.lane_var, g.unroll_var, k.vec, k.vec_u, k.rich ? "r" : "", prog.zsplit, n_temps, em.max_depth, prog.n_loads, prog.n_rows, prog.n_guards);
     k.listing = head + em.listing();
     // tables the code refers to: variables, loads, loops, bound rows
     auto coefs = [&](const int32_t *c) {

@@ -65,6 +65,7 @@ struct Kernel {
     int access = -1;
     int vec = 4;               // elements per thread along the lane variable (TA)
     int vec_u = 1;             // elements per thread along the element variable (UB)
+    bool rich = false;         // the build of the shape with more registers per thread and fewer warps per SM
     std::vector<int> stages_used;   // backward: staged adjoints it reads (indices into tad_plan::stages)
     KernelStats stats;
     std::string listing;

@@ -18,6 +18,7 @@ void set_error(const std::string &m);
 // One build of the interpreter per vector shape, each in an object file of its own (vm_inst.cu).
 #define TAD_DECLARE_VM(TA, UB) void tad_launch_vm_##TA##_##UB(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream);
 TAD_VM_SHAPES(TAD_DECLARE_VM)
+void tad_launch_vm_16_1_rich(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream);
 
 namespace {
 
@@ -105,7 +106,8 @@ tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStrea
     if (items64 == 0) return TAD_OK;
     if (items64 >= (1ull << 32)) { tad::set_error("too many work items"); return TAD_ERR_UNSUPPORTED; }
     const unsigned items = (unsigned)items64;
-    switch (k.vec * 100 + k.vec_u) {
+    if (k.rich && !debug && k.vec == 16 && k.vec_u == 1) tad_launch_vm_16_1_rich(k.prog, ptrs, debug, items, (unsigned)sm_count(), stream);
+    else switch (k.vec * 100 + k.vec_u) {
 #define TAD_CASE_VM(TA, UB) case TA * 100 + UB: tad_launch_vm_##TA##_##UB(k.prog, ptrs, debug, items, (unsigned)sm_count(), stream); break;
     TAD_VM_SHAPES(TAD_CASE_VM)
     default: tad::set_error("internal: no kernel for this vector shape"); return TAD_ERR_UNSUPPORTED;

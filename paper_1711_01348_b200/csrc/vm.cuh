@@ -91,13 +91,17 @@ __device__ __forceinline__ float fast_tanh(float x)
 // Per vector width: NTR temporaries kept in registers (the rest spill to local memory) and the
 // usable operand stack depth.  Wide vectors amortise the dispatch cost over more elements and
 // pay for it with a shallower stack; the host picks the widest variant a program fits.
+#ifndef TAD_RICH_BUILD
+#define TAD_RICH_BUILD 0
+#endif
 template <int TA, int UB>
 struct VmCfg {
     static constexpr int E = TA * UB;           // values per thread and operand
     static constexpr int NTR = E >= 16 ? 0 : E >= 8 ? 2 : TADP_NUM_TEMPS;
     // 32 values per thread: the shapes of the product kernels; one operand slot, blocks of 4 warps
     static constexpr int DEPTH = E >= 32 ? 1 : E >= 16 ? TADP_WIDE_DEPTH : STACK;
-    static constexpr int WARPS = E >= 32 ? 4 : TADP_WARPS_PER_BLOCK;
+    // TAD_RICH_BUILD: blocks of 6 warps, two per SM: 168 registers per thread instead of 128
+    static constexpr int WARPS = E >= 32 ? 4 : TAD_RICH_BUILD ? 6 : TADP_WARPS_PER_BLOCK;
 };
 
 template <int TA, int UB>

@@ -176,7 +176,12 @@ tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ Tad
 }  // namespace
 
 #define TAD_CAT3(a, b, c, d) a##b##c##d
+#if TAD_RICH_BUILD
+#define TAD_CAT4(a, b, c, d, e) a##b##c##d##e
+#define TAD_LAUNCH_NAME(TA, UB) TAD_CAT4(tad_launch_vm_, TA, _, UB, _rich)
+#else
 #define TAD_LAUNCH_NAME(TA, UB) TAD_CAT3(tad_launch_vm_, TA, _, UB)
+#endif
 
 // Builds per shape: plain, with the relative-loop support (no element variable) and, for narrow
 // shapes, with bounds checks.
