@@ -2,6 +2,7 @@
 
 The interpreter kernel is compiled once per vector shape (vm_inst.cu with -DTAD_TA / -DTAD_UB),
 every shape into an object file of its own, several at a time; the objects land in _build/.
+The 16 x 1 shape is compiled twice: once more with 168 registers per thread and blocks of 6 warps.
 """
 from __future__ import annotations
 

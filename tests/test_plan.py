@@ -325,3 +325,11 @@ def test_lane_loop_bounds_do_not_depend_on_the_element_variable():
             u = int(_header(listing)["unroll_var"])
             if u >= 0:
                 assert u not in _lane_loop_row_variables(listing), (seed, level, which)
+
+
+def test_masked_fused_loops_get_the_register_rich_build():
+    """cfg4 dx walks its summation under per-element masks: the 16 x 1 build with more registers per thread."""
+    from workloads import configs as W
+    plan = Plan(W.FULL["cfg4"]())
+    assert _header(plan.disassemble(0))["vec"] == "16x1r"
+    assert _header(plan.disassemble(-1))["vec"] == "16x1" and _header(plan.disassemble(1))["vec"] == "16x1"
