@@ -1,0 +1,347 @@
+// Tile kernel for contraction programs (contract.h): a thread block owns a BM x BN tile of
+// outputs, gathers BK summation indices of both operands at a time into shared memory with
+// asynchronous copies (three stages in flight), and every thread keeps a TM x TN tile of sums in
+// registers that it feeds from shared memory with 128-bit loads.  Operand elements outside a
+// guard, past the end of the summation range or in the ragged edge of a tile arrive as zeros
+// (zero-fill copies), so the multiply-add loop has no tests.  No atomics: a summation split over
+// several blocks writes planes of partial sums that tad_contract_reduce adds in a fixed order.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <climits>
+
+#include "contract.h"
+#include "program.h"
+
+namespace {
+
+constexpr int BK = TADC_BK;
+constexpr int STAGES = 3;
+constexpr int DEAD = INT_MIN / 2;      // guard part of a row or summation index that does not exist
+
+__device__ __forceinline__ void cp_async4(float *dst, const float *src, bool live)
+{
+    const unsigned d = (unsigned)__cvta_generic_to_shared(dst);
+    const int bytes = live ? 4 : 0;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;\n" ::"r"(d), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async16(float *dst, const float *src, bool live)
+{
+    const unsigned d = (unsigned)__cvta_generic_to_shared(dst);
+    const int bytes = live ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(d), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+struct Parts { int a, b, o, ga, gb; };
+
+// digits of a flattened index, last digit fastest, folded into the offset parts of the group
+__device__ __forceinline__ Parts decode(const TadcGroup &G, unsigned idx)
+{
+    Parts p{0, 0, 0, 0, 0};
+#pragma unroll
+    for (int d = TADC_MAX_DIGITS - 1; d >= 0; --d) {
+        if (d < G.n_digits) {
+            const unsigned e = (unsigned)G.ext[d];
+            const unsigned q = idx / e;
+            const int r = (int)(idx - q * e);
+            idx = q;
+            p.a += r * G.sA[d]; p.b += r * G.sB[d]; p.o += r * G.sO[d];
+            p.ga += r * G.gA[d]; p.gb += r * G.gB[d];
+        }
+    }
+    return p;
+}
+
+// one stage of one operand: BK x BR values into smem[kl * (BR + 4) + rl]
+template <int BR, int NT>
+__device__ __forceinline__ void gather(float *smem, const float *__restrict__ src, const int2 *rows, const int4 *ktab,
+                                       const bool second, const int mode, const unsigned gext, const int tid)
+{
+    constexpr int LD = BR + 4;
+    if (mode == TG_ROW16) {
+        constexpr int CH = BR / 4, TOTAL = CH * BK, PER = (TOTAL + NT - 1) / NT;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const int c = tid + NT * j;
+            if (TOTAL % NT == 0 || c < TOTAL) {
+                const int rl = (c % CH) * 4, kl = c / CH;
+                const int2 r = rows[rl];
+                const int4 kt = ktab[kl];
+                const bool live = (unsigned)(r.y + (second ? kt.w : kt.z)) < gext;
+                cp_async16(smem + kl * LD + rl, src + (live ? (unsigned)(r.x + (second ? kt.y : kt.x)) : 0u), live);
+            }
+        }
+    } else if (mode == TG_ROW) {
+        constexpr int TOTAL = BR * BK, PER = (TOTAL + NT - 1) / NT;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const int e = tid + NT * j;
+            if (TOTAL % NT == 0 || e < TOTAL) {
+                const int rl = e % BR, kl = e / BR;
+                const int2 r = rows[rl];
+                const int4 kt = ktab[kl];
+                const bool live = (unsigned)(r.y + (second ? kt.w : kt.z)) < gext;
+                cp_async4(smem + kl * LD + rl, src + (live ? (unsigned)(r.x + (second ? kt.y : kt.x)) : 0u), live);
+            }
+        }
+    } else {
+        constexpr int TOTAL = BR * BK, PER = (TOTAL + NT - 1) / NT;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const int e = tid + NT * j;
+            if (TOTAL % NT == 0 || e < TOTAL) {
+                const int kl = e % BK, rl = e / BK;
+                const int2 r = rows[rl];
+                const int4 kt = ktab[kl];
+                const bool live = (unsigned)(r.y + (second ? kt.w : kt.z)) < gext;
+                cp_async4(smem + kl * LD + rl, src + (live ? (unsigned)(r.x + (second ? kt.y : kt.x)) : 0u), live);
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ float own_tanh(float x)
+{
+    const float ax = fabsf(x);
+    const float e = __expf(2.f * ax);
+    const float t = 1.f - __fdividef(2.f, e + 1.f);
+    const float x2 = x * x;
+    const float small = x * (1.f + x2 * (-0.33333334f + x2 * (0.13333334f + x2 * -0.05396825f)));
+    return ax < 0.25f ? small : copysignf(t, x);
+}
+
+// the steps every finished sum goes through before it is stored
+__device__ __forceinline__ float epilogue(const TadcProgram &P, const TadpPointers &ptrs, float v, unsigned off)
+{
+    for (int s = 0; s < P.n_epi; ++s) {
+        switch (P.epi_op[s]) {
+        case TE_NEG: v = -v; break;
+        case TE_EXP: v = __expf(v); break;
+        case TE_MULC: v *= P.epi_imm[s]; break;
+        case TE_ADDC: v += P.epi_imm[s]; break;
+        case TE_SQR: v *= v; break;
+        case TE_TANH: v = own_tanh(v); break;
+        case TE_MUL_LOAD: v *= __ldg(ptrs.in[P.epi_ptr[s]] + (unsigned)(P.epi_base[s] + (int)off)); break;
+        case TE_ADD_LOAD: v += __ldg(ptrs.in[P.epi_ptr[s]] + (unsigned)(P.epi_base[s] + (int)off)); break;
+        default: break;
+        }
+    }
+    return v;
+}
+
+template <int BM, int BN, int TM, int TN>
+struct Cfg {
+    static constexpr int NT = (BM / TM) * (BN / TN);
+    static constexpr int LDA = BM + 4, LDB = BN + 4;
+    static constexpr int STAGE_FLOATS = BK * (LDA + LDB);
+    static constexpr size_t SMEM = size_t(STAGES) * STAGE_FLOATS * 4 + size_t(BM + BN) * 8 + size_t(BM + BN) * 4 +
+                                   size_t(STAGES + 1) * BK * 16;
+};
+
+template <int BM, int BN, int TM, int TN>
+__global__ void __launch_bounds__(Cfg<BM, BN, TM, TN>::NT, (TM * TN >= 64 ? 2 : 3))
+tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant__ TadpPointers ptrs, const unsigned tiles_m, const unsigned tiles_n)
+{
+    using C = Cfg<BM, BN, TM, TN>;
+    constexpr int NT = C::NT, LDA = C::LDA, LDB = C::LDB;
+    constexpr int GM = TM / 4, GN = TN / 4;           // groups of four rows / columns per thread
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *stage_mem = reinterpret_cast<float *>(smem_raw);
+    int4 *ktab = reinterpret_cast<int4 *>(stage_mem + STAGES * C::STAGE_FLOATS);
+    int2 *rowA = reinterpret_cast<int2 *>(ktab + (STAGES + 1) * BK);
+    int2 *rowB = rowA + BM;
+    int *outM = reinterpret_cast<int *>(rowB + BN);
+    int *outN = outM + BM;
+
+    const int tid = threadIdx.x;
+    const unsigned tile = blockIdx.x;
+    const unsigned tile_m = tile % tiles_m, tile_n = tile / tiles_m;
+    const unsigned ks = blockIdx.y, zb = blockIdx.z;
+    const Parts z = decode(P.Z, zb);
+    // Offsets are sums of signed 32-bit parts that may be negative one by one (a band that starts below
+    // zero, a negative stride); only the complete sum of a live element is a valid element offset, so the
+    // constant parts go into the row tables and the pointer stays the tensor's own.
+    const float *__restrict__ A = ptrs.in[P.ptrA];
+    const float *__restrict__ B = ptrs.in[P.ptrB];
+    const int constA = P.baseA + z.a, constB = P.baseB + z.b;
+    const unsigned Mext = (unsigned)P.M.extent, Next = (unsigned)P.N.extent;
+    const unsigned kbeg = ks * (unsigned)P.kchunk;
+    const unsigned kend = min((unsigned)P.K.extent, kbeg + (unsigned)P.kchunk);
+    const int n_stages = (int)((kend - kbeg + BK - 1) / BK);
+
+    // per-row parts of the operand offsets, guards and output offsets of this tile
+    for (int r = tid; r < BM; r += NT) {
+        const unsigned m = tile_m * BM + r;
+        if (m < Mext) { const Parts p = decode(P.M, m); rowA[r] = make_int2(constA + p.a, P.guardA_c0 + z.ga + p.ga); outM[r] = p.o; }
+        else { rowA[r] = make_int2(0, DEAD); outM[r] = 0; }
+    }
+    for (int r = tid; r < BN; r += NT) {
+        const unsigned n = tile_n * BN + r;
+        if (n < Next) { const Parts p = decode(P.N, n); rowB[r] = make_int2(constB + p.b, P.guardB_c0 + z.gb + p.gb); outN[r] = p.o; }
+        else { rowB[r] = make_int2(0, DEAD); outN[r] = 0; }
+    }
+    auto fill_ktab = [&](int kstage) {
+        if (tid < BK) {
+            const unsigned k = kbeg + (unsigned)kstage * BK + tid;
+            int4 e = make_int4(0, 0, DEAD, DEAD);
+            if (k < kend) { const Parts p = decode(P.K, k); e = make_int4(p.a, p.b, p.ga, p.gb); }
+            ktab[(kstage % (STAGES + 1)) * BK + tid] = e;
+        }
+    };
+    for (int s = 0; s < STAGES; ++s) fill_ktab(s);
+    __syncthreads();
+    const unsigned gextA = (unsigned)P.guardA_ext, gextB = (unsigned)P.guardB_ext;
+    const int modeA = P.modeA, modeB = P.modeB;
+    auto issue = [&](int kstage) {
+        if (kstage < n_stages) {
+            float *as = stage_mem + (kstage % STAGES) * C::STAGE_FLOATS;
+            float *bs = as + BK * LDA;
+            const int4 *kt = ktab + (kstage % (STAGES + 1)) * BK;
+            gather<BM, NT>(as, A, rowA, kt, false, modeA, gextA, tid);
+            gather<BN, NT>(bs, B, rowB, kt, true, modeB, gextB, tid);
+        }
+        cp_async_commit();
+    };
+    for (int s = 0; s < STAGES - 1; ++s) issue(s);
+
+    const int tx = tid % (BN / TN), ty = tid / (BN / TN);
+    float acc[TM][TN];
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
+
+    for (int it = 0; it < n_stages; ++it) {
+        cp_async_wait<STAGES - 2>();
+        __syncthreads();
+        fill_ktab(it + STAGES);
+        issue(it + STAGES - 1);
+        const float *as = stage_mem + (it % STAGES) * C::STAGE_FLOATS;
+        const float *bs = as + BK * LDA;
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            float a[TM], b[TN];
+#pragma unroll
+            for (int g = 0; g < GM; ++g) {
+                const float4 v = *reinterpret_cast<const float4 *>(as + kk * LDA + g * (BM / GM) + ty * 4);
+                a[4 * g] = v.x; a[4 * g + 1] = v.y; a[4 * g + 2] = v.z; a[4 * g + 3] = v.w;
+            }
+#pragma unroll
+            for (int g = 0; g < GN; ++g) {
+                const float4 v = *reinterpret_cast<const float4 *>(bs + kk * LDB + g * (BN / GN) + tx * 4);
+                b[4 * g] = v.x; b[4 * g + 1] = v.y; b[4 * g + 2] = v.z; b[4 * g + 3] = v.w;
+            }
+#pragma unroll
+            for (int i = 0; i < TM; ++i)
+#pragma unroll
+                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+    }
+    cp_async_wait<0>();
+
+    // ---- store ----
+    const bool partial = P.ksplit > 1;
+    float *__restrict__ out = partial ? ptrs.part : ptrs.out;
+    const float scale = P.scale;
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+        const int rl = (i / 4) * (BM / GM) + ty * 4 + (i % 4);
+        const unsigned m = tile_m * BM + rl;
+        if (m >= Mext) continue;
+#pragma unroll
+        for (int g = 0; g < GN; ++g) {
+            const int cl = g * (BN / GN) + tx * 4;
+            const unsigned n = tile_n * BN + cl;
+            if (n >= Next) continue;
+            if (partial) {
+                float *dst = out + ((size_t)(zb * (unsigned)P.ksplit + ks) * Mext + m) * Next + n;
+                if ((Next & 3u) == 0) *reinterpret_cast<float4 *>(dst) = make_float4(acc[i][4 * g], acc[i][4 * g + 1], acc[i][4 * g + 2], acc[i][4 * g + 3]);
+                else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) if (n + j < Next) dst[j] = acc[i][4 * g + j];
+                }
+            } else {
+                const int ob = P.baseO + z.o + outM[rl];
+                if (P.out_vec4) {
+                    const unsigned off = (unsigned)(ob + outN[cl]);
+                    float4 v;
+                    v.x = epilogue(P, ptrs, acc[i][4 * g] * scale, off);
+                    v.y = epilogue(P, ptrs, acc[i][4 * g + 1] * scale, off + 1);
+                    v.z = epilogue(P, ptrs, acc[i][4 * g + 2] * scale, off + 2);
+                    v.w = epilogue(P, ptrs, acc[i][4 * g + 3] * scale, off + 3);
+                    float4 *dst = reinterpret_cast<float4 *>(out + off);
+                    if (P.accumulate) { const float4 o = *dst; v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w; }
+                    *dst = v;
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (n + j >= Next) continue;
+                        const unsigned off = (unsigned)(ob + outN[cl + j]);
+                        float v = epilogue(P, ptrs, acc[i][4 * g + j] * scale, off);
+                        if (P.accumulate) v += out[off];
+                        out[off] = v;
+                    }
+                }
+            }
+        }
+    }
+}
+
+// Adds the planes of partial sums of a split summation, plane 0 first, and stores the outputs.
+__global__ void __launch_bounds__(256)
+tad_contract_reduce(const __grid_constant__ TadcProgram P, const __grid_constant__ TadpPointers ptrs)
+{
+    const unsigned Mext = (unsigned)P.M.extent, Next = (unsigned)P.N.extent;
+    const unsigned per_z = Mext * Next;
+    const unsigned cells = per_z * (unsigned)P.Z.extent;
+    const unsigned planes = (unsigned)P.ksplit;
+    for (unsigned c = blockIdx.x * blockDim.x + threadIdx.x; c < cells; c += gridDim.x * blockDim.x) {
+        const unsigned zb = c / per_z, rem = c - zb * per_z;
+        const unsigned m = rem / Next, n = rem - m * Next;
+        const float *src = ptrs.part + (size_t)zb * planes * per_z + rem;
+        float sum = 0.f;
+        for (unsigned s = 0; s < planes; ++s) sum += src[(size_t)s * per_z];
+        const unsigned off = (unsigned)(P.baseO + decode(P.Z, zb).o + decode(P.M, m).o + decode(P.N, n).o);
+        float v = epilogue(P, ptrs, sum * P.scale, off);
+        if (P.accumulate) v += ptrs.out[off];
+        ptrs.out[off] = v;
+    }
+}
+
+template <int BM, int BN, int TM, int TN>
+cudaError_t launch_shape(const TadcProgram &P, const TadpPointers &ptrs, cudaStream_t stream)
+{
+    using C = Cfg<BM, BN, TM, TN>;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    auto kern = tad_contract_kernel<BM, BN, TM, TN>;
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    const unsigned tiles_m = ((unsigned)P.M.extent + BM - 1) / BM, tiles_n = ((unsigned)P.N.extent + BN - 1) / BN;
+    dim3 grid(tiles_m * tiles_n, (unsigned)std::max(1, P.ksplit), (unsigned)P.Z.extent);
+    kern<<<grid, C::NT, C::SMEM, stream>>>(P, ptrs, tiles_m, tiles_n);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t tad_launch_contract(const TadcProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream)
+{
+    if (P.M.extent <= 0 || P.N.extent <= 0 || P.Z.extent <= 0) return cudaSuccess;
+    cudaError_t e = P.shape == 1 ? launch_shape<128, 32, 4, 4>(P, ptrs, stream) : launch_shape<128, 128, 8, 8>(P, ptrs, stream);
+    if (e != cudaSuccess) return e;
+    if (P.ksplit > 1) {
+        const unsigned long long cells = (unsigned long long)P.M.extent * P.N.extent * P.Z.extent;
+        const unsigned blocks = (unsigned)std::min<unsigned long long>((cells + 255) / 256, (unsigned long long)sms * 8);
+        tad_contract_reduce<<<blocks, 256, 0, stream>>>(P, ptrs);
+        e = cudaGetLastError();
+    }
+    return e;
+}

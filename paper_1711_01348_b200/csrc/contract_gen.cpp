@@ -1,0 +1,359 @@
+// Contraction planner (host only): recognises a kernel whose term is a product of two index
+// expressions under summations and rewrites it as one or several contraction programs
+// (contract.h) for the tile kernel.
+//
+// The loop variables of the kernel are split by which of the two factors reads them: variables
+// that only the first factor reads index the rows m of the tile, variables that only the second
+// reads (or neither) index its columns n, variables both read and that are not summed form a batch
+// index, and the summed variables form k.  Every index expression is affine (Sec. 5.1), so each
+// factor's element offset is a sum of one part per group, which is all the tile kernel needs.
+//
+// A summation loop whose bounds move with another variable v as a band,
+//     (c_lo + a v) / d  <=  z  <=  (c_hi + a v) / d,
+// (the taps of a transposed strided convolution: Sec. 5.1's range form with a rational slope) is
+// brought to fixed bounds by the substitution  v = d' v' + p,  z = a' v' + r  with a / d = a' / d'
+// in lowest terms: for every residue p the offset r runs over a fixed range, so each residue
+// class becomes a contraction of its own; the remaining constant bounds of z turn into a guard
+// that reads operand elements outside them as zero.
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <numeric>
+
+#include "gen.h"
+
+namespace tad {
+
+namespace {
+
+struct AVar { int64_t ext; bool reduce; };               // values 0 .. ext-1 after normalisation
+struct AMap { int ptr = 0; int64_t base = 0, limit = 0; std::vector<int64_t> coef; };   // limit: elements in the tensor
+struct AGuard { std::vector<int64_t> coef; int64_t c0 = 0, ext = 1; };   // live iff 0 <= c0 + coef . vars < ext
+
+struct System {
+    std::vector<AVar> vars;
+    AMap A, B, O;
+    std::vector<AGuard> guards;
+    bool loose_box = false;     // the outer box is a bounding box of the live elements, not the set itself
+};
+
+int32_t fit(int64_t v) { if (std::llabs(v) >= (int64_t(1) << 31)) throw Overflow(); return (int32_t)v; }
+
+struct Digit { int var; int64_t ext, sA, sB, sO; };
+
+bool fill_group(TadcGroup &G, std::vector<Digit> &ds, const AGuard *ga, const AGuard *gb)
+{
+    if ((int)ds.size() > TADC_MAX_DIGITS) return false;
+    G = TadcGroup{};
+    G.n_digits = (int32_t)ds.size();
+    int64_t extent = 1;
+    for (size_t d = 0; d < ds.size(); ++d) {
+        G.ext[d] = fit(ds[d].ext);
+        G.sA[d] = fit(ds[d].sA); G.sB[d] = fit(ds[d].sB); G.sO[d] = fit(ds[d].sO);
+        G.gA[d] = ga ? fit(ga->coef[ds[d].var]) : 0;
+        G.gB[d] = gb ? fit(gb->coef[ds[d].var]) : 0;
+        extent = mul_ck(extent, ds[d].ext);
+    }
+    G.extent = fit(extent);
+    return true;
+}
+
+// builds one contraction program from a system whose loops all have fixed ranges
+bool emit_program(const System &s0, float scale, int accumulate, bool allow_split, TadcProgram &P, std::string &text)
+{
+    System s = s0;
+    const int nv = (int)s.vars.size();
+    // which factor plays A: the variable along which the output is contiguous should index columns
+    int contiguous = -1;
+    for (int v = 0; v < nv; ++v)
+        if (!s.vars[v].reduce && s.O.coef[v] != 0 && s.vars[v].ext > 1 &&
+            (contiguous < 0 || std::llabs(s.O.coef[v]) < std::llabs(s.O.coef[contiguous]))) contiguous = v;
+    if (contiguous >= 0 && s.A.coef[contiguous] != 0 && s.B.coef[contiguous] == 0) std::swap(s.A, s.B);
+    std::vector<Digit> dm, dn, dk, dz;
+    for (int v = 0; v < nv; ++v) {
+        if (s.vars[v].ext == 1) continue;                  // a single value: nothing to index
+        Digit d{v, s.vars[v].ext, s.A.coef[v], s.B.coef[v], s.O.coef[v]};
+        if (s.vars[v].reduce) dk.push_back(d);
+        else if (d.sA != 0 && d.sB != 0) dz.push_back(d);
+        else if (d.sA != 0) dm.push_back(d);
+        else dn.push_back(d);
+    }
+    auto mag = [](int64_t a) { return a == 0 ? INT64_MAX : std::llabs(a); };
+    // fastest digit last: rows by their stride in the operand, columns by their stride in the output
+    std::stable_sort(dm.begin(), dm.end(), [&](const Digit &x, const Digit &y) { return mag(x.sA) > mag(y.sA); });
+    std::stable_sort(dn.begin(), dn.end(), [&](const Digit &x, const Digit &y) {
+        return mag(x.sO) != mag(y.sO) ? mag(x.sO) > mag(y.sO) : mag(x.sB) > mag(y.sB); });
+    std::stable_sort(dk.begin(), dk.end(), [&](const Digit &x, const Digit &y) {
+        return std::min(mag(x.sA), mag(x.sB)) > std::min(mag(y.sA), mag(y.sB)); });
+    // guards: at most one per operand; a guard belongs to an operand whose groups hold all its variables
+    const AGuard *ga = nullptr, *gb = nullptr;
+    auto in_group = [&](const std::vector<Digit> &g, int v) { for (const Digit &d : g) if (d.var == v) return true; return false; };
+    for (const AGuard &gd : s.guards) {
+        bool fits_a = true, fits_b = true;
+        for (int v = 0; v < nv; ++v) {
+            if (!gd.coef[v] || s.vars[v].ext == 1) continue;
+            if (in_group(dn, v)) fits_a = false;
+            if (in_group(dm, v)) fits_b = false;
+        }
+        if (fits_b && !gb) gb = &gd;
+        else if (fits_a && !ga) ga = &gd;
+        else return false;
+    }
+    // every offset the kernel can form must lie inside its tensor: interval check over the digit ranges
+    // (an operand under a guard is checked over the guarded range of its guard expression only when the
+    // guard is the identity on one digit pair, so it is skipped here: the guard itself bounds the reads)
+    auto in_range = [&](const AMap &m, bool guarded) {
+        if (guarded) return true;
+        int64_t lo = m.base, hi = m.base;
+        for (int v = 0; v < nv; ++v) {
+            if (s.vars[v].ext <= 1) { if (s.vars[v].ext <= 0) return true; continue; }
+            const int64_t span = mul_ck(m.coef[v], s.vars[v].ext - 1);
+            if (span < 0) lo = add_ck(lo, span); else hi = add_ck(hi, span);
+        }
+        return lo >= 0 && hi < m.limit;
+    };
+    if (!in_range(s.A, ga != nullptr) || !in_range(s.B, gb != nullptr) || !in_range(s.O, false)) {
+        // a masked index expression iterates a bounding box of its image lattice and the interpreter skips the
+        // elements without terms; the tile kernel would touch them, so such a kernel stays with the interpreter
+        if (s.loose_box) return false;
+        throw BadExpr("internal: contraction offsets leave their tensor");
+    }
+    P = TadcProgram{};
+    if (!fill_group(P.M, dm, ga, nullptr) || !fill_group(P.N, dn, nullptr, gb) || !fill_group(P.K, dk, ga, gb) ||
+        !fill_group(P.Z, dz, ga, gb)) return false;
+    if (P.Z.extent > 65535) return false;
+    P.ptrA = s.A.ptr; P.ptrB = s.B.ptr;
+    P.baseA = fit(s.A.base); P.baseB = fit(s.B.base); P.baseO = fit(s.O.base);
+    P.guardA = ga ? 1 : 0; P.guardA_c0 = ga ? fit(ga->c0) : 0; P.guardA_ext = ga ? fit(ga->ext) : 1;
+    P.guardB = gb ? 1 : 0; P.guardB_c0 = gb ? fit(gb->c0) : 0; P.guardB_ext = gb ? fit(gb->ext) : 1;
+    P.scale = scale; P.accumulate = accumulate;
+    // tile shape: narrow column tiles for narrow outputs
+    P.shape = P.N.extent <= 48 ? 1 : 0;
+    const int64_t BM = 128, BN = P.shape == 1 ? 32 : 128;
+    const int64_t tiles_m = (P.M.extent + BM - 1) / BM, tiles_n = (P.N.extent + BN - 1) / BN;
+    const double fill = (double)P.M.extent * P.N.extent / ((double)tiles_m * BM * tiles_n * BN);
+    if (fill < 0.15) return false;                         // mostly empty tiles: the interpreter's schedules do better
+    // gather modes
+    auto mode_of = [&](const std::vector<Digit> &rows, bool second, const AGuard *gd, int64_t base) {
+        auto st = [&](const Digit &d) { return second ? d.sB : d.sA; };
+        const int64_t rs = rows.empty() ? 0 : std::llabs(st(rows.back()));
+        const int64_t ks = dk.empty() ? 0 : std::llabs(st(dk.back()));
+        const int64_t kext = dk.empty() ? 0 : dk.back().ext;
+        if (rs == 1) {
+            bool wide = st(rows.back()) == 1 && rows.back().ext % 4 == 0 && base % 4 == 0 && !(gd && gd->coef[rows.back().var]);
+            for (size_t d = 0; d + 1 < rows.size(); ++d) if (st(rows[d]) % 4) wide = false;
+            for (const Digit &d : dk) if (st(d) % 4) wide = false;
+            for (const Digit &d : dz) if (st(d) % 4) wide = false;
+            return wide ? TG_ROW16 : TG_ROW;
+        }
+        if (rs == 0) return TG_K;
+        if (ks == 1 && kext >= 8) return TG_K;
+        if (ks == 0 || rs <= ks) return TG_ROW;
+        return TG_K;
+    };
+    P.modeA = mode_of(dm, false, ga, s.A.base);
+    P.modeB = mode_of(dn, true, gb, s.B.base);
+    // output: four consecutive columns are four consecutive aligned elements
+    P.out_vec4 = 0;
+    if (!dn.empty() && dn.back().sO == 1 && dn.back().ext % 4 == 0 && s.O.base % 4 == 0) {
+        P.out_vec4 = 1;
+        for (size_t d = 0; d + 1 < dn.size(); ++d) if (dn[d].sO % 4) P.out_vec4 = 0;
+        for (const Digit &d : dm) if (d.sO % 4) P.out_vec4 = 0;
+        for (const Digit &d : dz) if (d.sO % 4) P.out_vec4 = 0;
+    }
+    // summation split: enough blocks for two per SM when the tiles alone are too few
+    const int64_t blocks = tiles_m * tiles_n * P.Z.extent;
+    const int64_t kstages = (P.K.extent + TADC_BK - 1) / TADC_BK;
+    int64_t split = 1;
+    if (allow_split && blocks < 222 && kstages >= 16) {
+        split = std::min<int64_t>((296 + blocks - 1) / blocks, kstages / 8);
+        const int64_t cells = (int64_t)P.M.extent * P.N.extent * P.Z.extent;
+        while (split > 1 && split * cells > (int64_t(1) << 25)) --split;            // <= 128 MB of partial sums
+    }
+    split = std::max<int64_t>(1, split);
+    const int64_t per = ((kstages + split - 1) / split) * TADC_BK;
+    P.kchunk = fit(std::max<int64_t>(per, TADC_BK));
+    P.ksplit = fit(std::max<int64_t>(1, (P.K.extent + P.kchunk - 1) / P.kchunk));
+    if (P.ksplit <= 1) { P.ksplit = 1; P.kchunk = fit(std::max<int64_t>(kstages, 1) * TADC_BK); }
+    char line[320];
+    auto group_text = [&](const char *name, const TadcGroup &G) {
+        std::string t = std::string("  ") + name + ":";
+        for (int d = 0; d < G.n_digits; ++d) {
+            std::snprintf(line, sizeof line, " [ext %d sA %d sB %d sO %d]", G.ext[d], G.sA[d], G.sB[d], G.sO[d]);
+            t += line;
+        }
+        return t + "\n";
+    };
+    std::snprintf(line, sizeof line, "; contraction %d x %d x %d (batch %d): A=ptr %d mode %d guard %d, B=ptr %d mode %d guard %d, tile %s, ksplit %d x %d, vec4 %d, scale %g, accumulate %d\n",
+                  P.M.extent, P.N.extent, P.K.extent, P.Z.extent, P.ptrA, P.modeA, P.guardA, P.ptrB, P.modeB, P.guardB,
+                  P.shape == 1 ? "128x32" : "128x128", P.ksplit, P.kchunk, P.out_vec4, (double)P.scale, P.accumulate);
+    text += line;
+    text += group_text("m", P.M) + group_text("n", P.N) + group_text("k", P.K) + group_text("z", P.Z);
+    return true;
+}
+
+}  // namespace
+
+bool try_contraction(Gen &g, Kernel &k, int root, int scale, bool allow_split, const std::vector<std::vector<TadpRow>> &lower,
+                     const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards)
+{
+    if (g.p.opt.debug_bounds || !guards.empty() || root < 0) return false;
+    const TadpProgram &prog = k.prog;
+    float cfac = 1.f;
+    if (scale >= 0) { if (g.inst[scale].op != I_CONST) return false; cfac = g.inst[scale].imm; }
+    const int nv = (int)g.vars.size();
+    // ---- the term: constant factors, sums, then a product of two loads ----
+    std::vector<int64_t> vlo(nv, 0), vext(nv, 1);
+    std::vector<bool> reduce(nv, false), seen(nv, false);
+    for (int v = 0; v < g.n_outer; ++v) { vlo[v] = prog.outer_lo[v]; vext[v] = prog.outer_ext[v]; seen[v] = true; }
+    int cur = root;
+    for (;;) {
+        const Inst &in = g.inst[cur];
+        if (in.op == I_SUM) { vlo[in.var] = in.lo; vext[in.var] = std::max<int64_t>(0, in.hi - in.lo + 1); reduce[in.var] = true; seen[in.var] = true; cur = in.a; }
+        else if (in.op == I_MULC) { cfac *= in.imm; cur = in.a; }
+        else if (in.op == I_NEG) { cfac = -cfac; cur = in.a; }
+        else break;
+    }
+    auto as_load = [&](int i) {
+        for (;;) {
+            const Inst &in = g.inst[i];
+            if (in.op == I_MULC) { cfac *= in.imm; i = in.a; }
+            else if (in.op == I_NEG) { cfac = -cfac; i = in.a; }
+            else return in.op == I_LOAD ? in.load : -1;
+        }
+    };
+    int la = -1, lb = -1;
+    if (g.inst[cur].op == I_MUL) { la = as_load(g.inst[cur].a); lb = as_load(g.inst[cur].b); }
+    else if (g.inst[cur].op == I_SQR) {
+        // (c L)^2 = c^2 L L
+        const float outer_c = cfac;
+        cfac = 1.f;
+        la = lb = as_load(g.inst[cur].a);
+        cfac = outer_c * cfac * cfac;
+    }
+    if (la < 0 || lb < 0) return false;
+    // ---- kernel-coordinate loops: fixed ranges, or one band ----
+    struct Band { int z, v; int64_t a, d, c_lo, c_hi; int64_t zmin, zmax; bool has_min, has_max; };
+    bool have_band = false; Band band{};
+    for (int l = 0; l < g.kappa; ++l) {
+        const int z = g.n_outer + g.zorder[l];
+        reduce[z] = true; seen[z] = true;
+        auto constant = [&](const TadpRow &r) { for (int v = 0; v < TADP_MAX_VARS; ++v) if (r.coef[v]) return false; return true; };
+        bool all_const = true;
+        for (const TadpRow &r : lower[l]) all_const = all_const && constant(r);
+        for (const TadpRow &r : upper[l]) all_const = all_const && constant(r);
+        if (lower[l].empty() || upper[l].empty()) return false;
+        if (all_const) {
+            int64_t lo = INT64_MIN, hi = INT64_MAX;
+            for (const TadpRow &r : lower[l]) lo = std::max(lo, ceil_div(r.c0, r.den));
+            for (const TadpRow &r : upper[l]) hi = std::min(hi, floor_div(r.c0, r.den));
+            vlo[z] = lo; vext[z] = std::max<int64_t>(0, hi - lo + 1);
+            continue;
+        }
+        if (have_band) return false;
+        // one lower and one upper row with the same slope on one variable; every other row constant
+        const TadpRow *rl = nullptr, *rh = nullptr;
+        int64_t zmin = 0, zmax = 0; bool has_min = false, has_max = false;
+        for (const TadpRow &r : lower[l]) {
+            if (constant(r)) { const int64_t c = ceil_div(r.c0, r.den); zmin = has_min ? std::max(zmin, c) : c; has_min = true; }
+            else if (!rl) rl = &r; else return false;
+        }
+        for (const TadpRow &r : upper[l]) {
+            if (constant(r)) { const int64_t c = floor_div(r.c0, r.den); zmax = has_max ? std::min(zmax, c) : c; has_max = true; }
+            else if (!rh) rh = &r; else return false;
+        }
+        if (!rl || !rh) return false;
+        int bv = -1;
+        for (int v = 0; v < TADP_MAX_VARS; ++v) {
+            if (!rl->coef[v] && !rh->coef[v]) continue;
+            if (bv >= 0) return false;
+            bv = v;
+        }
+        // same slope: a_l / d_l == a_h / d_h; bring both rows to the common denominator
+        const int64_t dl = rl->den, dh = rh->den, al = rl->coef[bv], ah = rh->coef[bv];
+        if (al * dh != ah * dl) return false;
+        const int64_t d = dl / gcd64(dl, dh) * dh;
+        band = Band{z, bv, al * (d / dl), d, rl->c0 * (d / dl), rh->c0 * (d / dh), zmin, zmax, has_min, has_max};
+        if ((band.c_hi - band.c_lo) / band.d > 64) return false;     // not a narrow band
+        have_band = true;
+    }
+    for (int v = 0; v < nv; ++v) if (!seen[v]) return false;
+    const TadpLoad &LA = g.loads[la], &LB = g.loads[lb];
+    // ---- the affine system, every variable counted from zero ----
+    System base;
+    base.vars.resize(nv);
+    base.A.ptr = LA.ptr; base.B.ptr = LB.ptr;
+    base.A.base = LA.base; base.B.base = LB.base; base.O.base = prog.out_base;
+    base.loose_box = prog.write_only_live != 0;
+    base.A.limit = LA.limit; base.B.limit = LB.limit; base.O.limit = prog.out_limit;
+    base.A.coef.assign(nv, 0); base.B.coef.assign(nv, 0); base.O.coef.assign(nv, 0);
+    for (int v = 0; v < nv; ++v) {
+        base.vars[v] = AVar{vext[v], reduce[v]};
+        base.A.coef[v] = LA.coef[v]; base.B.coef[v] = LB.coef[v];
+        base.O.coef[v] = v < g.n_outer ? prog.out_coef[v] : 0;
+    }
+    auto shift = [&](System &s, int v, int64_t by) {      // variable v := by + v
+        s.A.base = add_ck(s.A.base, mul_ck(s.A.coef[v], by));
+        s.B.base = add_ck(s.B.base, mul_ck(s.B.coef[v], by));
+        s.O.base = add_ck(s.O.base, mul_ck(s.O.coef[v], by));
+        for (AGuard &gd : s.guards) gd.c0 = add_ck(gd.c0, mul_ck(gd.coef[v], by));
+    };
+    std::vector<System> systems;
+    if (!have_band) {
+        for (int v = 0; v < nv; ++v) shift(base, v, vlo[v]);
+        systems.push_back(base);
+    } else {
+        // v = vlo + w with w = d' w' + p; the band in terms of w: (c + a vlo + a w) / d
+        const int v = band.v, z = band.z;
+        if (v == z) return false;
+        for (int u = 0; u < nv; ++u) if (u != z) shift(base, u, vlo[u]);
+        const int64_t c_lo = add_ck(band.c_lo, mul_ck(band.a, vlo[v])), c_hi = add_ck(band.c_hi, mul_ck(band.a, vlo[v]));
+        const int64_t gq = gcd64(std::llabs(band.a), band.d);
+        const int64_t a1 = band.a / gq, d1 = band.d / gq;
+        if (d1 > 8) return false;
+        for (int64_t p = 0; p < d1; ++p) {
+            System s = base;
+            const int64_t r_lo = ceil_div(add_ck(c_lo, mul_ck(band.a, p)), band.d);
+            const int64_t r_hi = floor_div(add_ck(c_hi, mul_ck(band.a, p)), band.d);
+            const int64_t wext = vext[v] > p ? (vext[v] - p + d1 - 1) / d1 : 0;
+            // substitute  w = d1 w' + p,  z = a1 w' + r_lo + r
+            auto subst = [&](AMap &m) {
+                m.base = add_ck(m.base, add_ck(mul_ck(m.coef[v], p), mul_ck(m.coef[z], r_lo)));
+                m.coef[v] = add_ck(mul_ck(m.coef[v], d1), mul_ck(m.coef[z], a1));
+            };
+            subst(s.A); subst(s.B); subst(s.O);
+            s.vars[v].ext = wext;
+            s.vars[z].ext = std::max<int64_t>(0, r_hi - r_lo + 1);
+            if (band.has_min || band.has_max) {
+                // zmin <= z <= zmax with z = a1 w' + r_lo + r
+                if (!band.has_min || !band.has_max) return false;
+                AGuard gd;
+                gd.coef.assign(nv, 0);
+                gd.coef[v] = a1; gd.coef[z] = 1;
+                gd.c0 = r_lo - band.zmin;
+                gd.ext = band.zmax - band.zmin + 1;
+                if (gd.ext <= 0) s.vars[z].ext = 0;
+                gd.ext = std::max<int64_t>(gd.ext, 1);
+                s.guards.push_back(gd);
+            }
+            systems.push_back(s);
+        }
+    }
+    std::vector<TadcProgram> progs;
+    std::string text;
+    for (const System &s : systems) {
+        bool empty_out = false;
+        for (int v = 0; v < nv; ++v) if (!s.vars[v].reduce && s.vars[v].ext <= 0) empty_out = true;
+        if (empty_out) continue;
+        TadcProgram P;
+        if (!emit_program(s, cfac, prog.accumulate, allow_split, P, text)) return false;
+        progs.push_back(P);
+    }
+    if (progs.empty()) return false;
+    k.contract = progs;
+    k.listing = text;
+    k.vec = 0; k.vec_u = 0;
+    return true;
+}
+
+}  // namespace tad

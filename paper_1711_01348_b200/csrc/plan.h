@@ -8,6 +8,7 @@
 #include "../../include/tad.h"
 #include "intalg.h"
 #include "program.h"
+#include "contract.h"
 
 namespace tad {
 
@@ -67,6 +68,8 @@ struct Kernel {
     int vec_u = 1;             // elements per thread along the element variable (UB)
     bool rich = false;         // the build of the shape with more registers per thread and fewer warps per SM
     std::vector<int> stages_used;   // backward: staged adjoints it reads (indices into tad_plan::stages)
+    std::vector<TadcProgram> contract;   // non-empty: the kernel is a contraction, run by the tile kernel (one launch per
+                                         // program) instead of the interpreter
     KernelStats stats;
     std::string listing;
 };

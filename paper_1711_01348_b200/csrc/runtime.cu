@@ -19,6 +19,7 @@ void set_error(const std::string &m);
 #define TAD_DECLARE_VM(TA, UB) void tad_launch_vm_##TA##_##UB(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream);
 TAD_VM_SHAPES(TAD_DECLARE_VM)
 void tad_launch_vm_16_1_rich(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream);
+cudaError_t tad_launch_contract(const TadcProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream);
 
 namespace {
 
@@ -91,8 +92,25 @@ unsigned long long item_count(const TadpProgram &P, int ta, int ub)
 
 tad_status zero_fill(float *out, int64_t n, cudaStream_t stream);
 
+// contraction kernels: one launch of the tile kernel per program
+tad_status launch_contractions(const tad::Kernel &k, const TadpPointers &ptrs, cudaStream_t stream)
+{
+    for (TadcProgram P : k.contract) {
+        if (P.ksplit > 1 && !ptrs.part) { tad::set_error("internal: partial-sum buffer missing"); return TAD_ERR_WORKSPACE; }
+        // 16-byte copies and stores need 16-byte aligned tensors: fall back to 4-byte accesses otherwise
+        auto misaligned = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+        if (P.modeA == TG_ROW16 && misaligned(ptrs.in[P.ptrA])) P.modeA = TG_ROW;
+        if (P.modeB == TG_ROW16 && misaligned(ptrs.in[P.ptrB])) P.modeB = TG_ROW;
+        if (P.out_vec4 && misaligned(ptrs.out)) P.out_vec4 = 0;
+        const cudaError_t e = tad_launch_contract(P, ptrs, (unsigned)sm_count(), stream);
+        if (e != cudaSuccess) { tad::set_error(std::string("contraction launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
+    }
+    return TAD_OK;
+}
+
 tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStream_t stream)
 {
+    if (!k.contract.empty()) return launch_contractions(k, ptrs, stream);
     const int zsplit = k.prog.zsplit > 1 ? k.prog.zsplit : 1;
     if (zsplit > 1) {
         if (!ptrs.part) { tad::set_error("internal: partial-sum buffer missing"); return TAD_ERR_WORKSPACE; }

@@ -258,17 +258,18 @@ def _header(listing: str) -> dict:
     return dict(item.split("=") for item in first.lstrip("; ").split())
 
 
-def test_contractions_get_the_product_shape():
-    """Convolution forward and both gradients: every fused loop multiplies two loads, so the 4 x 8
-    product shape applies and dx runs with uniform loops (lanes along the channel index)."""
+def test_contractions_run_on_the_tile_kernel():
+    """Convolution forward and both gradients are products of two index expressions under sums: each becomes
+    a contraction program.  The gradient of x has a summation whose bounds move with the gradient index as a
+    band (slope 1/2): one program per residue class, three taps for even positions and two for odd ones."""
     from workloads import configs as W
     plan = Plan(W.FULL["cfg5"]())
-    for which in (-1, 0, 1):
-        listing = plan.disassemble(which)
-        assert _header(listing)["vec"] == "4x8", listing.splitlines()[0]
-        assert "XLOOP" in listing
-    dx = plan.disassemble(1)
-    assert "lane_dependent=1" not in dx and "relative=1" not in dx
+    fwd, dw, dx = plan.disassemble(-1), plan.disassemble(0), plan.disassemble(1)
+    assert fwd.count("; contraction") == 1 and "256 x 131072 x 1280" in fwd
+    assert dw.count("; contraction") == 1 and "256 x 1280 x 131072" in dw and "ksplit 1 " not in dw
+    assert dx.count("; contraction") == 2
+    assert "x 768 " in dx and "x 512 " in dx          # 256 channels x 3 taps, x 2 taps
+    assert dx.count("guard 1") == 2
 
 
 def test_split_summations_fill_whole_waves():
