@@ -192,10 +192,8 @@ def run_ours(opts):
     expr, args, df = W.workload(opts.config, full=True)
     if opts.rows:
         # profiler captures only: the same workload with fewer rows of the first output index
-        if opts.config != "cfg2":
-            raise SystemExit("--rows is implemented for cfg2 only")
-        expr = W.intro(opts.rows, 8192, 32, name=f"cfg2_intro_scaled_rows{opts.rows}")
-        args, df = W.make_inputs(expr, W.DIST["cfg2"], seed=0)
+        expr = W.profile_case(opts.config, opts.rows)
+        args, df = W.make_inputs(expr, W.DIST[opts.config], seed=0)
     plan = Plan(expr, saved_forward=opts.saved_forward)
     d_args = [a.to(dev) for a in args]
     d_df = df.to(dev)
@@ -356,7 +354,7 @@ def main():
     ap.add_argument("--saved-forward", action="store_true",
                     help="compile the plan with saved_forward: the backward kernels read f of the same step")
     ap.add_argument("--rows", type=int, default=0,
-                    help="profiler captures only: shrink the first output extent of cfg2 (not a bench number)")
+                    help="profiler captures only: the workload with a smaller leading extent (not a bench number)")
     opts = ap.parse_args()
     if opts.impl == "reference":
         run_reference(opts)

@@ -16,20 +16,21 @@
 namespace {
 
 constexpr int BK = TADC_BK;
-constexpr int STAGES = 3;
+constexpr int KK_UNROLL = 8;           // summation indices per unrolled body of the multiply-add loop
+constexpr int STAGES = 2;
 constexpr int DEAD = INT_MIN / 2;      // guard part of a row or summation index that does not exist
 
 __device__ __forceinline__ void cp_async4(float *dst, const float *src, bool live)
 {
     const unsigned d = (unsigned)__cvta_generic_to_shared(dst);
     const int bytes = live ? 4 : 0;
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;\n" ::"r"(d), "l"(src), "r"(bytes) : "memory");
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;\n" ::"r"(d), "l"(src), "r"(bytes));
 }
 __device__ __forceinline__ void cp_async16(float *dst, const float *src, bool live)
 {
     const unsigned d = (unsigned)__cvta_generic_to_shared(dst);
     const int bytes = live ? 16 : 0;
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(d), "l"(src), "r"(bytes) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(d), "l"(src), "r"(bytes));
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
@@ -54,51 +55,60 @@ __device__ __forceinline__ Parts decode(const TadcGroup &G, unsigned idx)
     return p;
 }
 
-// one stage of one operand: BK x BR values into smem[kl * (BR + 4) + rl]
-template <int BR, int NT>
-__device__ __forceinline__ void gather(float *smem, const float *__restrict__ src, const int2 *rows, const int4 *ktab,
-                                       const bool second, const int mode, const unsigned gext, const int tid)
+// One stage of one operand: BK x BR values into smem[kl * (BR + 4) + rl].  rows[rl] = (offset part, guard
+// part) of tile row rl, ktab[kl] the same for the stage's summation index kl.  CHECK = false is the path
+// of a stage whose every element exists and is read (no guard on the operand, tile and stage inside
+// the ranges): offset add, copy.  pre = rows[row of this thread] for the modes whose threads keep one row.
+template <int BR, int NT, bool CHECK>
+__device__ __forceinline__ void gather(float *smem, const float *__restrict__ src, const int2 *rows, const int2 *ktab,
+                                       const int2 pre, const int mode, const unsigned gext, const unsigned tid)
 {
+    // The copies carry no memory clobber (the group commit and wait do), and every table entry of a stage is
+    // read before the first copy is issued, so that the table reads overlap instead of each waiting its turn.
     constexpr int LD = BR + 4;
     if (mode == TG_ROW16) {
-        constexpr int CH = BR / 4, TOTAL = CH * BK, PER = (TOTAL + NT - 1) / NT;
+        constexpr unsigned CH = BR / 4, TOTAL = CH * BK, PER = (TOTAL + NT - 1) / NT, KSTEP = NT / CH;
+        static_assert(NT % CH == 0, "threads per stage row");
+        const unsigned rl = (tid % CH) * 4, kl0 = tid / CH;
+        if (TOTAL % NT != 0 && kl0 >= BK) return;
+        unsigned off[PER]; bool live[PER];
 #pragma unroll
-        for (int j = 0; j < PER; ++j) {
-            const int c = tid + NT * j;
-            if (TOTAL % NT == 0 || c < TOTAL) {
-                const int rl = (c % CH) * 4, kl = c / CH;
-                const int2 r = rows[rl];
-                const int4 kt = ktab[kl];
-                const bool live = (unsigned)(r.y + (second ? kt.w : kt.z)) < gext;
-                cp_async16(smem + kl * LD + rl, src + (live ? (unsigned)(r.x + (second ? kt.y : kt.x)) : 0u), live);
-            }
+        for (unsigned j = 0; j < PER; ++j) {
+            const int2 kt = ktab[kl0 + KSTEP * j];
+            live[j] = !CHECK || (unsigned)(pre.y + kt.y) < gext;
+            off[j] = live[j] ? (unsigned)(pre.x + kt.x) : 0u;
         }
+#pragma unroll
+        for (unsigned j = 0; j < PER; ++j) cp_async16(smem + (kl0 + KSTEP * j) * LD + rl, src + off[j], live[j]);
     } else if (mode == TG_ROW) {
-        constexpr int TOTAL = BR * BK, PER = (TOTAL + NT - 1) / NT;
+        constexpr unsigned TOTAL = BR * BK, PER = TOTAL / NT, KSTEP = NT / BR;
+        static_assert(NT % BR == 0 && TOTAL % NT == 0, "threads per stage row");
+        const unsigned rl = tid % BR, kl0 = tid / BR;
+        unsigned off[PER]; bool live[PER];
 #pragma unroll
-        for (int j = 0; j < PER; ++j) {
-            const int e = tid + NT * j;
-            if (TOTAL % NT == 0 || e < TOTAL) {
-                const int rl = e % BR, kl = e / BR;
-                const int2 r = rows[rl];
-                const int4 kt = ktab[kl];
-                const bool live = (unsigned)(r.y + (second ? kt.w : kt.z)) < gext;
-                cp_async4(smem + kl * LD + rl, src + (live ? (unsigned)(r.x + (second ? kt.y : kt.x)) : 0u), live);
-            }
+        for (unsigned j = 0; j < PER; ++j) {
+            const int2 kt = ktab[kl0 + KSTEP * j];
+            live[j] = !CHECK || (unsigned)(pre.y + kt.y) < gext;
+            off[j] = live[j] ? (unsigned)(pre.x + kt.x) : 0u;
         }
+#pragma unroll
+        for (unsigned j = 0; j < PER; ++j) cp_async4(smem + (kl0 + KSTEP * j) * LD + rl, src + off[j], live[j]);
     } else {
-        constexpr int TOTAL = BR * BK, PER = (TOTAL + NT - 1) / NT;
+        // a warp copies 8 summation indices x 4 rows: full 32-byte sectors of a row-major operand, and the
+        // 32 shared-memory words it writes (row stride BR + 4) fall into 32 different banks
+        constexpr unsigned TOTAL = BR * BK, PER = TOTAL / NT, RSTEP = NT / BK;
+        static_assert(BK % 8 == 0 && NT % (4 * BK) == 0 && TOTAL % NT == 0, "copy pattern of the summation-index mode");
+        const unsigned kl = (tid % 8) + 8 * ((tid / 32) % (BK / 8)), rl0 = (tid / 8) % 4 + 4 * (tid / (4 * BK));
+        const int2 kt = ktab[kl];
+        unsigned off[PER]; bool live[PER];
 #pragma unroll
-        for (int j = 0; j < PER; ++j) {
-            const int e = tid + NT * j;
-            if (TOTAL % NT == 0 || e < TOTAL) {
-                const int kl = e % BK, rl = e / BK;
-                const int2 r = rows[rl];
-                const int4 kt = ktab[kl];
-                const bool live = (unsigned)(r.y + (second ? kt.w : kt.z)) < gext;
-                cp_async4(smem + kl * LD + rl, src + (live ? (unsigned)(r.x + (second ? kt.y : kt.x)) : 0u), live);
-            }
+        for (unsigned j = 0; j < PER; ++j) {
+            const int2 r = rows[rl0 + RSTEP * j];
+            live[j] = !CHECK || (unsigned)(r.y + kt.y) < gext;
+            off[j] = live[j] ? (unsigned)(r.x + kt.x) : 0u;
         }
+#pragma unroll
+        for (unsigned j = 0; j < PER; ++j) cp_async4(smem + kl * LD + rl0 + RSTEP * j, src + off[j], live[j]);
     }
 }
 
@@ -137,7 +147,7 @@ struct Cfg {
     static constexpr int LDA = BM + 4, LDB = BN + 4;
     static constexpr int STAGE_FLOATS = BK * (LDA + LDB);
     static constexpr size_t SMEM = size_t(STAGES) * STAGE_FLOATS * 4 + size_t(BM + BN) * 8 + size_t(BM + BN) * 4 +
-                                   size_t(STAGES + 1) * BK * 16;
+                                   size_t(STAGES + 1) * BK * 16;      // stages, row tables, output offsets, two k tables
 };
 
 template <int BM, int BN, int TM, int TN>
@@ -149,13 +159,14 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
     constexpr int GM = TM / 4, GN = TN / 4;           // groups of four rows / columns per thread
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *stage_mem = reinterpret_cast<float *>(smem_raw);
-    int4 *ktab = reinterpret_cast<int4 *>(stage_mem + STAGES * C::STAGE_FLOATS);
-    int2 *rowA = reinterpret_cast<int2 *>(ktab + (STAGES + 1) * BK);
+    int2 *ktabA = reinterpret_cast<int2 *>(stage_mem + STAGES * C::STAGE_FLOATS);
+    int2 *ktabB = ktabA + (STAGES + 1) * BK;
+    int2 *rowA = ktabB + (STAGES + 1) * BK;
     int2 *rowB = rowA + BM;
     int *outM = reinterpret_cast<int *>(rowB + BN);
     int *outN = outM + BM;
 
-    const int tid = threadIdx.x;
+    const unsigned tid = threadIdx.x;
     const unsigned tile = blockIdx.x;
     const unsigned tile_m = tile % tiles_m, tile_n = tile / tiles_m;
     const unsigned ks = blockIdx.y, zb = blockIdx.z;
@@ -172,12 +183,12 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
     const int n_stages = (int)((kend - kbeg + BK - 1) / BK);
 
     // per-row parts of the operand offsets, guards and output offsets of this tile
-    for (int r = tid; r < BM; r += NT) {
+    for (unsigned r = tid; r < BM; r += NT) {
         const unsigned m = tile_m * BM + r;
         if (m < Mext) { const Parts p = decode(P.M, m); rowA[r] = make_int2(constA + p.a, P.guardA_c0 + z.ga + p.ga); outM[r] = p.o; }
         else { rowA[r] = make_int2(0, DEAD); outM[r] = 0; }
     }
-    for (int r = tid; r < BN; r += NT) {
+    for (unsigned r = tid; r < BN; r += NT) {
         const unsigned n = tile_n * BN + r;
         if (n < Next) { const Parts p = decode(P.N, n); rowB[r] = make_int2(constB + p.b, P.guardB_c0 + z.gb + p.gb); outN[r] = p.o; }
         else { rowB[r] = make_int2(0, DEAD); outN[r] = 0; }
@@ -185,28 +196,41 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
     auto fill_ktab = [&](int kstage) {
         if (tid < BK) {
             const unsigned k = kbeg + (unsigned)kstage * BK + tid;
-            int4 e = make_int4(0, 0, DEAD, DEAD);
-            if (k < kend) { const Parts p = decode(P.K, k); e = make_int4(p.a, p.b, p.ga, p.gb); }
-            ktab[(kstage % (STAGES + 1)) * BK + tid] = e;
+            int2 ea = make_int2(0, DEAD), eb = make_int2(0, DEAD);
+            if (k < kend) { const Parts p = decode(P.K, k); ea = make_int2(p.a, p.ga); eb = make_int2(p.b, p.gb); }
+            ktabA[(kstage % (STAGES + 1)) * BK + tid] = ea;
+            ktabB[(kstage % (STAGES + 1)) * BK + tid] = eb;
         }
     };
     for (int s = 0; s < STAGES; ++s) fill_ktab(s);
     __syncthreads();
     const unsigned gextA = (unsigned)P.guardA_ext, gextB = (unsigned)P.guardB_ext;
     const int modeA = P.modeA, modeB = P.modeB;
+    // the row a thread keeps through all stages (modes with the lanes along the row index)
+    const int2 preA = rowA[modeA == TG_ROW16 ? (tid % (BM / 4)) * 4 : tid % BM];
+    const int2 preB = rowB[modeB == TG_ROW16 ? (tid % (BN / 4)) * 4 : tid % BN];
+    // tiles inside the ranges and operands without a guard take the copy path without tests
+    const bool plainA = !P.guardA && (tile_m + 1) * BM <= Mext, plainB = !P.guardB && (tile_n + 1) * BN <= Next;
     auto issue = [&](int kstage) {
         if (kstage < n_stages) {
             float *as = stage_mem + (kstage % STAGES) * C::STAGE_FLOATS;
             float *bs = as + BK * LDA;
-            const int4 *kt = ktab + (kstage % (STAGES + 1)) * BK;
-            gather<BM, NT>(as, A, rowA, kt, false, modeA, gextA, tid);
-            gather<BN, NT>(bs, B, rowB, kt, true, modeB, gextB, tid);
+            const int slot = (kstage % (STAGES + 1)) * BK;
+            const bool full = kbeg + (unsigned)(kstage + 1) * BK <= kend;
+            if (plainA && full) gather<BM, NT, false>(as, A, rowA, ktabA + slot, preA, modeA, gextA, tid);
+            else gather<BM, NT, true>(as, A, rowA, ktabA + slot, preA, modeA, gextA, tid);
+            if (plainB && full) gather<BN, NT, false>(bs, B, rowB, ktabB + slot, preB, modeB, gextB, tid);
+            else gather<BN, NT, true>(bs, B, rowB, ktabB + slot, preB, modeB, gextB, tid);
         }
         cp_async_commit();
     };
     for (int s = 0; s < STAGES - 1; ++s) issue(s);
 
-    const int tx = tid % (BN / TN), ty = tid / (BN / TN);
+    // a warp covers 8 thread columns x 4 thread rows: its 128-bit reads of a stage touch 128 consecutive bytes
+    // of the B tile and 64 of the A tile, one shared-memory wavefront each
+    constexpr unsigned WARPS_N = (BN / TN) / 8;
+    const unsigned warp = tid / 32, lane = tid % 32;
+    const int tx = (int)((warp % WARPS_N) * 8 + lane % 8), ty = (int)((warp / WARPS_N) * 4 + lane / 8);
     float acc[TM][TN];
 #pragma unroll
     for (int i = 0; i < TM; ++i)
@@ -220,23 +244,28 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
         issue(it + STAGES - 1);
         const float *as = stage_mem + (it % STAGES) * C::STAGE_FLOATS;
         const float *bs = as + BK * LDA;
-#pragma unroll
-        for (int kk = 0; kk < BK; ++kk) {
-            float a[TM], b[TN];
+        // operands of summation index kk + 1 are fetched from shared memory while those of kk are multiplied
+        float a[2][TM], b[2][TN];
+        auto fetch = [&](int kk, float *av, float *bv) {
 #pragma unroll
             for (int g = 0; g < GM; ++g) {
                 const float4 v = *reinterpret_cast<const float4 *>(as + kk * LDA + g * (BM / GM) + ty * 4);
-                a[4 * g] = v.x; a[4 * g + 1] = v.y; a[4 * g + 2] = v.z; a[4 * g + 3] = v.w;
+                av[4 * g] = v.x; av[4 * g + 1] = v.y; av[4 * g + 2] = v.z; av[4 * g + 3] = v.w;
             }
 #pragma unroll
             for (int g = 0; g < GN; ++g) {
                 const float4 v = *reinterpret_cast<const float4 *>(bs + kk * LDB + g * (BN / GN) + tx * 4);
-                b[4 * g] = v.x; b[4 * g + 1] = v.y; b[4 * g + 2] = v.z; b[4 * g + 3] = v.w;
+                bv[4 * g] = v.x; bv[4 * g + 1] = v.y; bv[4 * g + 2] = v.z; bv[4 * g + 3] = v.w;
             }
+        };
+        fetch(0, a[0], b[0]);
+#pragma unroll KK_UNROLL
+        for (int kk = 0; kk < BK; ++kk) {
+            if (kk + 1 < BK) fetch(kk + 1, a[(kk + 1) & 1], b[(kk + 1) & 1]);
 #pragma unroll
             for (int i = 0; i < TM; ++i)
 #pragma unroll
-                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[kk & 1][i], b[kk & 1][j], acc[i][j]);
         }
     }
     cp_async_wait<0>();

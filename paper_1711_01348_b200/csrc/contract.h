@@ -13,7 +13,7 @@
 #include <stdint.h>
 
 #define TADC_MAX_DIGITS 4
-#define TADC_BK 16            // summation indices per shared-memory stage
+#define TADC_BK 32            // summation indices per shared-memory stage
 
 struct TadcGroup {             // flattened index group, last digit fastest
     int32_t n_digits;

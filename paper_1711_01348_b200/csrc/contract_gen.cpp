@@ -133,23 +133,39 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     const int64_t tiles_m = (P.M.extent + BM - 1) / BM, tiles_n = (P.N.extent + BN - 1) / BN;
     const double fill = (double)P.M.extent * P.N.extent / ((double)tiles_m * BM * tiles_n * BN);
     if (fill < 0.15) return false;                         // mostly empty tiles: the interpreter's schedules do better
-    // gather modes
+    // gather modes: the one whose warp-wide copy touches fewer 128-byte lines (lanes along the row index:
+    // 32 rows at one summation index; lanes along the summation index: 2 rows x 16 indices)
     auto mode_of = [&](const std::vector<Digit> &rows, bool second, const AGuard *gd, int64_t base) {
-        auto st = [&](const Digit &d) { return second ? d.sB : d.sA; };
-        const int64_t rs = rows.empty() ? 0 : std::llabs(st(rows.back()));
-        const int64_t ks = dk.empty() ? 0 : std::llabs(st(dk.back()));
-        const int64_t kext = dk.empty() ? 0 : dk.back().ext;
+        auto st = [&](const Digit &d) { return std::llabs(second ? d.sB : d.sA); };
+        // longest run of consecutive elements along the fastest digits of a group
+        auto run_of = [&](const std::vector<Digit> &ds) {
+            int64_t run = 1;
+            for (int d = (int)ds.size() - 1; d >= 0; --d) {
+                if (st(ds[d]) != run) break;
+                run *= ds[d].ext;
+            }
+            return run;
+        };
+        const int64_t rs = rows.empty() ? 0 : st(rows.back());
+        const int64_t ks = dk.empty() ? 0 : st(dk.back());
+        auto lines = [&](int64_t stride, int64_t run, int64_t ext, int64_t n) {     // n consecutive indices of a group
+            if (stride == 0) return int64_t(1);
+            if (stride == 1) return run >= n ? int64_t(1) : (n + run - 1) / run;
+            if (ext >= n) return std::min<int64_t>(n, (n * stride + 31) / 32);
+            return (n + ext - 1) / ext * std::max<int64_t>(1, (ext * stride + 31) / 32);
+        };
+        const int64_t lines_row = lines(rs, run_of(rows), rows.empty() ? 1 : rows.back().ext, 32);
+        const int64_t lines_k = lines(ks, run_of(dk), dk.empty() ? 1 : dk.back().ext, 16) * (rs * 2 <= 32 ? 1 : 2);
+        if (lines_k < lines_row) return TG_K;
         if (rs == 1) {
-            bool wide = st(rows.back()) == 1 && rows.back().ext % 4 == 0 && base % 4 == 0 && !(gd && gd->coef[rows.back().var]);
+            bool wide = (second ? rows.back().sB : rows.back().sA) == 1 && rows.back().ext % 4 == 0 && base % 4 == 0 &&
+                        !(gd && gd->coef[rows.back().var]);
             for (size_t d = 0; d + 1 < rows.size(); ++d) if (st(rows[d]) % 4) wide = false;
             for (const Digit &d : dk) if (st(d) % 4) wide = false;
             for (const Digit &d : dz) if (st(d) % 4) wide = false;
-            return wide ? TG_ROW16 : TG_ROW;
+            if (wide) return TG_ROW16;
         }
-        if (rs == 0) return TG_K;
-        if (ks == 1 && kext >= 8) return TG_K;
-        if (ks == 0 || rs <= ks) return TG_ROW;
-        return TG_K;
+        return TG_ROW;
     };
     P.modeA = mode_of(dm, false, ga, s.A.base);
     P.modeB = mode_of(dn, true, gb, s.B.base);
@@ -166,9 +182,17 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     const int64_t kstages = (P.K.extent + TADC_BK - 1) / TADC_BK;
     int64_t split = 1;
     if (allow_split && blocks < 222 && kstages >= 16) {
-        split = std::min<int64_t>((296 + blocks - 1) / blocks, kstages / 8);
+        // the number of chunks that fills whole waves of resident blocks best (two blocks per SM), every
+        // chunk at least eight stages long; fewer chunks win ties (less partial-sum traffic)
+        const int64_t wave = P.shape == 1 ? 444 : 296;
         const int64_t cells = (int64_t)P.M.extent * P.N.extent * P.Z.extent;
-        while (split > 1 && split * cells > (int64_t(1) << 25)) --split;            // <= 128 MB of partial sums
+        double best = 0;
+        for (int64_t s = 1; s <= std::min<int64_t>(kstages / 8, 256); ++s) {
+            if (s > 1 && s * cells > (int64_t(1) << 25)) break;                     // <= 128 MB of partial sums
+            const int64_t grid = blocks * s;
+            const double eff = (double)grid / (double)((grid + wave - 1) / wave * wave);
+            if (eff > best + 0.02) { best = eff; split = s; }
+        }
     }
     split = std::max<int64_t>(1, split);
     const int64_t per = ((kstages + split - 1) / split) * TADC_BK;

@@ -107,6 +107,22 @@ REDUCED = {
     "cfg5": lambda: conv1d(3, 13, 11, 70, 5, name="cfg5_reduced"),
 }
 
+def profile_case(key: str, rows: int) -> Expr:
+    """The structure of a full workload with a smaller leading extent: for profiler captures (a few
+    launches of a kernel whose tensors still exceed the L2 cache), never a benchmark number."""
+    if key == "cfg2":
+        return intro(rows, 8192, 32, name=f"cfg2_intro_scaled_rows{rows}")
+    if key == "cfg3":
+        return shifted(rows, name=f"cfg3_shifted_rows{rows}")
+    if key == "cfg4":
+        return nonunimodular(rows, name=f"cfg4_nonunimodular_rows{rows}")
+    if key == "cfg5":
+        e = conv1d(rows, 256, 256, 2048, 5, name=f"cfg5_conv1d_rows{rows}")
+        e.arg_shapes[0] = [rows, 256, 4099]
+        return e
+    raise ValueError("no reduced profile case for " + key)
+
+
 # value distributions per workload: ("uniform", lo, hi) or ("normal", mean, std)
 DIST = {
     "cfg1": ("uniform", -0.5, 0.5),
