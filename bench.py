@@ -215,7 +215,7 @@ def run_ours(opts):
         e = 0
         if events is not None:
             events[e].record(); e += 1
-        plan.forward(arg_ptrs, f.data_ptr(), stream)
+        plan.forward(arg_ptrs, f.data_ptr(), stream, ws.data_ptr(), ws.numel())
         if n_stages:
             if events is not None:
                 events[e].record(); e += 1

@@ -140,18 +140,25 @@ tad_status tad_compile(const tad_expr *expr, const tad_options *opt, tad_plan **
 /* Frees a plan (NULL is allowed).  The caller makes sure no launch still uses it. */
 void tad_destroy(tad_plan *plan);
 
-/* Bytes of device workspace tad_backward needs for this plan (may be 0).  The workspace
- * must be 256-byte aligned.  It holds the partial sums of gradients whose summation is
- * split over several thread blocks, and the debug word of a debug_bounds plan. */
+/* Bytes of device workspace tad_forward and tad_backward need for this plan (may be 0).  The
+ * workspace must be 256-byte aligned.  It holds the staged adjoints, the partial sums of
+ * summations that are split over several thread blocks, the auxiliary tensors of the
+ * expression optimisation (sums pushed inside the term: small pre-evaluated tensors and
+ * contraction results, Sec. 6's clean-up step), and the debug word of a debug_bounds plan.
+ * One workspace serves both calls; calls that share it must not overlap on the device. */
 size_t tad_workspace_bytes(const tad_plan *plan);
 
 /*
  * tad_forward: f[alpha] for every alpha of the output box (definition of an element-wise
  * specified function, Sec. 5.1; inner sums per Sec. 5.2).
- *   args  host array of n_args DEVICE pointers (read-only inputs), none NULL
- *   f     DEVICE pointer, prod(out_shape) floats, fully overwritten
+ *   args       host array of n_args DEVICE pointers (read-only inputs), none NULL
+ *   f          DEVICE pointer, prod(out_shape) floats, fully overwritten
+ *   workspace  DEVICE pointer, tad_workspace_bytes() bytes, 256-byte aligned, caller-owned.  Only plans
+ *              whose forward pass uses auxiliary tensors or a split summation read it; for every other
+ *              plan NULL / 0 is accepted.  TAD_ERR_WORKSPACE when it is needed and missing or too small.
  */
-tad_status tad_forward(const tad_plan *plan, const float *const *args, float *f, void *cuda_stream);
+tad_status tad_forward(const tad_plan *plan, const float *const *args, float *f,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * tad_backward: dx^p[beta] for every element of every requested argument, by the final

@@ -188,8 +188,10 @@ class Plan:
     def staging_bytes(self) -> int:
         return int(lib.tad_staging_bytes(self._h))
 
-    def forward(self, arg_ptrs: Sequence[int], f_ptr: int, stream: int = 0) -> None:
-        _check(lib.tad_forward(self._h, self._ptr_array(arg_ptrs), f_ptr, stream or None))
+    def forward(self, arg_ptrs: Sequence[int], f_ptr: int, stream: int = 0,
+                workspace_ptr: int = 0, workspace_bytes: int = 0) -> None:
+        _check(lib.tad_forward(self._h, self._ptr_array(arg_ptrs), f_ptr, workspace_ptr or None, workspace_bytes,
+                               stream or None))
 
     def backward(self, arg_ptrs: Sequence[int], df_ptr: int, darg_ptrs: Sequence[Optional[int]],
                  workspace_ptr: int = 0, workspace_bytes: int = 0, stream: int = 0) -> None:

@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <cstring>
 #include <map>
+#include <functional>
 #include <tuple>
 
 #include "gen.h"
@@ -556,7 +557,8 @@ int body_fetch_kind(const TadpLoad &L, int ta, int ub)
 
 // shared tail: choose temps, emit, fill the program
 void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<TadpRow>> &lower,
-                 const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards, bool allow_split = false)
+                 const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards, bool allow_split = false,
+                 bool may_factor = true)
 {
     TadpProgram &prog = k.prog;
     place(g);
@@ -596,6 +598,8 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     }
     // a product of two index expressions under summations runs on the tile kernel, not in the interpreter
     if (try_contraction(g, k, root, scale, allow_split, lower, upper, guards)) return;
+    // sums that can be pushed inside the term (Sec. 6's missing clean-up step): auxiliary kernels + a smaller kernel
+    if (may_factor && try_factoring(g, k, root, scale, allow_split, lower, upper, guards)) return;
     // a short loop whose range shifts from lane to lane will be walked relative to every element's own
     // start, which needs the elements of a thread to lie along the lane variable only
     bool relative_candidate = false;
@@ -899,6 +903,36 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
 
 }  // namespace
 
+void emit_plain_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<TadpRow>> &lower,
+                       const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards, bool allow_split)
+{
+    count_uses(g, root);
+    emit_kernel(g, k, root, lower, upper, guards, allow_split, false);
+}
+
+// workspace needs and launches of a kernel with its auxiliary kernels
+static void account(tad_plan &p, Kernel &k)
+{
+    std::function<void(const Kernel &)> walk = [&](const Kernel &x) {
+        if (x.contract.empty() && x.prog.zsplit > 1)
+            p.partial_bytes = std::max(p.partial_bytes, (size_t(x.prog.zsplit) + 1) * size_t(x.prog.part_limit) * 4);
+        for (const TadcProgram &cp : x.contract)
+            if (cp.ksplit > 1)
+                p.partial_bytes = std::max(p.partial_bytes, size_t(cp.ksplit) * size_t(cp.M.extent) * size_t(cp.N.extent) * size_t(cp.Z.extent) * 4);
+        for (const Kernel &y : x.pre) walk(y);
+    };
+    walk(k);
+    p.aux_bytes = std::max(p.aux_bytes, k.aux_bytes);
+    std::function<int(const Kernel &)> launches = [&](const Kernel &x) {
+        int n = 0;
+        if (x.contract.empty()) n = 1 + (x.prog.zsplit > 1 ? 1 + (x.prog.write_only_live ? 1 : 0) : 0);
+        for (const TadcProgram &cp : x.contract) n += 1 + (cp.ksplit > 1 ? 1 : 0);
+        for (const Kernel &y : x.pre) n += launches(y);
+        return n;
+    };
+    k.stats.n_launches = launches(k);
+}
+
 // ---------------------------------------------------------------------------------------
 // forward: outer variables are the output indices, every sum is a bound loop
 // ---------------------------------------------------------------------------------------
@@ -929,8 +963,9 @@ void finish_alpha_kernel(tad_plan &p, Gen &g, Kernel &k, int root)
     }
     prog.out_base = 0; prog.out_limit = to_i32(p.out_elems);
     prog.accumulate = 0; prog.write_only_live = 0;
-    emit_kernel(g, k, root, {}, {}, {});
+    emit_kernel(g, k, root, {}, {}, {}, true);
     finish_stats(g, k, false, p.out_elems, 0, false);
+    account(p, k);
 }
 
 }  // namespace
@@ -1193,16 +1228,8 @@ void generate_backward(tad_plan &p, int q)
     int64_t terms = 1;
     for (int d = 0; d < n; ++d) terms = mul_ck(terms, ap.box_hi[d] - ap.box_lo[d] + 1);
     finish_stats(g, k, true, p.arg_elems[ap.arg], terms, zero_fill && first_of_arg);
-    if (prog.zsplit > 1 && k.contract.empty()) {
-        p.partial_bytes = std::max(p.partial_bytes, (size_t(prog.zsplit) + 1) * size_t(prog.part_limit) * 4);
-        k.stats.n_launches += 1 + (prog.write_only_live ? 1 : 0);
-    }
-    for (const TadcProgram &cp : k.contract)
-        if (cp.ksplit > 1) {
-            p.partial_bytes = std::max(p.partial_bytes, size_t(cp.ksplit) * size_t(cp.M.extent) * size_t(cp.N.extent) * size_t(cp.Z.extent) * 4);
-            k.stats.n_launches += 1;
-        }
-    if (k.contract.size() > 1) k.stats.n_launches += (int)k.contract.size() - 1;
+    account(p, k);
+    if (zero_fill && first_of_arg) k.stats.n_launches += 1;
 }
 
 }  // namespace tad

@@ -174,8 +174,9 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
     // Offsets are sums of signed 32-bit parts that may be negative one by one (a band that starts below
     // zero, a negative stride); only the complete sum of a live element is a valid element offset, so the
     // constant parts go into the row tables and the pointer stays the tensor's own.
+    const bool onesB = P.ptrB < 0;                // B is a tensor of ones: a plain summation of A
     const float *__restrict__ A = ptrs.in[P.ptrA];
-    const float *__restrict__ B = ptrs.in[P.ptrB];
+    const float *__restrict__ B = onesB ? A : ptrs.in[P.ptrB];
     const int constA = P.baseA + z.a, constB = P.baseB + z.b;
     const unsigned Mext = (unsigned)P.M.extent, Next = (unsigned)P.N.extent;
     const unsigned kbeg = ks * (unsigned)P.kchunk;
@@ -203,6 +204,11 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
         }
     };
     for (int s = 0; s < STAGES; ++s) fill_ktab(s);
+    if (onesB)
+        for (unsigned e = tid; e < (unsigned)(STAGES * BK * LDB); e += NT) {
+            const unsigned s = e / (BK * LDB), r = e - s * (BK * LDB);
+            stage_mem[s * C::STAGE_FLOATS + BK * LDA + r] = 1.f;
+        }
     __syncthreads();
     const unsigned gextA = (unsigned)P.guardA_ext, gextB = (unsigned)P.guardB_ext;
     const int modeA = P.modeA, modeB = P.modeB;
@@ -219,7 +225,8 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
             const bool full = kbeg + (unsigned)(kstage + 1) * BK <= kend;
             if (plainA && full) gather<BM, NT, false>(as, A, rowA, ktabA + slot, preA, modeA, gextA, tid);
             else gather<BM, NT, true>(as, A, rowA, ktabA + slot, preA, modeA, gextA, tid);
-            if (plainB && full) gather<BN, NT, false>(bs, B, rowB, ktabB + slot, preB, modeB, gextB, tid);
+            if (onesB) {}
+            else if (plainB && full) gather<BN, NT, false>(bs, B, rowB, ktabB + slot, preB, modeB, gextB, tid);
             else gather<BN, NT, true>(bs, B, rowB, ktabB + slot, preB, modeB, gextB, tid);
         }
         cp_async_commit();
@@ -364,7 +371,8 @@ cudaError_t launch_shape(const TadcProgram &P, const TadpPointers &ptrs, cudaStr
 cudaError_t tad_launch_contract(const TadcProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream)
 {
     if (P.M.extent <= 0 || P.N.extent <= 0 || P.Z.extent <= 0) return cudaSuccess;
-    cudaError_t e = P.shape == 1 ? launch_shape<128, 32, 4, 4>(P, ptrs, stream) : launch_shape<128, 128, 8, 8>(P, ptrs, stream);
+    cudaError_t e = P.shape == 1 ? launch_shape<128, 32, 4, 4>(P, ptrs, stream)
+                  : P.shape == 2 ? launch_shape<128, 64, 8, 4>(P, ptrs, stream) : launch_shape<128, 128, 8, 8>(P, ptrs, stream);
     if (e != cudaSuccess) return e;
     if (P.ksplit > 1) {
         const unsigned long long cells = (unsigned long long)P.M.extent * P.N.extent * P.Z.extent;

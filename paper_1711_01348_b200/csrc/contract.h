@@ -39,7 +39,7 @@ enum TadcEpilogueOp : int { TE_END = 0, TE_NEG, TE_EXP, TE_MULC, TE_ADDC, TE_MUL
 
 struct alignas(16) TadcProgram {
     TadcGroup M, N, K, Z;
-    int32_t ptrA, ptrB;            // pointer slots of the operands
+    int32_t ptrA, ptrB;            // pointer slots of the operands; ptrB < 0: B is all ones (a plain summation of A)
     int32_t baseA, baseB, baseO;   // constant element offsets
     // an operand element is read as zero unless 0 <= c0 + sum(g * digit) < ext (guard = 1), always read when guard = 0
     int32_t guardA, guardA_c0, guardA_ext;
@@ -49,7 +49,7 @@ struct alignas(16) TadcProgram {
     int32_t kchunk;                // summation indices per chunk (a multiple of TADC_BK)
     int32_t accumulate;            // 1: out += result
     int32_t out_vec4;              // 1: four consecutive n are four consecutive, 16-byte aligned output elements
-    int32_t shape;                 // tile shape: 0 = 128 x 128 (8 x 8 per thread), 1 = 128 x 32 (4 x 4 per thread)
+    int32_t shape;                 // tile shape: 0 = 128 x 128 (8 x 8 per thread), 1 = 128 x 32 (4 x 4), 2 = 128 x 64 (8 x 4)
     float scale;
     int32_t n_epi;
     int32_t epi_op[TADC_MAX_EPI];

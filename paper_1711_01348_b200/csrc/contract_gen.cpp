@@ -26,17 +26,6 @@ namespace tad {
 
 namespace {
 
-struct AVar { int64_t ext; bool reduce; };               // values 0 .. ext-1 after normalisation
-struct AMap { int ptr = 0; int64_t base = 0, limit = 0; std::vector<int64_t> coef; };   // limit: elements in the tensor
-struct AGuard { std::vector<int64_t> coef; int64_t c0 = 0, ext = 1; };   // live iff 0 <= c0 + coef . vars < ext
-
-struct System {
-    std::vector<AVar> vars;
-    AMap A, B, O;
-    std::vector<AGuard> guards;
-    bool loose_box = false;     // the outer box is a bounding box of the live elements, not the set itself
-};
-
 int32_t fit(int64_t v) { if (std::llabs(v) >= (int64_t(1) << 31)) throw Overflow(); return (int32_t)v; }
 
 struct Digit { int var; int64_t ext, sA, sB, sO; };
@@ -58,17 +47,20 @@ bool fill_group(TadcGroup &G, std::vector<Digit> &ds, const AGuard *ga, const AG
     return true;
 }
 
+}  // namespace
+
 // builds one contraction program from a system whose loops all have fixed ranges
-bool emit_program(const System &s0, float scale, int accumulate, bool allow_split, TadcProgram &P, std::string &text)
+bool emit_program(const System &s0, float scale, int accumulate, bool allow_split, bool strict_fill, TadcProgram &P, std::string &text)
 {
     System s = s0;
     const int nv = (int)s.vars.size();
+    if (s.A.ptr < 0) std::swap(s.A, s.B);                  // an operand of ones plays B
     // which factor plays A: the variable along which the output is contiguous should index columns
     int contiguous = -1;
     for (int v = 0; v < nv; ++v)
         if (!s.vars[v].reduce && s.O.coef[v] != 0 && s.vars[v].ext > 1 &&
             (contiguous < 0 || std::llabs(s.O.coef[v]) < std::llabs(s.O.coef[contiguous]))) contiguous = v;
-    if (contiguous >= 0 && s.A.coef[contiguous] != 0 && s.B.coef[contiguous] == 0) std::swap(s.A, s.B);
+    if (contiguous >= 0 && s.A.coef[contiguous] != 0 && s.B.coef[contiguous] == 0 && s.B.ptr >= 0) std::swap(s.A, s.B);
     std::vector<Digit> dm, dn, dk, dz;
     for (int v = 0; v < nv; ++v) {
         if (s.vars[v].ext == 1) continue;                  // a single value: nothing to index
@@ -103,7 +95,7 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     // (an operand under a guard is checked over the guarded range of its guard expression only when the
     // guard is the identity on one digit pair, so it is skipped here: the guard itself bounds the reads)
     auto in_range = [&](const AMap &m, bool guarded) {
-        if (guarded) return true;
+        if (guarded || m.ptr < 0) return true;
         int64_t lo = m.base, hi = m.base;
         for (int v = 0; v < nv; ++v) {
             if (s.vars[v].ext <= 1) { if (s.vars[v].ext <= 0) return true; continue; }
@@ -116,7 +108,13 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
         // a masked index expression iterates a bounding box of its image lattice and the interpreter skips the
         // elements without terms; the tile kernel would touch them, so such a kernel stays with the interpreter
         if (s.loose_box) return false;
-        throw BadExpr("internal: contraction offsets leave their tensor");
+        std::string what = "internal: contraction offsets leave their tensor:";
+        for (const AMap *m : {&s.A, &s.B, &s.O}) {
+            what += " [ptr " + std::to_string(m->ptr) + " base " + std::to_string(m->base) + " limit " + std::to_string(m->limit) + " coef";
+            for (int v = 0; v < nv; ++v) if (m->coef[v]) what += " " + std::to_string(v) + ":" + std::to_string(m->coef[v]) + "x" + std::to_string(s.vars[v].ext);
+            what += "]";
+        }
+        throw BadExpr(what);
     }
     P = TadcProgram{};
     if (!fill_group(P.M, dm, ga, nullptr) || !fill_group(P.N, dn, nullptr, gb) || !fill_group(P.K, dk, ga, gb) ||
@@ -128,11 +126,11 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     P.guardB = gb ? 1 : 0; P.guardB_c0 = gb ? fit(gb->c0) : 0; P.guardB_ext = gb ? fit(gb->ext) : 1;
     P.scale = scale; P.accumulate = accumulate;
     // tile shape: narrow column tiles for narrow outputs
-    P.shape = P.N.extent <= 48 ? 1 : 0;
-    const int64_t BM = 128, BN = P.shape == 1 ? 32 : 128;
+    P.shape = P.N.extent <= 32 ? 1 : P.N.extent <= 64 ? 2 : 0;
+    const int64_t BM = 128, BN = P.shape == 1 ? 32 : P.shape == 2 ? 64 : 128;
     const int64_t tiles_m = (P.M.extent + BM - 1) / BM, tiles_n = (P.N.extent + BN - 1) / BN;
     const double fill = (double)P.M.extent * P.N.extent / ((double)tiles_m * BM * tiles_n * BN);
-    if (fill < 0.15) return false;                         // mostly empty tiles: the interpreter's schedules do better
+    if (strict_fill && fill < 0.15) return false;          // mostly empty tiles: the interpreter's schedules do better
     // gather modes: the one whose warp-wide copy touches fewer 128-byte lines (lanes along the row index:
     // 32 rows at one summation index; lanes along the summation index: 2 rows x 16 indices)
     auto mode_of = [&](const std::vector<Digit> &rows, bool second, const AGuard *gd, int64_t base) {
@@ -168,7 +166,7 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
         return TG_ROW;
     };
     P.modeA = mode_of(dm, false, ga, s.A.base);
-    P.modeB = mode_of(dn, true, gb, s.B.base);
+    P.modeB = s.B.ptr < 0 ? TG_ROW : mode_of(dn, true, gb, s.B.base);
     // output: four consecutive columns are four consecutive aligned elements
     P.out_vec4 = 0;
     if (!dn.empty() && dn.back().sO == 1 && dn.back().ext % 4 == 0 && s.O.base % 4 == 0) {
@@ -184,7 +182,7 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     if (allow_split && blocks < 222 && kstages >= 16) {
         // the number of chunks that fills whole waves of resident blocks best (two blocks per SM), every
         // chunk at least eight stages long; fewer chunks win ties (less partial-sum traffic)
-        const int64_t wave = P.shape == 1 ? 444 : 296;
+        const int64_t wave = P.shape == 0 ? 296 : 444;
         const int64_t cells = (int64_t)P.M.extent * P.N.extent * P.Z.extent;
         double best = 0;
         for (int64_t s = 1; s <= std::min<int64_t>(kstages / 8, 256); ++s) {
@@ -210,13 +208,11 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     };
     std::snprintf(line, sizeof line, "; contraction %d x %d x %d (batch %d): A=ptr %d mode %d guard %d, B=ptr %d mode %d guard %d, tile %s, ksplit %d x %d, vec4 %d, scale %g, accumulate %d\n",
                   P.M.extent, P.N.extent, P.K.extent, P.Z.extent, P.ptrA, P.modeA, P.guardA, P.ptrB, P.modeB, P.guardB,
-                  P.shape == 1 ? "128x32" : "128x128", P.ksplit, P.kchunk, P.out_vec4, (double)P.scale, P.accumulate);
+                  P.shape == 1 ? "128x32" : P.shape == 2 ? "128x64" : "128x128", P.ksplit, P.kchunk, P.out_vec4, (double)P.scale, P.accumulate);
     text += line;
     text += group_text("m", P.M) + group_text("n", P.N) + group_text("k", P.K) + group_text("z", P.Z);
     return true;
 }
-
-}  // namespace
 
 bool try_contraction(Gen &g, Kernel &k, int root, int scale, bool allow_split, const std::vector<std::vector<TadpRow>> &lower,
                      const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards)
@@ -370,7 +366,7 @@ bool try_contraction(Gen &g, Kernel &k, int root, int scale, bool allow_split, c
         for (int v = 0; v < nv; ++v) if (!s.vars[v].reduce && s.vars[v].ext <= 0) empty_out = true;
         if (empty_out) continue;
         TadcProgram P;
-        if (!emit_program(s, cfac, prog.accumulate, allow_split, P, text)) return false;
+        if (!emit_program(s, cfac, prog.accumulate, allow_split, true, P, text)) return false;
         progs.push_back(P);
     }
     if (progs.empty()) return false;

@@ -321,10 +321,34 @@ struct Gen {
 
 inline int32_t to_i32(int64_t v) { if (std::llabs(v) >= (int64_t(1) << 31)) throw Overflow(); return (int32_t)v; }
 
+// ---- affine description of a contraction (contract_gen.cpp) ---------------------------------
+struct AVar { int64_t ext; bool reduce; };               // values 0 .. ext-1 after normalisation
+struct AMap { int ptr = 0; int64_t base = 0, limit = 0; std::vector<int64_t> coef; };   // limit: elements in the tensor
+struct AGuard { std::vector<int64_t> coef; int64_t c0 = 0, ext = 1; };   // live iff 0 <= c0 + coef . vars < ext
+
+struct System {
+    std::vector<AVar> vars;
+    AMap A, B, O;
+    std::vector<AGuard> guards;
+    bool loose_box = false;     // the outer box is a bounding box of the live elements, not the set itself
+};
+
+// builds one contraction program from a system whose loops all have fixed ranges; an operand with ptr < 0 is
+// a tensor of ones (a plain summation of the other operand).  strict_fill: refuse mostly empty tiles
+bool emit_program(const System &s, float scale, int accumulate, bool allow_split, bool strict_fill, TadcProgram &P, std::string &text);
+
 // contract_gen.cpp: recognises a kernel whose term is a product of two index expressions summed over
 // loops with fixed ranges and fills k.contract; returns false (and leaves k alone) otherwise.
 // allow_split: the caller has a workspace for partial sums of a split summation
 bool try_contraction(Gen &g, Kernel &k, int root, int scale, bool allow_split, const std::vector<std::vector<TadpRow>> &lower,
                      const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards);
+
+// factor.cpp: the expression optimisation pass; fills k.pre / k.aux and emits the kernel itself when it
+// finds summations worth pushing inside the term, returns false (k untouched) otherwise
+bool try_factoring(Gen &g, Kernel &k, int root, int scale, bool allow_split, const std::vector<std::vector<TadpRow>> &lower,
+                   const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards);
+// codegen.cpp: schedules and emits one kernel without running the optimisation pass on it
+void emit_plain_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<TadpRow>> &lower,
+                       const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards, bool allow_split);
 
 }  // namespace tad

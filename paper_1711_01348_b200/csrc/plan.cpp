@@ -33,7 +33,8 @@ void build_expression(tad_plan &p, const tad_expr *e, const tad_options *opt)
         throw InvalidArg("NULL array in tad_expr");
     const int n_idx = e->n_out_dims + e->n_sum_idx;
     if (n_idx > TAD_MAX_IDX) throw Unsupported("more than TAD_MAX_IDX output + sum indices");
-    if (e->n_args + 1 > TADP_MAX_PTRS) throw Unsupported("too many arguments");
+    // pointer slots: the arguments, df, and the saved forward output when the plan reads it
+    if (e->n_args + 1 + ((opt && opt->saved_forward) ? 1 : 0) > TADP_MAX_PTRS) throw Unsupported("too many arguments");
     p.n_out = e->n_out_dims; p.n_sum = e->n_sum_idx; p.n_args = e->n_args;
     p.out_shape.assign(e->out_shape, e->out_shape + e->n_out_dims);
     p.out_elems = 1;

@@ -70,6 +70,13 @@ struct Kernel {
     std::vector<int> stages_used;   // backward: staged adjoints it reads (indices into tad_plan::stages)
     std::vector<TadcProgram> contract;   // non-empty: the kernel is a contraction, run by the tile kernel (one launch per
                                          // program) instead of the interpreter
+    // Expression optimisation: tensors in the auxiliary area of the workspace and the kernels that fill them
+    // (launched in this order before the kernel itself, each writing the tensor out_aux)
+    struct Aux { size_t offset = 0, bytes = 0; int slot = 0; };
+    std::vector<Aux> aux;
+    size_t aux_bytes = 0;
+    std::vector<Kernel> pre;
+    int out_aux = -1;
     KernelStats stats;
     std::string listing;
 };
@@ -99,6 +106,7 @@ struct tad_plan {
     std::vector<std::vector<int>> arg_kernels;  // per argument: indices into backward, launch order
     std::vector<bool> arg_zero_fill;            // the gradient is cleared before its kernels add into it
     size_t partial_bytes = 0;                   // workspace for the partial sums of split summations (largest kernel)
+    size_t aux_bytes = 0;                       // workspace for auxiliary tensors (largest kernel)
 };
 
 namespace tad {

@@ -11,7 +11,7 @@
 #define TADP_MAX_LOADS 20
 #define TADP_MAX_LOOPS 8
 #define TADP_MAX_ROWS 40      // bound rows + guard rows
-#define TADP_MAX_PTRS 8       // arguments + df + staged adjoints + saved forward output
+#define TADP_MAX_PTRS 16      // arguments + df + staged adjoints + saved forward output
 #define TADP_F_SLOT (TADP_MAX_PTRS - 1)   // pointer slot of the saved forward output (plans compiled with saved_forward)
 #define TADP_MAX_DEPTH 8      // handlers are encoded for operand stack depths 0..7
 #define TADP_NUM_TEMPS 8      // temporaries held in registers; further ones spill to local memory

@@ -100,7 +100,7 @@ tad_status launch_contractions(const tad::Kernel &k, const TadpPointers &ptrs, c
         // 16-byte copies and stores need 16-byte aligned tensors: fall back to 4-byte accesses otherwise
         auto misaligned = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
         if (P.modeA == TG_ROW16 && misaligned(ptrs.in[P.ptrA])) P.modeA = TG_ROW;
-        if (P.modeB == TG_ROW16 && misaligned(ptrs.in[P.ptrB])) P.modeB = TG_ROW;
+        if (P.ptrB >= 0 && P.modeB == TG_ROW16 && misaligned(ptrs.in[P.ptrB])) P.modeB = TG_ROW;
         if (P.out_vec4 && misaligned(ptrs.out)) P.out_vec4 = 0;
         const cudaError_t e = tad_launch_contract(P, ptrs, (unsigned)sm_count(), stream);
         if (e != cudaSuccess) { tad::set_error(std::string("contraction launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
@@ -108,8 +108,19 @@ tad_status launch_contractions(const tad::Kernel &k, const TadpPointers &ptrs, c
     return TAD_OK;
 }
 
-tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStream_t stream)
+tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStream_t stream, char *aux_base = nullptr)
 {
+    if (!k.aux.empty()) {
+        // auxiliary tensors of this kernel, then the kernels that fill them, in order
+        if (!aux_base) { tad::set_error("this plan needs a workspace (auxiliary tensors): pass one of tad_workspace_bytes() bytes"); return TAD_ERR_WORKSPACE; }
+        for (const tad::Kernel::Aux &a : k.aux) ptrs.in[a.slot] = reinterpret_cast<const float *>(aux_base + a.offset);
+        for (const tad::Kernel &pk : k.pre) {
+            TadpPointers pp = ptrs;
+            pp.out = reinterpret_cast<float *>(aux_base + k.aux[pk.out_aux].offset);
+            const tad_status st = launch(pk, pp, debug, stream);
+            if (st != TAD_OK) return st;
+        }
+    }
     if (!k.contract.empty()) return launch_contractions(k, ptrs, stream);
     const int zsplit = k.prog.zsplit > 1 ? k.prog.zsplit : 1;
     if (zsplit > 1) {
@@ -170,6 +181,20 @@ size_t stage_offset(const tad_plan *plan, int s)
     return (plan->opt.debug_bounds ? 256 : 0) + size_t(s) * pad256(size_t(plan->out_elems) * 4);
 }
 
+// workspace layout: ... [planes of partial sums][auxiliary tensors]
+size_t aux_offset(const tad_plan *plan)
+{
+    return stage_offset(plan, (int)plan->stages.size()) + pad256(plan->partial_bytes);
+}
+
+// some kernel of the forward pass divides a summation among blocks (planes of partial sums in the workspace)
+bool forward_splits(const tad::Kernel &k)
+{
+    for (const TadcProgram &cp : k.contract) if (cp.ksplit > 1) return true;
+    for (const tad::Kernel &pk : k.pre) if (forward_splits(pk) || (pk.contract.empty() && pk.prog.zsplit > 1)) return true;
+    return false;
+}
+
 bool check_workspace(const tad_plan *plan, void *workspace, size_t workspace_bytes)
 {
     const size_t need = tad_workspace_bytes(plan);
@@ -206,12 +231,15 @@ extern "C" {
 size_t tad_workspace_bytes(const tad_plan *plan)
 {
     if (!plan) return 0;
-    return stage_offset(plan, (int)plan->stages.size()) + pad256(plan->partial_bytes);
+    return aux_offset(plan) + pad256(plan->aux_bytes);
 }
 
-tad_status tad_forward(const tad_plan *plan, const float *const *args, float *f, void *cuda_stream)
+tad_status tad_forward(const tad_plan *plan, const float *const *args, float *f,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream)
 {
     if (!plan || !f || (plan->n_args && !args)) { tad::set_error("NULL argument"); return TAD_ERR_INVALID_ARG; }
+    const bool needs_ws = !plan->forward.aux.empty() || forward_splits(plan->forward);
+    if (needs_ws && !check_workspace(plan, workspace, workspace_bytes)) return TAD_ERR_WORKSPACE;
     TadpPointers ptrs{};
     for (int a = 0; a < plan->n_args; ++a) {
         if (!args[a]) { tad::set_error("NULL argument tensor"); return TAD_ERR_INVALID_ARG; }
@@ -219,7 +247,13 @@ tad_status tad_forward(const tad_plan *plan, const float *const *args, float *f,
     }
     ptrs.out = f;
     ptrs.debug = nullptr;
-    return launch(plan->forward, ptrs, false, (cudaStream_t)cuda_stream);
+    char *aux_base = nullptr;
+    if (needs_ws) {
+        ptrs.part = plan->partial_bytes
+            ? reinterpret_cast<float *>(static_cast<char *>(workspace) + stage_offset(plan, (int)plan->stages.size())) : nullptr;
+        aux_base = static_cast<char *>(workspace) + aux_offset(plan);
+    }
+    return launch(plan->forward, ptrs, false, (cudaStream_t)cuda_stream, aux_base);
 }
 
 tad_status tad_backward_stage(const tad_plan *plan, const float *const *args, const float *df,
@@ -231,7 +265,8 @@ tad_status tad_backward_stage(const tad_plan *plan, const float *const *args, co
     if (!fill_inputs(plan, args, df, workspace, ptrs)) return TAD_ERR_INVALID_ARG;
     for (int s = 0; s < (int)plan->stages.size(); ++s) {
         ptrs.out = reinterpret_cast<float *>(static_cast<char *>(workspace) + stage_offset(plan, s));
-        tad_status st = launch(plan->stages[s], ptrs, plan->opt.debug_bounds != 0, (cudaStream_t)cuda_stream);
+        tad_status st = launch(plan->stages[s], ptrs, plan->opt.debug_bounds != 0, (cudaStream_t)cuda_stream,
+                               workspace ? static_cast<char *>(workspace) + aux_offset(plan) : nullptr);
         if (st != TAD_OK) return st;
     }
     return TAD_OK;
@@ -252,7 +287,8 @@ tad_status tad_backward_arg(const tad_plan *plan, const float *const *args, cons
     }
     ptrs.out = darg;
     for (int ki : plan->arg_kernels[arg]) {
-        tad_status st = launch(plan->backward[ki], ptrs, plan->opt.debug_bounds != 0, stream);
+        tad_status st = launch(plan->backward[ki], ptrs, plan->opt.debug_bounds != 0, stream,
+                               workspace ? static_cast<char *>(workspace) + aux_offset(plan) : nullptr);
         if (st != TAD_OK) return st;
     }
     return TAD_OK;
@@ -353,7 +389,7 @@ tad_status tad_step_host(const tad_plan *plan, const float *const *h_args, const
     tad_status st = TAD_OK;
     if (!check(cudaStreamWaitEvent(stream, ev_args, 0), "stream wait")) return TAD_ERR_CUDA;
     if (h_f || plan->opt.saved_forward) {
-        st = tad_forward(plan, d_args, d_f, stream);
+        st = tad_forward(plan, d_args, d_f, ws, tad_workspace_bytes(plan), stream);
         if (st != TAD_OK) return st;
         if (h_f) {
             if (!check(cudaEventRecord(ev_f, stream), "event record") || !check(cudaStreamWaitEvent(side.out, ev_f, 0), "stream wait") ||

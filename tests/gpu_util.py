@@ -27,7 +27,7 @@ class GpuRun:
 
     def forward(self):
         stream = torch.cuda.current_stream().cuda_stream
-        self.plan.forward([a.data_ptr() for a in self.args], self.f.data_ptr(), stream)
+        self.plan.forward([a.data_ptr() for a in self.args], self.f.data_ptr(), stream, self.ws.data_ptr(), self.ws.numel())
         torch.cuda.synchronize()
         return self.f.cpu().numpy()
 
