@@ -16,7 +16,7 @@
 namespace {
 
 constexpr int BK = TADC_BK;
-constexpr int KK_UNROLL = 8;           // summation indices per unrolled body of the multiply-add loop
+constexpr int KK_UNROLL = 8;          // summation indices per unrolled body of the multiply-add loop
 constexpr int STAGES = 2;
 constexpr int DEAD = INT_MIN / 2;      // guard part of a row or summation index that does not exist
 
@@ -266,61 +266,103 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
             }
         };
         fetch(0, a[0], b[0]);
-#pragma unroll KK_UNROLL
-        for (int kk = 0; kk < BK; ++kk) {
-            if (kk + 1 < BK) fetch(kk + 1, a[(kk + 1) & 1], b[(kk + 1) & 1]);
+        // bodies of KK_UNROLL summation indices; a last stage with few indices left runs only the bodies that hold some
+        const int n_bodies = min(BK / KK_UNROLL, (int)(((kend - kbeg) - (unsigned)it * BK + KK_UNROLL - 1) / KK_UNROLL));
+        for (int body = 0; body < n_bodies; ++body) {
+            const float *as_b = as + body * KK_UNROLL * LDA, *bs_b = bs + body * KK_UNROLL * LDB;
 #pragma unroll
-            for (int i = 0; i < TM; ++i)
+            for (int u = 0; u < KK_UNROLL; ++u) {
+                if (u + 1 < KK_UNROLL || body + 1 < n_bodies) {
 #pragma unroll
-                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[kk & 1][i], b[kk & 1][j], acc[i][j]);
+                    for (int q = 0; q < GM; ++q) {
+                        const float4 v = *reinterpret_cast<const float4 *>(as_b + (u + 1) * LDA + q * (BM / GM) + ty * 4);
+                        a[(u + 1) & 1][4 * q] = v.x; a[(u + 1) & 1][4 * q + 1] = v.y; a[(u + 1) & 1][4 * q + 2] = v.z; a[(u + 1) & 1][4 * q + 3] = v.w;
+                    }
+#pragma unroll
+                    for (int q = 0; q < GN; ++q) {
+                        const float4 v = *reinterpret_cast<const float4 *>(bs_b + (u + 1) * LDB + q * (BN / GN) + tx * 4);
+                        b[(u + 1) & 1][4 * q] = v.x; b[(u + 1) & 1][4 * q + 1] = v.y; b[(u + 1) & 1][4 * q + 2] = v.z; b[(u + 1) & 1][4 * q + 3] = v.w;
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < TM; ++i)
+#pragma unroll
+                    for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[u & 1][i], b[u & 1][j], acc[i][j]);
+            }
         }
     }
     cp_async_wait<0>();
 
     // ---- store ----
-    const bool partial = P.ksplit > 1;
-    float *__restrict__ out = partial ? ptrs.part : ptrs.out;
-    const float scale = P.scale;
+    // The sums go through shared memory (the stage buffers are free now): a compact loop then applies the epilogue
+    // to four columns at a time and writes whole rows of the tile, consecutive threads to consecutive columns.
+    // (Storing straight from the 64 registers would unroll the epilogue 64 times: code that no longer fits the
+    // instruction cache and is run once per tile.)
+    constexpr int LDC = BN + 4;
+    static_assert(BM * LDC <= STAGES * C::STAGE_FLOATS, "the tile of sums must fit into the stage buffers");
+    float *cs = stage_mem;
+    __syncthreads();
 #pragma unroll
     for (int i = 0; i < TM; ++i) {
         const int rl = (i / 4) * (BM / GM) + ty * 4 + (i % 4);
-        const unsigned m = tile_m * BM + rl;
-        if (m >= Mext) continue;
 #pragma unroll
-        for (int g = 0; g < GN; ++g) {
-            const int cl = g * (BN / GN) + tx * 4;
-            const unsigned n = tile_n * BN + cl;
-            if (n >= Next) continue;
-            if (partial) {
-                float *dst = out + ((size_t)(zb * (unsigned)P.ksplit + ks) * Mext + m) * Next + n;
-                if ((Next & 3u) == 0) *reinterpret_cast<float4 *>(dst) = make_float4(acc[i][4 * g], acc[i][4 * g + 1], acc[i][4 * g + 2], acc[i][4 * g + 3]);
-                else {
+        for (int q = 0; q < GN; ++q)
+            *reinterpret_cast<float4 *>(cs + rl * LDC + q * (BN / GN) + tx * 4) =
+                make_float4(acc[i][4 * q], acc[i][4 * q + 1], acc[i][4 * q + 2], acc[i][4 * q + 3]);
+    }
+    __syncthreads();
+    const bool partial = P.ksplit > 1;
+    float *__restrict__ out = partial ? ptrs.part : ptrs.out;
+    const float scale = P.scale;
+    const int n_epi = partial ? 0 : P.n_epi;
+    const int obase = P.baseO + z.o;
+    const bool vec_ok = partial ? (Next & 3u) == 0 : P.out_vec4 != 0;
+    for (unsigned e = tid; e < (unsigned)(BM * BN / 4); e += NT) {
+        const unsigned rl = e / (BN / 4), cl = (e % (BN / 4)) * 4;
+        const unsigned m = tile_m * BM + rl, n = tile_n * BN + cl;
+        if (m >= Mext || n >= Next) continue;
+        const float4 s4 = *reinterpret_cast<const float4 *>(cs + rl * LDC + cl);
+        float v[4] = {s4.x, s4.y, s4.z, s4.w};
+        unsigned off[4];
+        if (partial) {
+            const unsigned o0 = (unsigned)(((zb * (unsigned)P.ksplit + ks) * Mext + m) * Next + n);     // < 2^25 cells per plane set
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) if (n + j < Next) dst[j] = acc[i][4 * g + j];
-                }
-            } else {
-                const int ob = P.baseO + z.o + outM[rl];
-                if (P.out_vec4) {
-                    const unsigned off = (unsigned)(ob + outN[cl]);
-                    float4 v;
-                    v.x = epilogue(P, ptrs, acc[i][4 * g] * scale, off);
-                    v.y = epilogue(P, ptrs, acc[i][4 * g + 1] * scale, off + 1);
-                    v.z = epilogue(P, ptrs, acc[i][4 * g + 2] * scale, off + 2);
-                    v.w = epilogue(P, ptrs, acc[i][4 * g + 3] * scale, off + 3);
-                    float4 *dst = reinterpret_cast<float4 *>(out + off);
-                    if (P.accumulate) { const float4 o = *dst; v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w; }
-                    *dst = v;
-                } else {
+            for (int j = 0; j < 4; ++j) off[j] = o0 + j;
+        } else {
+            const int ob = obase + outM[rl];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (n + j >= Next) continue;
-                        const unsigned off = (unsigned)(ob + outN[cl + j]);
-                        float v = epilogue(P, ptrs, acc[i][4 * g + j] * scale, off);
-                        if (P.accumulate) v += out[off];
-                        out[off] = v;
-                    }
+            for (int j = 0; j < 4; ++j) { off[j] = (unsigned)(ob + outN[cl + j]); v[j] *= scale; }
+        }
+        const int live = (int)min(4u, Next - n);
+        for (int s = 0; s < n_epi; ++s) {
+            const int op = P.epi_op[s];
+            const float imm = P.epi_imm[s];
+            const float *src = (op == TE_MUL_LOAD || op == TE_ADD_LOAD) ? ptrs.in[P.epi_ptr[s]] : nullptr;
+            const int sb = P.epi_base[s];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                switch (op) {
+                case TE_NEG: v[j] = -v[j]; break;
+                case TE_EXP: v[j] = __expf(v[j]); break;
+                case TE_MULC: v[j] *= imm; break;
+                case TE_ADDC: v[j] += imm; break;
+                case TE_SQR: v[j] *= v[j]; break;
+                case TE_TANH: v[j] = own_tanh(v[j]); break;
+                case TE_MUL_LOAD: if (j < live) v[j] *= __ldg(src + (unsigned)(sb + (int)off[j])); break;
+                case TE_ADD_LOAD: if (j < live) v[j] += __ldg(src + (unsigned)(sb + (int)off[j])); break;
+                default: break;
                 }
             }
+        }
+        if (vec_ok) {
+            float4 *dst = reinterpret_cast<float4 *>(out + off[0]);
+            float4 r = make_float4(v[0], v[1], v[2], v[3]);
+            if (!partial && P.accumulate) { const float4 o = *dst; r.x += o.x; r.y += o.y; r.z += o.z; r.w += o.w; }
+            *dst = r;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (j < live) out[off[j]] = (!partial && P.accumulate) ? v[j] + out[off[j]] : v[j];
         }
     }
 }

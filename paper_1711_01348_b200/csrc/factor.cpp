@@ -510,6 +510,111 @@ static bool factor_kernel(Gen &g, Kernel &k, int root, int scale, bool allow_spl
     if (!F.changed) return false;
     if (scale >= 0) term = w.bin(I_MUL, term, scale);
 
+    // ---- fusion: an element-wise kernel around one contraction becomes that contraction's epilogue -------------
+    // What is left may be  h(S)  with h a chain of unary steps (and products with tensors laid out like the output)
+    // and S a sum of monomials of which one holds the result T of a contraction sum_k A[m, k] B[n, k] and all others
+    // are products of a factor over the row variables and a factor over the column variables.  Then S itself is a
+    // contraction: the factors of T's monomial scale A and B, every other monomial adds one summation index
+    // (A' = its row factor, B' = its column factor).  A' and B' are small pre-evaluated matrices, the finished sums
+    // go through h in registers, and T never exists in memory.
+    struct Fusion {
+        bool on = false;
+        int a_tensor = -1, b_tensor = -1;
+        uint32_t mmask = 0, nmask = 0;
+        int64_t cols = 0;
+        std::vector<int> op; std::vector<float> imm; std::vector<int> load;    // epilogue steps, innermost first
+    } fusion;
+    if (summed.size() == (size_t)g.kappa) {
+        std::vector<int> op; std::vector<float> imm; std::vector<int> lds;
+        int cur = term;
+        auto elementwise = [&](int i) {
+            if (w.inst[i].op != I_LOAD) return false;
+            const TadpLoad &L = w.loads[w.inst[i].load];
+            for (int v = 0; v < TADP_MAX_VARS; ++v) if (L.coef[v] != (v < g.n_outer ? prog.out_coef[v] : 0)) return false;
+            return L.ptr >= 0;
+        };
+        for (bool go = true; go && (int)op.size() < TADC_MAX_EPI;) {
+            const Inst in = w.inst[cur];
+            switch (in.op) {
+            case I_NEG: op.push_back(TE_NEG); imm.push_back(0); lds.push_back(-1); cur = in.a; break;
+            case I_EXP: op.push_back(TE_EXP); imm.push_back(0); lds.push_back(-1); cur = in.a; break;
+            case I_TANH: op.push_back(TE_TANH); imm.push_back(0); lds.push_back(-1); cur = in.a; break;
+            case I_SQR: op.push_back(TE_SQR); imm.push_back(0); lds.push_back(-1); cur = in.a; break;
+            case I_MULC: op.push_back(TE_MULC); imm.push_back(in.imm); lds.push_back(-1); cur = in.a; break;
+            case I_ADDC: op.push_back(TE_ADDC); imm.push_back(in.imm); lds.push_back(-1); cur = in.a; break;
+            case I_MUL:
+                if (elementwise(in.a) && !elementwise(in.b)) { op.push_back(TE_MUL_LOAD); imm.push_back(0); lds.push_back(w.inst[in.a].load); cur = in.b; }
+                else if (elementwise(in.b) && !elementwise(in.a)) { op.push_back(TE_MUL_LOAD); imm.push_back(0); lds.push_back(w.inst[in.b].load); cur = in.a; }
+                else go = false;
+                break;
+            default: go = false; break;
+            }
+        }
+        Poly S;
+        int t_group = -1, t_mono = -1, t_atom = -1, n_results = 0;
+        if (F.expand(cur, S) && S.size() >= 1 && S.size() <= 6) {
+            for (size_t mi = 0; mi < S.size(); ++mi)
+                for (int a : S[mi].atoms) {
+                    if (w.inst[a].op != I_LOAD) continue;
+                    const int ptr = w.loads[w.inst[a].load].ptr;
+                    if (ptr <= -1000) { ++n_results; t_group = -1000 - ptr; t_mono = (int)mi; t_atom = a; }
+                }
+        }
+        uint32_t outer_mask = 0;
+        for (int v = 0; v < g.n_outer; ++v) if (F.vext[v] > 1) outer_mask |= 1u << v;
+        bool ok = n_results == 1 && t_group >= 0;
+        if (ok) {
+            const Group &G = F.groups[t_group];
+            ok = G.reqs.size() == 1 && G.reqs[0].b_atoms.size() == 1 && F.is_plain_load(G.reqs[0].b_atoms[0]);
+            if (ok) {
+                fusion.mmask = w.inst[G.a_inst].deps & ~G.kmask;
+                fusion.nmask = w.inst[G.reqs[0].b_atoms[0]].deps & ~G.kmask;
+                ok = fusion.mmask && fusion.nmask && !(fusion.mmask & fusion.nmask) && ((fusion.mmask | fusion.nmask) & outer_mask) == outer_mask &&
+                     !((fusion.mmask | fusion.nmask) & ~outer_mask & ~0u) ;
+                // every other factor lives on the row side or on the column side
+                for (const Mono &m : S)
+                    for (int a : m.atoms) {
+                        if (a == t_atom) continue;
+                        const uint32_t d = w.inst[a].deps;
+                        if ((d & ~fusion.mmask) && (d & ~fusion.nmask)) ok = false;
+                    }
+            }
+        }
+        if (ok) {
+            Group &G = F.groups[t_group];
+            int64_t kext = 1;
+            for (int v = 0; v < TADP_MAX_VARS; ++v) if (G.kmask & (1u << v)) kext = mul_ck(kext, F.vext[v]);
+            fusion.cols = kext + (int64_t)S.size() - 1;
+            fusion.a_tensor = F.new_tensor(F.vars_of(fusion.mmask), fusion.cols);
+            fusion.b_tensor = F.new_tensor(F.vars_of(fusion.nmask), fusion.cols);
+            int64_t col = kext;
+            for (size_t mi = 0; mi < S.size(); ++mi) {
+                Mono ma, mb; ma.c = S[mi].c; mb.c = 1;
+                bool t_seen = false;
+                for (int a : S[mi].atoms) {
+                    if (a == t_atom && !t_seen) { t_seen = true; continue; }
+                    ((w.inst[a].deps & ~fusion.mmask) ? mb : ma).atoms.push_back(a);
+                }
+                Node na, nb;
+                na.kind = nb.kind = 0; na.tensor = fusion.a_tensor; nb.tensor = fusion.b_tensor;
+                if ((int)mi == t_mono) {
+                    ma.atoms.push_back(G.a_inst); mb.atoms.push_back(G.reqs[0].b_atoms[0]);
+                    na.col0 = nb.col0 = 0;
+                    na.dims = F.vars_of(fusion.mmask | G.kmask); nb.dims = F.vars_of(fusion.nmask | G.kmask);
+                } else {
+                    na.col0 = nb.col0 = col++;
+                    na.dims = F.vars_of(fusion.mmask); nb.dims = F.vars_of(fusion.nmask);
+                }
+                na.poly = Poly{ma}; nb.poly = Poly{mb};
+                F.nodes.push_back(na); F.nodes.push_back(nb);
+            }
+            G.reqs.clear();                          // the contraction itself is the kernel now
+            std::reverse(op.begin(), op.end()); std::reverse(imm.begin(), imm.end()); std::reverse(lds.begin(), lds.end());
+            fusion.op = op; fusion.imm = imm; fusion.load = lds;
+            fusion.on = true;
+        }
+    }
+
     // ---- layouts of the merged contractions ----
     const int slot0 = p.n_args + 1 + (int)p.stages.size();
     const int max_aux = (p.opt.saved_forward ? TADP_F_SLOT : TADP_MAX_PTRS) - slot0;
@@ -782,7 +887,39 @@ static bool factor_kernel(Gen &g, Kernel &k, int root, int scale, bool allow_spl
         pre.push_back(ak);
     }
 
-    // ---- the kernel itself: the rewritten term under the loops that are left ----
+    // ---- the kernel itself: the fused contraction, or the rewritten term under the loops that are left ----
+    if (fusion.on) {
+        System s;
+        const int nv = TADP_MAX_VARS + 1;
+        s.vars.assign(nv, AVar{1, false});
+        s.A.coef.assign(nv, 0); s.B.coef.assign(nv, 0); s.O.coef.assign(nv, 0);
+        const Tensor &TA = F.tensors[fusion.a_tensor], &TB = F.tensors[fusion.b_tensor];
+        s.A.ptr = slot_of[fusion.a_tensor]; s.A.limit = TA.elems;
+        s.B.ptr = slot_of[fusion.b_tensor]; s.B.limit = TB.elems;
+        for (size_t d = 0; d < TA.vars.size(); ++d) { s.vars[TA.vars[d]] = AVar{F.vext[TA.vars[d]], false}; s.A.coef[TA.vars[d]] = TA.stride[d]; }
+        for (size_t d = 0; d < TB.vars.size(); ++d) { s.vars[TB.vars[d]] = AVar{F.vext[TB.vars[d]], false}; s.B.coef[TB.vars[d]] = TB.stride[d]; }
+        s.vars[nv - 1] = AVar{fusion.cols, true};
+        s.A.coef[nv - 1] = 1; s.B.coef[nv - 1] = 1;
+        s.O.base = prog.out_base; s.O.limit = prog.out_limit;
+        for (int v = 0; v < g.n_outer; ++v) { s.O.coef[v] = prog.out_coef[v]; s.O.base += (int64_t)prog.out_coef[v] * F.vlo[v]; }
+        TadcProgram cp;
+        if (!emit_program(s, 1.f, prog.accumulate, false, false, cp, text)) return false;
+        cp.n_epi = (int32_t)fusion.op.size();
+        for (size_t e = 0; e < fusion.op.size(); ++e) {
+            cp.epi_op[e] = fusion.op[e]; cp.epi_imm[e] = fusion.imm[e];
+            if (fusion.load[e] >= 0) {
+                const TadpLoad &L = w.loads[fusion.load[e]];
+                cp.epi_ptr[e] = L.ptr; cp.epi_base[e] = to_i32((int64_t)L.base - prog.out_base);
+            }
+        }
+        k.contract = {cp};
+        k.vec = 0; k.vec_u = 0;
+        char line[96];
+        std::snprintf(line, sizeof line, "; the kernel is the contraction above with %d epilogue steps\n", cp.n_epi);
+        k.listing = text + line;
+        k.pre = pre;
+        return true;
+    }
     Gen g3(p, g.q);
     Translator tr(w, g3, slot_of);
     g3.n_outer = g.n_outer;

@@ -237,9 +237,12 @@ def test_kernel_stats_and_listing():
     e = W.FULL["cfg2"]()
     plan = Plan(e)
     fwd = plan.kernel_stats(-1)
-    # the sum over k is pushed inside the term: two small pre-evaluated tensors, one contraction, the kernel itself
-    assert fwd.outputs == 8192 * 8192 and fwd.n_launches == 4
-    assert "; factored" in plan.disassemble(-1) and "; contraction 8192 x 8192 x 32" in plan.disassemble(-1)
+    # the sum over k is pushed inside the term and the kernel is one contraction with exp(-.) as its epilogue: 32
+    # summation indices for a_ik b_jk plus one each for the terms that depend on i only and on i and j separately;
+    # before it, small kernels pre-evaluate those terms and the two operand matrices
+    assert fwd.outputs == 8192 * 8192 and fwd.n_launches == 9
+    listing = plan.disassemble(-1)
+    assert "; factored" in listing and "; contraction 8192 x 8192 x 34" in listing and "2 epilogue steps" in listing
     # forward: per (i,j,k) add, square, multiply, add, accumulate (5) + cube per (i,k) + neg, exp per (i,j)
     nij, nk = 8192.0 * 8192.0, 32.0
     assert fwd.alg_flops == pytest.approx(5 * nij * nk + 2 * 8192 * nk + 2 * nij, rel=1e-6)
