@@ -61,14 +61,39 @@ __device__ __forceinline__ Parts decode(const TadcGroup &G, unsigned idx)
 // the ranges): offset add, copy.  pre = rows[row of this thread] for the modes whose threads keep one row.
 template <int BR, int NT, bool CHECK>
 __device__ __forceinline__ void gather(float *smem, const float *__restrict__ src, const int2 *rows, const int2 *ktab,
-                                       const int2 pre, const int mode, const unsigned gext, const unsigned tid)
+                                       const int2 pre, const int mode, const unsigned gext, const unsigned tid, const unsigned klimit)
 {
-    // The copies carry no memory clobber (the group commit and wait do), and every table entry of a stage is
-    // read before the first copy is issued, so that the table reads overlap instead of each waiting its turn.
+    // The copies carry no memory clobber (the group commit and wait do), and the table entries of a batch of
+    // copies are read before the first of them is issued, so that the table reads overlap instead of each
+    // waiting its turn.  klimit: summation indices of this stage that the multiply-add loop will read.
     constexpr int LD = BR + 4;
+    constexpr bool REGULAR = NT % BR == 0 && (BR * BK) % NT == 0 && NT % (BR / 4) == 0 && NT % (4 * BK) == 0;
+    if constexpr (!REGULAR) {
+        // any number of threads: element e of the stage -> (row, summation index) by the mode's own order
+        const unsigned total = mode == TG_ROW16 ? (BR / 4) * BK : BR * BK;
+        for (unsigned e0 = tid; e0 < total; e0 += 4 * NT) {
+            unsigned off[4], dst[4]; bool live[4], use[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const unsigned e = e0 + j * NT;
+                unsigned rl, kl;
+                if (mode == TG_ROW16) { rl = (e % (BR / 4)) * 4; kl = e / (BR / 4); }
+                else if (mode == TG_ROW) { rl = e % BR; kl = e / BR; }
+                else { kl = e % BK; rl = e / BK; }
+                use[j] = e < total && kl < klimit;
+                const int2 r = rows[use[j] ? rl : 0], kt = ktab[use[j] ? kl : 0];
+                live[j] = !CHECK || (unsigned)(r.y + kt.y) < gext;
+                off[j] = live[j] ? (unsigned)(r.x + kt.x) : 0u;
+                dst[j] = kl * LD + rl;
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (use[j]) { if (mode == TG_ROW16) cp_async16(smem + dst[j], src + off[j], live[j]); else cp_async4(smem + dst[j], src + off[j], live[j]); }
+        }
+        return;
+    } else {
     if (mode == TG_ROW16) {
         constexpr unsigned CH = BR / 4, TOTAL = CH * BK, PER = (TOTAL + NT - 1) / NT, KSTEP = NT / CH;
-        static_assert(NT % CH == 0, "threads per stage row");
         const unsigned rl = (tid % CH) * 4, kl0 = tid / CH;
         if (TOTAL % NT != 0 && kl0 >= BK) return;
         unsigned off[PER]; bool live[PER];
@@ -79,10 +104,10 @@ __device__ __forceinline__ void gather(float *smem, const float *__restrict__ sr
             off[j] = live[j] ? (unsigned)(pre.x + kt.x) : 0u;
         }
 #pragma unroll
-        for (unsigned j = 0; j < PER; ++j) cp_async16(smem + (kl0 + KSTEP * j) * LD + rl, src + off[j], live[j]);
+        for (unsigned j = 0; j < PER; ++j)
+            if (kl0 + KSTEP * j < klimit) cp_async16(smem + (kl0 + KSTEP * j) * LD + rl, src + off[j], live[j]);
     } else if (mode == TG_ROW) {
         constexpr unsigned TOTAL = BR * BK, PER = TOTAL / NT, KSTEP = NT / BR;
-        static_assert(NT % BR == 0 && TOTAL % NT == 0, "threads per stage row");
         const unsigned rl = tid % BR, kl0 = tid / BR;
         unsigned off[PER]; bool live[PER];
 #pragma unroll
@@ -92,13 +117,14 @@ __device__ __forceinline__ void gather(float *smem, const float *__restrict__ sr
             off[j] = live[j] ? (unsigned)(pre.x + kt.x) : 0u;
         }
 #pragma unroll
-        for (unsigned j = 0; j < PER; ++j) cp_async4(smem + (kl0 + KSTEP * j) * LD + rl, src + off[j], live[j]);
+        for (unsigned j = 0; j < PER; ++j)
+            if (kl0 + KSTEP * j < klimit) cp_async4(smem + (kl0 + KSTEP * j) * LD + rl, src + off[j], live[j]);
     } else {
         // a warp copies 8 summation indices x 4 rows: full 32-byte sectors of a row-major operand, and the
         // 32 shared-memory words it writes (row stride BR + 4) fall into 32 different banks
         constexpr unsigned TOTAL = BR * BK, PER = TOTAL / NT, RSTEP = NT / BK;
-        static_assert(BK % 8 == 0 && NT % (4 * BK) == 0 && TOTAL % NT == 0, "copy pattern of the summation-index mode");
         const unsigned kl = (tid % 8) + 8 * ((tid / 32) % (BK / 8)), rl0 = (tid / 8) % 4 + 4 * (tid / (4 * BK));
+        if (kl >= klimit) return;
         const int2 kt = ktab[kl];
         unsigned off[PER]; bool live[PER];
 #pragma unroll
@@ -109,6 +135,7 @@ __device__ __forceinline__ void gather(float *smem, const float *__restrict__ sr
         }
 #pragma unroll
         for (unsigned j = 0; j < PER; ++j) cp_async4(smem + kl * LD + rl0 + RSTEP * j, src + off[j], live[j]);
+    }
     }
 }
 
@@ -151,7 +178,7 @@ struct Cfg {
 };
 
 template <int BM, int BN, int TM, int TN>
-__global__ void __launch_bounds__(Cfg<BM, BN, TM, TN>::NT, (TM * TN >= 64 ? 2 : 3))
+__global__ void __launch_bounds__(Cfg<BM, BN, TM, TN>::NT, (TM * TN >= 64 ? 2 : Cfg<BM, BN, TM, TN>::NT <= 160 ? 4 : 3))
 tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant__ TadpPointers ptrs, const unsigned tiles_m, const unsigned tiles_n)
 {
     using C = Cfg<BM, BN, TM, TN>;
@@ -214,7 +241,7 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
     const int modeA = P.modeA, modeB = P.modeB;
     // the row a thread keeps through all stages (modes with the lanes along the row index)
     const int2 preA = rowA[modeA == TG_ROW16 ? (tid % (BM / 4)) * 4 : tid % BM];
-    const int2 preB = rowB[modeB == TG_ROW16 ? (tid % (BN / 4)) * 4 : tid % BN];
+    const int2 preB = rowB[modeB == TG_ROW16 ? (tid % (BN / 4)) * 4 : tid % BN];      // (unused by tiles with irregular thread counts)
     // tiles inside the ranges and operands without a guard take the copy path without tests
     const bool plainA = !P.guardA && (tile_m + 1) * BM <= Mext, plainB = !P.guardB && (tile_n + 1) * BN <= Next;
     auto issue = [&](int kstage) {
@@ -222,22 +249,26 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
             float *as = stage_mem + (kstage % STAGES) * C::STAGE_FLOATS;
             float *bs = as + BK * LDA;
             const int slot = (kstage % (STAGES + 1)) * BK;
-            const bool full = kbeg + (unsigned)(kstage + 1) * BK <= kend;
-            if (plainA && full) gather<BM, NT, false>(as, A, rowA, ktabA + slot, preA, modeA, gextA, tid);
-            else gather<BM, NT, true>(as, A, rowA, ktabA + slot, preA, modeA, gextA, tid);
+            const unsigned left = kend - kbeg - (unsigned)kstage * BK;
+            const bool full = left >= BK;
+            const unsigned klimit = full ? BK : (left + KK_UNROLL - 1) / KK_UNROLL * KK_UNROLL;
+            if (plainA && full) gather<BM, NT, false>(as, A, rowA, ktabA + slot, preA, modeA, gextA, tid, klimit);
+            else gather<BM, NT, true>(as, A, rowA, ktabA + slot, preA, modeA, gextA, tid, klimit);
             if (onesB) {}
-            else if (plainB && full) gather<BN, NT, false>(bs, B, rowB, ktabB + slot, preB, modeB, gextB, tid);
-            else gather<BN, NT, true>(bs, B, rowB, ktabB + slot, preB, modeB, gextB, tid);
+            else if (plainB && full) gather<BN, NT, false>(bs, B, rowB, ktabB + slot, preB, modeB, gextB, tid, klimit);
+            else gather<BN, NT, true>(bs, B, rowB, ktabB + slot, preB, modeB, gextB, tid, klimit);
         }
         cp_async_commit();
     };
     for (int s = 0; s < STAGES - 1; ++s) issue(s);
 
     // a warp covers 8 thread columns x 4 thread rows: its 128-bit reads of a stage touch 128 consecutive bytes
-    // of the B tile and 64 of the A tile, one shared-memory wavefront each
-    constexpr unsigned WARPS_N = (BN / TN) / 8;
+    // of the B tile and 64 of the A tile, one shared-memory wavefront each (tiles whose thread columns do not
+    // come in eights number their threads row by row)
+    constexpr unsigned TCOLS = BN / TN;
     const unsigned warp = tid / 32, lane = tid % 32;
-    const int tx = (int)((warp % WARPS_N) * 8 + lane % 8), ty = (int)((warp / WARPS_N) * 4 + lane / 8);
+    const int tx = TCOLS % 8 == 0 ? (int)((warp % (TCOLS / 8 ? TCOLS / 8 : 1)) * 8 + lane % 8) : (int)(tid % TCOLS);
+    const int ty = TCOLS % 8 == 0 ? (int)((warp / (TCOLS / 8 ? TCOLS / 8 : 1)) * 4 + lane / 8) : (int)(tid / TCOLS);
     float acc[TM][TN];
 #pragma unroll
     for (int i = 0; i < TM; ++i)
@@ -339,19 +370,45 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
             const float imm = P.epi_imm[s];
             const float *src = (op == TE_MUL_LOAD || op == TE_ADD_LOAD) ? ptrs.in[P.epi_ptr[s]] : nullptr;
             const int sb = P.epi_base[s];
+            switch (op) {
+            case TE_NEG:
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                switch (op) {
-                case TE_NEG: v[j] = -v[j]; break;
-                case TE_EXP: v[j] = __expf(v[j]); break;
-                case TE_MULC: v[j] *= imm; break;
-                case TE_ADDC: v[j] += imm; break;
-                case TE_SQR: v[j] *= v[j]; break;
-                case TE_TANH: v[j] = own_tanh(v[j]); break;
-                case TE_MUL_LOAD: if (j < live) v[j] *= __ldg(src + (unsigned)(sb + (int)off[j])); break;
-                case TE_ADD_LOAD: if (j < live) v[j] += __ldg(src + (unsigned)(sb + (int)off[j])); break;
-                default: break;
+                for (int j = 0; j < 4; ++j) v[j] = -v[j];
+                break;
+            case TE_EXP:
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[j] = __expf(v[j]);
+                break;
+            case TE_MULC:
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[j] *= imm;
+                break;
+            case TE_ADDC:
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[j] += imm;
+                break;
+            case TE_SQR:
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[j] *= v[j];
+                break;
+            case TE_TANH:
+#pragma unroll
+                for (int j = 0; j < 4; ++j) v[j] = own_tanh(v[j]);
+                break;
+            case TE_MUL_LOAD:
+                if (vec_ok && ((sb & 3) == 0)) {
+                    const float4 w4 = __ldg(reinterpret_cast<const float4 *>(src + (unsigned)(sb + (int)off[0])));
+                    v[0] *= w4.x; v[1] *= w4.y; v[2] *= w4.z; v[3] *= w4.w;
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) if (j < live) v[j] *= __ldg(src + (unsigned)(sb + (int)off[j]));
                 }
+                break;
+            case TE_ADD_LOAD:
+#pragma unroll
+                for (int j = 0; j < 4; ++j) if (j < live) v[j] += __ldg(src + (unsigned)(sb + (int)off[j]));
+                break;
+            default: break;
             }
         }
         if (vec_ok) {
@@ -388,6 +445,48 @@ tad_contract_reduce(const __grid_constant__ TadcProgram P, const __grid_constant
     }
 }
 
+// Plain summation of one operand (contraction with a tensor of ones and a single output column):
+//     out[m] (+)= scale * sum_k A[row(m) + k * stride]
+// One warp per output; its lanes walk the summation index (128-bit loads when that index is contiguous
+// and aligned), then a fixed-order shuffle tree.  Bound by HBM: every element of A is read once.
+__global__ void __launch_bounds__(256)
+tad_rowsum_kernel(const __grid_constant__ TadcProgram P, const __grid_constant__ TadpPointers ptrs)
+{
+    const unsigned lane = threadIdx.x & 31u;
+    const unsigned warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, n_warps = (gridDim.x * blockDim.x) >> 5;
+    const float *__restrict__ A = ptrs.in[P.ptrA];
+    const unsigned K = (unsigned)P.K.extent;
+    const int ks = P.K.n_digits ? P.K.sA[0] : 0;
+    for (unsigned m = warp; m < (unsigned)P.M.extent; m += n_warps) {
+        const Parts p = decode(P.M, m);
+        const int base = P.baseA + p.a;
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+        if (ks == 1 && ((base & 3) == 0) && ((reinterpret_cast<uintptr_t>(A) & 15u) == 0)) {
+            const float4 *row = reinterpret_cast<const float4 *>(A + (unsigned)base);
+            const unsigned K4 = K / 4;
+            unsigned k = lane;
+            for (; k + 96 < K4; k += 128) {
+                const float4 a = __ldg(row + k), b = __ldg(row + k + 32), c = __ldg(row + k + 64), d = __ldg(row + k + 96);
+                s0 += (a.x + a.y) + (a.z + a.w); s1 += (b.x + b.y) + (b.z + b.w);
+                s2 += (c.x + c.y) + (c.z + c.w); s3 += (d.x + d.y) + (d.z + d.w);
+            }
+            for (; k < K4; k += 32) { const float4 a = __ldg(row + k); s0 += (a.x + a.y) + (a.z + a.w); }
+            for (unsigned t = K4 * 4 + lane; t < K; t += 32) s1 += __ldg(A + (unsigned)(base + (int)t));
+        } else {
+            for (unsigned k = lane; k < K; k += 32) s0 += __ldg(A + (unsigned)(base + (int)k * ks));
+        }
+        float s = (s0 + s1) + (s2 + s3);
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+        if (lane == 0) {
+            const unsigned off = (unsigned)(P.baseO + p.o);
+            float v = s * P.scale;
+            if (P.accumulate) v += ptrs.out[off];
+            ptrs.out[off] = v;
+        }
+    }
+}
+
 template <int BM, int BN, int TM, int TN>
 cudaError_t launch_shape(const TadcProgram &P, const TadpPointers &ptrs, cudaStream_t stream)
 {
@@ -413,7 +512,13 @@ cudaError_t launch_shape(const TadcProgram &P, const TadpPointers &ptrs, cudaStr
 cudaError_t tad_launch_contract(const TadcProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream)
 {
     if (P.M.extent <= 0 || P.N.extent <= 0 || P.Z.extent <= 0) return cudaSuccess;
-    cudaError_t e = P.shape == 1 ? launch_shape<128, 32, 4, 4>(P, ptrs, stream)
+    if (P.shape == 4) {
+        const unsigned warps = (unsigned)P.M.extent;
+        const unsigned blocks = std::min((warps + 7u) / 8u, sms * 16u);
+        tad_rowsum_kernel<<<blocks, 256, 0, stream>>>(P, ptrs);
+        return cudaGetLastError();
+    }
+    cudaError_t e = P.shape == 3 ? launch_shape<128, 36, 8, 4>(P, ptrs, stream)
                   : P.shape == 2 ? launch_shape<128, 64, 8, 4>(P, ptrs, stream) : launch_shape<128, 128, 8, 8>(P, ptrs, stream);
     if (e != cudaSuccess) return e;
     if (P.ksplit > 1) {

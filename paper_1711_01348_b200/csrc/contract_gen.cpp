@@ -126,8 +126,8 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     P.guardB = gb ? 1 : 0; P.guardB_c0 = gb ? fit(gb->c0) : 0; P.guardB_ext = gb ? fit(gb->ext) : 1;
     P.scale = scale; P.accumulate = accumulate;
     // tile shape: narrow column tiles for narrow outputs
-    P.shape = P.N.extent <= 32 ? 1 : P.N.extent <= 64 ? 2 : 0;
-    const int64_t BM = 128, BN = P.shape == 1 ? 32 : P.shape == 2 ? 64 : 128;
+    P.shape = P.N.extent <= 36 ? 3 : P.N.extent <= 64 ? 2 : 0;
+    const int64_t BM = 128, BN = P.shape == 3 ? 36 : P.shape == 2 ? 64 : 128;
     const int64_t tiles_m = (P.M.extent + BM - 1) / BM, tiles_n = (P.N.extent + BN - 1) / BN;
     const double fill = (double)P.M.extent * P.N.extent / ((double)tiles_m * BM * tiles_n * BN);
     if (strict_fill && fill < 0.15) return false;          // mostly empty tiles: the interpreter's schedules do better
@@ -182,7 +182,7 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     if (allow_split && blocks < 222 && kstages >= 16) {
         // the number of chunks that fills whole waves of resident blocks best (two blocks per SM), every
         // chunk at least eight stages long; fewer chunks win ties (less partial-sum traffic)
-        const int64_t wave = P.shape == 0 ? 296 : 444;
+        const int64_t wave = P.shape == 0 ? 296 : P.shape == 2 ? 444 : 592;
         const int64_t cells = (int64_t)P.M.extent * P.N.extent * P.Z.extent;
         double best = 0;
         for (int64_t s = 1; s <= std::min<int64_t>(kstages / 8, 256); ++s) {
@@ -192,6 +192,7 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
             if (eff > best + 0.02) { best = eff; split = s; }
         }
     }
+    if (s.B.ptr < 0 && P.N.extent == 1 && P.Z.extent == 1 && P.K.n_digits <= 1 && !P.guardA && P.M.extent >= 1024) { P.shape = 4; split = 1; }
     split = std::max<int64_t>(1, split);
     const int64_t per = ((kstages + split - 1) / split) * TADC_BK;
     P.kchunk = fit(std::max<int64_t>(per, TADC_BK));
@@ -208,7 +209,7 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     };
     std::snprintf(line, sizeof line, "; contraction %d x %d x %d (batch %d): A=ptr %d mode %d guard %d, B=ptr %d mode %d guard %d, tile %s, ksplit %d x %d, vec4 %d, scale %g, accumulate %d\n",
                   P.M.extent, P.N.extent, P.K.extent, P.Z.extent, P.ptrA, P.modeA, P.guardA, P.ptrB, P.modeB, P.guardB,
-                  P.shape == 1 ? "128x32" : P.shape == 2 ? "128x64" : "128x128", P.ksplit, P.kchunk, P.out_vec4, (double)P.scale, P.accumulate);
+                  P.shape == 4 ? "row sums" : P.shape == 3 ? "128x36" : P.shape == 2 ? "128x64" : "128x128", P.ksplit, P.kchunk, P.out_vec4, (double)P.scale, P.accumulate);
     text += line;
     text += group_text("m", P.M) + group_text("n", P.N) + group_text("k", P.K) + group_text("z", P.Z);
     return true;
