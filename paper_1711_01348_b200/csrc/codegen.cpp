@@ -794,8 +794,11 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
         // compact index of an output inside a plane of partial sums: row-major over the outer box
         int64_t cells = 1;
         for (int v = g.n_outer - 1; v >= 0; --v) { prog.part_coef[v] = to_i32(cells); cells = mul_ck(cells, prog.outer_ext[v]); }
-        // splitting costs a pass over zsplit planes: only when the outputs are too few to fill the GPU
-        if (items_for(pick) < target_warps / 2 && cells <= (1 << 22)) {
+        // splitting costs a pass over zsplit planes: only when the outputs are too few to fill the GPU and every
+        // output has enough terms to share out (a few dozen terms per output are summed faster than split)
+        double terms_per_output = 1;
+        for (int l = 0; l < g.kappa; ++l) terms_per_output *= (double)std::max<int64_t>(1, g.vars[g.n_outer + g.zorder[l]].ext);
+        if (items_for(pick) < target_warps / 2 && cells <= (1 << 22) && terms_per_output >= 256) {
             TadpLoop &L0 = prog.loops[em.code[zbegin[0]].a];
             // shares of the outermost loop first; when that loop is too short, the next one is divided too
             // (share number s = s0 * S1 + s1)
@@ -827,6 +830,9 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
                 if (S0 > 1) { L0.is_split = 1; L0.split_n = (int32_t)S0; L0.split_div = (int32_t)S1; }
                 if (S1 > 1) { L1->is_split = 1; L1->split_n = (int32_t)S1; L1->split_div = 1; }
             }
+        } else if (items_for(pick) < target_warps / 2) {
+            // few outputs with short summations: the narrowest shape that fills the GPU (more warps, fewer values each)
+            for (const Shape &sh : shapes) { pick = sh; if (items_for(sh) >= target_warps / 2) break; }
         }
     } else {
         // element-wise kernel: the widest shape that still leaves enough warps

@@ -130,7 +130,8 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     const int64_t BM = 128, BN = P.shape == 3 ? 36 : P.shape == 2 ? 64 : 128;
     const int64_t tiles_m = (P.M.extent + BM - 1) / BM, tiles_n = (P.N.extent + BN - 1) / BN;
     const double fill = (double)P.M.extent * P.N.extent / ((double)tiles_m * BM * tiles_n * BN);
-    if (strict_fill && fill < 0.15) return false;          // mostly empty tiles: the interpreter's schedules do better
+    const bool row_sums = s.B.ptr < 0 && P.N.extent == 1 && P.Z.extent == 1 && P.K.n_digits <= 1 && !P.guardA && P.M.extent >= 1024;
+    if (!row_sums && fill < (strict_fill ? 0.15 : 0.05)) return false;    // mostly empty tiles: the interpreter's schedules do better
     // gather modes: the one whose warp-wide copy touches fewer 128-byte lines (lanes along the row index:
     // 32 rows at one summation index; lanes along the summation index: 2 rows x 16 indices)
     auto mode_of = [&](const std::vector<Digit> &rows, bool second, const AGuard *gd, int64_t base) {
@@ -192,7 +193,7 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
             if (eff > best + 0.02) { best = eff; split = s; }
         }
     }
-    if (s.B.ptr < 0 && P.N.extent == 1 && P.Z.extent == 1 && P.K.n_digits <= 1 && !P.guardA && P.M.extent >= 1024) { P.shape = 4; split = 1; }
+    if (row_sums) { P.shape = 4; split = 1; }
     split = std::max<int64_t>(1, split);
     const int64_t per = ((kstages + split - 1) / split) * TADC_BK;
     P.kchunk = fit(std::max<int64_t>(per, TADC_BK));

@@ -46,6 +46,7 @@ struct Node {                         // a kernel that fills (part of) a tensor
     std::vector<int> dims, sums;      // interpreter: output variables (beside the block's own), summed variables
     Poly poly;                        // interpreter: the summand
     int group = -1;                   // contraction: which group
+    int table_inst = -1, table_load = -1;   // kind 2: a function of one index expression, evaluated over that argument's elements
 };
 
 struct Request { std::vector<int> b_atoms; uint32_t nmask = 0; int load_id = -1; int64_t col0 = 0, width = 1; };
@@ -69,6 +70,9 @@ struct Factorizer {
     std::map<int, int> load_tensor;                   // load id -> tensor (auxiliary loads)
     std::map<int, int> memo;
     bool changed = false;
+    bool allow_sums = true;                           // false: only function tables (kernels with guards)
+    int n_outer_vars = 0;
+    std::map<int, int> table_memo;                    // instance -> load of its table
 
     Factorizer(Gen &gen, Kernel &kern) : w(gen), k(kern), nv0((int)gen.vars.size()), vlo(TADP_MAX_VARS, 0), vext(TADP_MAX_VARS, 1), can_sum(TADP_MAX_VARS, false) {}
 
@@ -279,6 +283,9 @@ struct Factorizer {
                 bool taken = false;
                 for (int a : best_s) { if (a == big && !taken) { taken = true; continue; } rest.push_back(a); }
                 if (!rest.empty() && space(deps_of(rest)) > SMALL_SPACE && !(rest.size() == 1 && is_plain_load(rest[0]))) return -1;
+                // the streamed operand must bring enough rows of its own to fill tiles (variables that the second
+                // operand reads too only number independent contractions)
+                if (space(w.inst[big].deps & ~best_k & ~deps_of(rest)) < 64) return -1;
                 // every summed variable must be read by the streamed operand or the second one
                 t_inst = request(big, best_k, rest);
             }
@@ -345,6 +352,63 @@ struct Factorizer {
     }
     uint32_t deps_of_poly(const Poly &p) const { uint32_t d = 0; for (const Mono &m : p) d |= deps_of(m.atoms); return d; }
 
+    // ---- function tables ------------------------------------------------------------------------
+    // An expression whose only leaf is one index expression of an argument (exp x[i + j], 1 - tanh^2 x[2i + 3j],
+    // sin x[...]) takes as many distinct values as the argument has elements.  When the kernel would evaluate it
+    // far more often than that, it is evaluated once per element of the argument into an auxiliary tensor of
+    // the argument's shape, and the kernel reads that tensor through the same index expression.
+    // returns the load id if instance i is such an expression (no sums, one load), else -1; cost: its operations
+    int single_load(int i, double &cost, bool &transcendental)
+    {
+        const Inst &in = w.inst[i];
+        switch (in.op) {
+        case I_CONST: return -2;
+        case I_LOAD: return w.loads[in.load].ptr >= 0 ? in.load : -1;
+        case I_SUM: return -1;
+        default: break;
+        }
+        if (in.op == I_EXP || in.op == I_LOG || in.op == I_SIN || in.op == I_COS || in.op == I_TANH || in.op == I_SINH || in.op == I_COSH ||
+            in.op == I_DIV || (in.op == I_POWI && (in.ipow < 0 || in.ipow > 4))) { transcendental = true; cost += 8; }
+        else cost += 1;
+        const int a = single_load(in.a, cost, transcendental);
+        if (a == -1) return -1;
+        if (in.b < 0) return a;
+        const int b = single_load(in.b, cost, transcendental);
+        if (b == -1) return -1;
+        if (a == -2) return b;
+        if (b == -2) return a;
+        return a == b ? a : -1;
+    }
+    int try_table(int i)
+    {
+        auto it = table_memo.find(i);
+        if (it != table_memo.end()) return it->second;
+        double cost = 0; bool tr = false;
+        const int ld = single_load(i, cost, tr);
+        if (ld < 0 || !tr) return -1;
+        const TadpLoad L = w.loads[ld];
+        // how often the kernel evaluates it: once per binding of its variables, and a value inside a loop is
+        // evaluated again for every output that runs the loop
+        uint32_t reach = w.inst[i].deps;
+        if (reach >> n_outer_vars) reach |= (1u << n_outer_vars) - 1u;
+        if (L.limit <= 0 || (double)L.limit * 8.0 > space(reach) || L.limit > (1 << 26)) return -1;
+        Tensor T; T.cols = 1; T.elems = L.limit;
+        tensors.push_back(T);
+        const int t = (int)tensors.size() - 1;
+        Node n; n.kind = 2; n.tensor = t; n.table_inst = i; n.table_load = ld;
+        nodes.push_back(n);
+        TadpLoad N = L;
+        N.ptr = -1 - t;
+        w.loads.push_back(N);
+        const int id = (int)w.loads.size() - 1;
+        load_tensor[id] = t;
+        Inst li; li.op = I_LOAD; li.load = id; li.deps = w.inst[i].deps; li.adeps = w.inst[i].adeps;
+        const int r = w.intern(li);
+        table_memo[i] = r;
+        changed = true;
+        return r;
+    }
+
     // rewrites the sums below instance i; returns the (possibly new) instance
     int rewrite(int i)
     {
@@ -352,6 +416,10 @@ struct Factorizer {
         if (it != memo.end()) return it->second;
         const Inst in = w.inst[i];
         int r = i;
+        if (in.op != I_CONST && in.op != I_LOAD && in.op != I_SUM) {
+            const int tbl = try_table(i);
+            if (tbl >= 0) { memo[i] = tbl; return tbl; }
+        }
         if (in.op == I_SUM) {
             std::vector<int> vars{in.var};
             int body = in.a;
@@ -365,7 +433,7 @@ struct Factorizer {
                 cur = s.a;
             }
             const int nb = rewrite(body);
-            const int solved = solve(vars, nb);
+            const int solved = allow_sums ? solve(vars, nb) : -1;
             if (solved >= 0) r = solved;
             else if (nb != body) r = wrap_sums(nb, vars);
         } else if (in.op != I_CONST && in.op != I_LOAD) {
@@ -392,6 +460,7 @@ struct Translator {
     std::vector<int> var_map;
     const std::vector<int> &slot_of_tensor;      // auxiliary tensor -> pointer slot
     std::map<int, int> memo;
+    int flat_load = -1;                          // this load is read at element index = variable 0 (function tables)
     Translator(Gen &s, Gen &d, const std::vector<int> &slots) : src(s), dst(d), var_map(TADP_MAX_VARS, -1), slot_of_tensor(slots) {}
     int run(int i)
     {
@@ -407,7 +476,8 @@ struct Translator {
             N.ptr = L.ptr < 0 ? slot_of_tensor[-1 - L.ptr] : L.ptr;
             N.base = L.base; N.limit = L.limit;
             uint32_t deps = 0;
-            for (int v = 0; v < TADP_MAX_VARS; ++v) {
+            if (in.load == flat_load) { N.base = 0; N.coef[0] = 1; deps = 1u; }
+            else for (int v = 0; v < TADP_MAX_VARS; ++v) {
                 if (!L.coef[v]) continue;
                 if (var_map[v] < 0) throw BadExpr("internal: variable outside the kernel");
                 N.coef[var_map[v]] += L.coef[v];
@@ -452,9 +522,11 @@ static bool factor_kernel(Gen &g, Kernel &k, int root, int scale, bool allow_spl
 {
     tad_plan &p = g.p;
     // kernels with guards own elements without any term; the auxiliary kernels would evaluate index expressions there
-    if (p.opt.debug_bounds || root < 0 || !guards.empty()) return false;
+    if (p.opt.debug_bounds || root < 0) return false;
     Gen w = g;                                    // the pass works on a copy: the caller's instances keep their meaning
     Factorizer F(w, k);
+    F.allow_sums = guards.empty();
+    F.n_outer_vars = g.n_outer;
     const TadpProgram &prog = k.prog;
     for (int v = 0; v < g.n_outer; ++v) { F.vlo[v] = prog.outer_lo[v]; F.vext[v] = prog.outer_ext[v]; }
     // kernel-coordinate loops with fixed ranges that no other loop's bounds read can be summed away
@@ -502,13 +574,14 @@ static bool factor_kernel(Gen &g, Kernel &k, int root, int scale, bool allow_spl
     {
         std::vector<int> cand;
         for (int l = g.kappa - 1; l >= 0; --l) if (F.can_sum[zvars[l]]) cand.push_back(zvars[l]);
-        if (!cand.empty()) {
+        if (!cand.empty() && F.allow_sums) {
             const int solved = F.solve(cand, term);
             if (solved >= 0) { term = solved; summed = cand; }
         }
     }
+    int scale_r = scale >= 0 ? F.rewrite(scale) : -1;
     if (!F.changed) return false;
-    if (scale >= 0) term = w.bin(I_MUL, term, scale);
+    if (scale_r >= 0) term = w.bin(I_MUL, term, scale_r);
 
     // ---- fusion: an element-wise kernel around one contraction becomes that contraction's epilogue -------------
     // What is left may be  h(S)  with h a chain of unary steps (and products with tensors laid out like the output)
@@ -606,7 +679,23 @@ static bool factor_kernel(Gen &g, Kernel &k, int root, int scale, bool allow_spl
                     na.dims = F.vars_of(fusion.mmask); nb.dims = F.vars_of(fusion.nmask);
                 }
                 na.poly = Poly{ma}; nb.poly = Poly{mb};
-                F.nodes.push_back(na); F.nodes.push_back(nb);
+                // a factor that is nothing but a small pre-evaluated sum: its kernel writes the column itself
+                auto redirect = [&](Node &col, const Mono &m, int tensor) {
+                    if (m.atoms.size() != 1 || m.c != 1.0 || w.inst[m.atoms[0]].op != I_LOAD) return false;
+                    auto it = F.load_tensor.find(w.inst[m.atoms[0]].load);
+                    if (it == F.load_tensor.end()) return false;
+                    int writer = -1, n_writers = 0;
+                    for (size_t q = 0; q < F.nodes.size(); ++q) if (F.nodes[q].tensor == it->second) { writer = (int)q; ++n_writers; }
+                    if (n_writers != 1 || F.nodes[writer].kind != 0 || F.nodes[writer].dims != col.dims) return false;
+                    // no other reader of that tensor in S
+                    int readers = 0;
+                    for (const Mono &o : S) for (int a : o.atoms) if (a == m.atoms[0]) ++readers;
+                    if (readers != 1) return false;
+                    F.nodes[writer].tensor = tensor; F.nodes[writer].col0 = col.col0;
+                    return true;
+                };
+                if ((int)mi == t_mono || !redirect(na, ma, fusion.a_tensor)) F.nodes.push_back(na);
+                if ((int)mi == t_mono || !redirect(nb, mb, fusion.b_tensor)) F.nodes.push_back(nb);
             }
             G.reqs.clear();                          // the contraction itself is the kernel now
             std::reverse(op.begin(), op.end()); std::reverse(imm.begin(), imm.end()); std::reverse(lds.begin(), lds.end());
@@ -736,7 +825,8 @@ static bool factor_kernel(Gen &g, Kernel &k, int root, int scale, bool allow_spl
     std::vector<std::set<int>> node_reads(F.nodes.size());
     for (size_t n = 0; n < F.nodes.size(); ++n) {
         const Node &N = F.nodes[n];
-        if (N.kind == 0) { for (const Mono &m : N.poly) for (int a : m.atoms) reads_of_inst(a, node_reads[n]); }
+        if (N.kind == 2) {}
+        else if (N.kind == 0) { for (const Mono &m : N.poly) for (int a : m.atoms) reads_of_inst(a, node_reads[n]); }
         else {
             const Group &G = F.groups[N.group];
             reads_of_inst(G.a_inst, node_reads[n]);
@@ -767,7 +857,21 @@ static bool factor_kernel(Gen &g, Kernel &k, int root, int scale, bool allow_spl
         std::memset(&ak.prog, 0, sizeof ak.prog);
         ak.out_arg = -1; ak.access = -1; ak.out_aux = N.tensor;
         const Tensor &T = F.tensors[N.tensor];
-        if (N.kind == 0) {
+        if (N.kind == 2) {
+            // one output per element of the argument: the expression with its load read at the flat element index
+            Gen g2(p, -1);
+            Translator tr(w, g2, slot_of);
+            g2.n_outer = 1; g2.kappa = 0;
+            g2.new_var(0, T.elems);
+            tr.flat_load = N.table_load;
+            TadpProgram &ap = ak.prog;
+            ap.outer_lo[0] = 0; ap.outer_ext[0] = to_i32(T.elems); ap.out_coef[0] = 1;
+            ap.out_base = 0; ap.out_limit = to_i32(T.elems); ap.accumulate = 0; ap.write_only_live = 0;
+            const int root2 = tr.run(N.table_inst);
+            g2.lane_var = 0;
+            emit_plain_kernel(g2, ak, root2, {}, {}, {}, false);
+            text += "; function table -> tensor " + std::to_string(N.tensor) + "\n" + ak.listing;
+        } else if (N.kind == 0) {
             Gen g2(p, -1);
             Translator tr(w, g2, slot_of);
             g2.n_outer = (int)N.dims.size(); g2.kappa = 0;
