@@ -555,6 +555,83 @@ int body_fetch_kind(const TadpLoad &L, int ta, int ub)
     return BF_EACH;
 }
 
+// A program without loops and temporaries whose pending values never exceed two becomes an element-wise program
+// (ew.h); a thread owns four consecutive values of the lane variable.
+bool try_elementwise(Gen &g, Kernel &k, const Emitter &em)
+{
+    const TadpProgram &prog = k.prog;
+    if (g.kappa != 0 || g.p.opt.debug_bounds || prog.n_guards || prog.write_only_live) return false;
+    if (g.lane_var < 0 || g.lane_var >= g.n_outer) return false;
+    if ((int)g.loads.size() > TADE_MAX_LOADS) return false;
+    const std::vector<TadpInsn> &code = em.code;
+    const int n = (int)code.size();
+    if (n < 3 || (code[n - 1].handler >> 3) != P_END) return false;
+    const int term_op = code[n - 2].handler >> 3;
+    if (term_op != P_ACC && term_op != P_MACC) return false;
+    std::vector<TadeStep> steps;
+    auto push_step = [&](int op, int a = 0, int b = 0, float imm = 0.f) { TadeStep s{}; s.op = (uint8_t)op; s.a = (int16_t)a; s.b = (uint8_t)b; s.imm = imm; steps.push_back(s); };
+    int vd = 0;                                  // pending values: 0, 1 (X) or 2 (Y below X)
+    for (int w = 0; w < n - 2; ++w) {
+        const TadpInsn &in = code[w];
+        const int op = in.handler >> 3;
+        float imm; std::memcpy(&imm, &in.imm, 4);
+        switch (op) {
+        case P_LOAD: case P_CONST:
+            if (vd == 2) return false;
+            if (vd == 1) push_step(E_PUSH);
+            if (op == P_LOAD) push_step(E_LD, in.a, 0); else push_step(E_CONST, 0, 0, imm);
+            ++vd;
+            break;
+        case P_LDADD: if (vd < 1) return false; push_step(E_LD, in.a, 1); break;
+        case P_LDMUL: if (vd < 1) return false; push_step(E_LD, in.a, 2); break;
+        case P_LDADDSQ: if (vd < 1) return false; push_step(E_LD, in.a, 3); break;
+        case P_NEG: if (vd < 1) return false; push_step(E_NEG); break;
+        case P_SQR: if (vd < 1) return false; push_step(E_SQR); break;
+        case P_CUBE: if (vd < 1) return false; push_step(E_CUBE); break;
+        case P_MULC: if (vd < 1) return false; push_step(E_MULC, 0, 0, imm); break;
+        case P_ADDC: if (vd < 1) return false; push_step(E_ADDC, 0, 0, imm); break;
+        case P_FN: if (vd < 1) return false; push_step(E_FN, in.imm, in.b); break;
+        case P_ADD: case P_SUB: case P_MUL: case P_DIV:
+            if (vd != 2) return false;
+            push_step(op == P_ADD ? E_ADDY : op == P_SUB ? E_SUBY : op == P_MUL ? E_MULY : E_DIVY);
+            vd = 1;
+            break;
+        default: return false;
+        }
+    }
+    if (term_op == P_MACC) { if (vd != 2) return false; push_step(E_MULY); }
+    else if (vd != 1) return false;
+    if ((int)steps.size() > TADE_MAX_STEPS) return false;
+    TadeProgram E{};
+    E.n_outer = g.n_outer; E.lane_var = g.lane_var;
+    for (int v = 0; v < g.n_outer; ++v) {
+        E.outer_lo[v] = prog.outer_lo[v]; E.outer_ext[v] = prog.outer_ext[v]; E.out_coef[v] = prog.out_coef[v];
+        // n / d = (n * mul) >> (31 + s) for n < 2^31 with s = ceil(log2 d), mul = floor(2^(31 + s) / d) + 1
+        const uint64_t d = (uint64_t)std::max(1, prog.outer_ext[v]);
+        int s = 0; while ((uint64_t(1) << s) < d) ++s;
+        E.div_mul[v] = (uint32_t)(((uint64_t(1) << (31 + s)) / d) + 1);
+        E.div_shift[v] = 31 + s;
+    }
+    E.out_base = prog.out_base; E.out_limit = prog.out_limit; E.accumulate = prog.accumulate;
+    E.n_loads = (int32_t)g.loads.size();
+    for (size_t i = 0; i < g.loads.size(); ++i) E.loads[i] = g.loads[i];
+    E.n_steps = (int32_t)steps.size();
+    std::copy(steps.begin(), steps.end(), E.steps);
+    k.ew = {E};
+    k.vec = 0; k.vec_u = 0;
+    char line[200];
+    std::snprintf(line, sizeof line, "; element-wise program: %d steps, %d loads, rows of %d along variable %d\n", E.n_steps, E.n_loads,
+                  E.outer_ext[E.lane_var], E.lane_var);
+    k.listing = line + em.listing();
+    for (int i = 0; i < E.n_loads; ++i) {
+        std::string t;
+        for (int v = 0; v < g.n_outer; ++v) t += " " + std::to_string(E.loads[i].coef[v]);
+        std::snprintf(line, sizeof line, "; load %d ptr=%d base=%d coef=[%s ]\n", i, E.loads[i].ptr, E.loads[i].base, t.c_str());
+        k.listing += line;
+    }
+    return true;
+}
+
 // shared tail: choose temps, emit, fill the program
 void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<TadpRow>> &lower,
                  const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards, bool allow_split = false,
@@ -670,6 +747,7 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     if (scale >= 0) { em.expr(scale); em.emit(P_SCALE, 0, 0, 0, -1); }
     em.emit(P_END);
     if (em.depth != 0) throw BadExpr("internal: unbalanced operand stack");
+    if (n_temps == 0 && try_elementwise(g, k, em)) return;
     // rows
     std::vector<TadpRow> rows;
     for (TadpLoop &L : em.loops) {
@@ -920,7 +998,7 @@ void emit_plain_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vecto
 static void account(tad_plan &p, Kernel &k)
 {
     std::function<void(const Kernel &)> walk = [&](const Kernel &x) {
-        if (x.contract.empty() && x.prog.zsplit > 1)
+        if (x.ew.empty() && x.contract.empty() && x.prog.zsplit > 1)
             p.partial_bytes = std::max(p.partial_bytes, (size_t(x.prog.zsplit) + 1) * size_t(x.prog.part_limit) * 4);
         for (const TadcProgram &cp : x.contract)
             if (cp.ksplit > 1)
@@ -931,7 +1009,8 @@ static void account(tad_plan &p, Kernel &k)
     p.aux_bytes = std::max(p.aux_bytes, k.aux_bytes);
     std::function<int(const Kernel &)> launches = [&](const Kernel &x) {
         int n = 0;
-        if (x.contract.empty()) n = 1 + (x.prog.zsplit > 1 ? 1 + (x.prog.write_only_live ? 1 : 0) : 0);
+        if (!x.ew.empty()) n = 1;
+        else if (x.contract.empty()) n = 1 + (x.prog.zsplit > 1 ? 1 + (x.prog.write_only_live ? 1 : 0) : 0);
         for (const TadcProgram &cp : x.contract) n += 1 + (cp.ksplit > 1 ? 1 : 0);
         for (const Kernel &y : x.pre) n += launches(y);
         return n;

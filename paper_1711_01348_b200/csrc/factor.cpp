@@ -1057,9 +1057,9 @@ static bool factor_kernel(Gen &g, Kernel &k, int root, int scale, bool allow_spl
     }
     g3.lane_var = lane;
     Kernel main = k;
-    main.pre.clear(); main.contract.clear();
+    main.pre.clear(); main.contract.clear(); main.ew.clear();
     emit_plain_kernel(g3, main, root3, lower3, upper3, guards3, allow_split);
-    k.prog = main.prog; k.vec = main.vec; k.vec_u = main.vec_u; k.rich = main.rich; k.contract = main.contract;
+    k.prog = main.prog; k.vec = main.vec; k.vec_u = main.vec_u; k.rich = main.rich; k.contract = main.contract; k.ew = main.ew;
     k.listing = text + main.listing;
     k.pre = pre;
     return true;

@@ -9,6 +9,7 @@
 #include "intalg.h"
 #include "program.h"
 #include "contract.h"
+#include "ew.h"
 
 namespace tad {
 
@@ -70,6 +71,7 @@ struct Kernel {
     std::vector<int> stages_used;   // backward: staged adjoints it reads (indices into tad_plan::stages)
     std::vector<TadcProgram> contract;   // non-empty: the kernel is a contraction, run by the tile kernel (one launch per
                                          // program) instead of the interpreter
+    std::vector<TadeProgram> ew;         // non-empty: a kernel without loops, run by the element-wise kernel
     // Expression optimisation: tensors in the auxiliary area of the workspace and the kernels that fill them
     // (launched in this order before the kernel itself, each writing the tensor out_aux)
     struct Aux { size_t offset = 0, bytes = 0; int slot = 0; };

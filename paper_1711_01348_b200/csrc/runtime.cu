@@ -20,6 +20,7 @@ void set_error(const std::string &m);
 TAD_VM_SHAPES(TAD_DECLARE_VM)
 void tad_launch_vm_16_1_rich(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream);
 cudaError_t tad_launch_contract(const TadcProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream);
+cudaError_t tad_launch_ew(const TadeProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream);
 
 namespace {
 
@@ -122,6 +123,11 @@ tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStrea
         }
     }
     if (!k.contract.empty()) return launch_contractions(k, ptrs, stream);
+    if (!k.ew.empty()) {
+        const cudaError_t e = tad_launch_ew(k.ew[0], ptrs, (unsigned)sm_count(), stream);
+        if (e != cudaSuccess) { tad::set_error(std::string("element-wise launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
+        return TAD_OK;
+    }
     const int zsplit = k.prog.zsplit > 1 ? k.prog.zsplit : 1;
     if (zsplit > 1) {
         if (!ptrs.part) { tad::set_error("internal: partial-sum buffer missing"); return TAD_ERR_WORKSPACE; }

@@ -43,26 +43,35 @@ class GpuRun:
         return [d.cpu().numpy() if w else None for d, w in zip(self.dargs, wanted)]
 
 
-def assert_close(got, want, scale, what=""):
+def assert_close(got, want, scale, what="", mask=None):
+    """mask: compare only the elements where it is True (the others are checked to be finite)."""
     got = np.asarray(got, dtype=np.float64)
     err = np.abs(got - want)
     tol = RTOL_TERMS * scale + ATOL
     bad = ~(err <= tol)      # also catches NaN
+    if mask is not None:
+        assert np.all(np.isfinite(got[~mask])), f"{what}: non-finite value"
+        bad &= mask
     if bad.any():
         idx = np.unravel_index(np.argmax(np.where(bad, err - tol, -np.inf)), err.shape)
         raise AssertionError(f"{what}: {int(bad.sum())} of {bad.size} elements out of tolerance; worst at {idx}: "
                              f"gpu={got[idx]!r} oracle={want[idx]!r} tol={tol[idx]!r}")
 
 
-def check_against_oracle(expr, args, df, nthreads=1, debug_bounds=False, saved_forward=False):
+def check_against_oracle(expr, args, df, nthreads=1, debug_bounds=False, saved_forward=False, oracle_results=None, masks=None):
+    """oracle_results: (f, |f| scale, gradients, term scales) if the caller has them already;
+    masks: per tensor (f first, then the gradients), the elements to compare."""
     run = GpuRun(expr, args, df, debug_bounds=debug_bounds, saved_forward=saved_forward)
-    orc = Oracle(expr)
-    f_o, fabs_o = orc.forward(args, nthreads=nthreads)
-    assert_close(run.forward(), f_o, fabs_o, f"{expr.name} forward")
-    dx_o, t_o = orc.backward(args, df, nthreads=nthreads)
+    if oracle_results is None:
+        orc = Oracle(expr)
+        f_o, fabs_o = orc.forward(args, nthreads=nthreads)
+        dx_o, t_o = orc.backward(args, df, nthreads=nthreads)
+    else:
+        f_o, fabs_o, dx_o, t_o = oracle_results
+    assert_close(run.forward(), f_o, fabs_o, f"{expr.name} forward", None if masks is None else masks[0])
     dx_g = run.backward()
     for p, name in enumerate(expr.arg_names):
-        assert_close(dx_g[p], dx_o[p], t_o[p], f"{expr.name} d{name}")
+        assert_close(dx_g[p], dx_o[p], t_o[p], f"{expr.name} d{name}", None if masks is None else masks[1 + p])
         # elements with an empty Gamma are exactly zero
         assert np.all(dx_g[p][t_o[p] == 0] == 0.0), f"{expr.name} d{name}: non-zero where Gamma is empty"
     if debug_bounds:
