@@ -178,23 +178,24 @@ def run_reference(opts):
     print(json.dumps(line), flush=True)
 
 
-def run_ours(opts):
+CONTRACT_HBM_GBS = 8000.0      # the bandwidth the benchmark spec names for the roofline (nominal HBM3e)
+
+
+def time_workload(key, opts, dev, distributed, replicas, rows=0, saved_forward=False, steps=None, warmup=None):
+    """Builds one workload on the device, runs warm-up + timed steps with a CUDA event around every part.
+    One step = tad_forward, then exactly what tad_backward does: staging kernels, then every gradient.
+    Returns a dict with the per-part times and what the caller needs for the end-to-end run."""
     import torch
     from paper_1711_01348_b200 import Plan
     from workloads import configs as W
-
-    from paper_1711_01348_b200 import replicas
-    rank, local_rank, world = replicas.rank_info()
-    dev = torch.device(f"cuda:{local_rank}")
-    torch.cuda.set_device(dev)
-    distributed = replicas.init("nccl")
-
-    expr, args, df = W.workload(opts.config, full=True)
-    if opts.rows:
-        # profiler captures only: the same workload with fewer rows of the first output index
-        expr = W.profile_case(opts.config, opts.rows)
-        args, df = W.make_inputs(expr, W.DIST[opts.config], seed=0)
-    plan = Plan(expr, saved_forward=opts.saved_forward)
+    steps = opts.steps if steps is None else steps
+    warmup = opts.warmup if warmup is None else warmup
+    if rows:
+        expr = W.profile_case(key, rows)
+        args, df = W.make_inputs(expr, W.DIST[key], seed=0)
+    else:
+        expr, args, df = W.workload(key, full=True)
+    plan = Plan(expr, saved_forward=saved_forward)
     d_args = [a.to(dev) for a in args]
     d_df = df.to(dev)
     f = torch.empty(expr.out_shape, dtype=torch.float32, device=dev)
@@ -203,7 +204,7 @@ def run_ours(opts):
     stream = torch.cuda.current_stream().cuda_stream
     arg_ptrs = [a.data_ptr() for a in d_args]
     # a plan compiled with saved_forward reads the forward output of the same step in its backward kernels
-    bwd_ptrs = arg_ptrs + ([f.data_ptr()] if opts.saved_forward else [])
+    bwd_ptrs = arg_ptrs + ([f.data_ptr()] if saved_forward else [])
     darg_ptrs = [d.data_ptr() for d in dargs]
     n_args = len(d_args)
     n_stages = plan.num_stages()
@@ -211,7 +212,6 @@ def run_ours(opts):
     n_parts = len(parts)
 
     def step(events=None):
-        """forward, then exactly what tad_backward does: staging kernels, then every gradient."""
         e = 0
         if events is not None:
             events[e].record(); e += 1
@@ -227,26 +227,76 @@ def run_ours(opts):
         if events is not None:
             events[e].record()
 
-    def barrier():
-        replicas.barrier(distributed)
-
-    for _ in range(opts.warmup):
+    for _ in range(warmup):
         step()
-    barrier()
+    replicas.barrier(distributed)
+    all_events = [[torch.cuda.Event(enable_timing=True) for _ in range(n_parts + 1)] for _ in range(steps)]
+    t_begin = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    replicas.barrier(distributed)
+    t_begin.record()
+    for k in range(steps):
+        step(all_events[k])
+    t_end.record()
+    replicas.barrier(distributed)
+    total_ms = replicas.max_over_ranks(t_begin.elapsed_time(t_end), distributed, dev)
+    part_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in all_events) / steps for i in range(n_parts)]
+    return {"expr": expr, "args": args, "df": df, "plan": plan, "parts": parts, "part_ms": part_ms,
+            "ms_per_step": total_ms / steps, "n_stages": n_stages, "steps": steps}
+
+
+def part_records(run, peaks, fp32_clock_tflops, fp32_measured_tflops):
+    """Per part: time, algorithmic work (the expression as written, counted by the plan), the roof that binds
+    it and the achieved fraction against three denominators: `frac` (measured HBM copy bandwidth / FP32 peak
+    by the maximum SM clock), `frac_measured_fma` (ALU parts: against the measured multiply-add rate) and
+    `frac_contract` (the benchmark spec's 8 TB/s and the same FP32 peak)."""
+    expr, plan = run["expr"], run["plan"]
+    first_access = {}
+    for q, a in enumerate(expr.accesses):
+        first_access.setdefault(a.arg, []).append(q)
+    out, launches = [], 0
+    for i, name in enumerate(run["parts"]):
+        if name == "forward":
+            qs = [-1]
+        elif name == "stage":
+            qs = [-2 - st for st in range(run["n_stages"])]
+        else:
+            qs = first_access.get(expr.arg_names.index(name[1:]), [])
+        flops = sum(plan.kernel_stats(q).alg_flops for q in qs)
+        byts = sum(plan.kernel_stats(q).alg_bytes for q in qs)
+        launches += sum(plan.kernel_stats(q).n_launches for q in qs)
+        ms = run["part_ms"][i]
+        t_alu = flops / (fp32_clock_tflops * 1e12)
+        t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
+        bound = "alu" if t_alu >= t_hbm else "hbm"
+        rec = {"part": name, "ms": ms, "alg_gflop": flops / 1e9, "alg_gb": byts / 1e9, "bound": bound,
+               "frac": max(t_alu, t_hbm) / (ms * 1e-3) if ms > 0 else None}
+        if ms > 0:
+            rec["frac_contract"] = max(t_alu, byts / (CONTRACT_HBM_GBS * 1e9)) / (ms * 1e-3)
+            if bound == "alu" and fp32_measured_tflops:
+                rec["frac_measured_fma"] = flops / (fp32_measured_tflops * 1e12) / (ms * 1e-3)
+        out.append(rec)
+    return out, launches
+
+
+def run_ours(opts):
+    import torch
+    from paper_1711_01348_b200 import measure_fp32_rate
+    from workloads import configs as W
+
+    from paper_1711_01348_b200 import replicas
+    rank, local_rank, world = replicas.rank_info()
+    dev = torch.device(f"cuda:{local_rank}")
+    torch.cuda.set_device(dev)
+    distributed = replicas.init("nccl")
+    stream = torch.cuda.current_stream().cuda_stream
+
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    all_events = [[torch.cuda.Event(enable_timing=True) for _ in range(n_parts + 1)] for _ in range(opts.steps)]
-    t_begin = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
-    barrier()
-    t_begin.record()
-    for k in range(opts.steps):
-        step(all_events[k])
-    t_end.record()
-    barrier()
+    run = time_workload(opts.config, opts, dev, distributed, replicas, rows=opts.rows, saved_forward=opts.saved_forward)
     clocks = sampler.stop() if rank == 0 else None
-    total_ms = replicas.max_over_ranks(t_begin.elapsed_time(t_end), distributed, dev)
-    part_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in all_events) / opts.steps for i in range(n_parts)]
+    expr, args, df, plan = run["expr"], run["args"], run["df"], run["plan"]
+    ms_per_step = run["ms_per_step"]
 
     # end to end: pinned host buffers in, results back, through tad_step_host
     e2e = None
@@ -264,7 +314,7 @@ def run_ours(opts):
             plan.step_host([a.data_ptr() for a in h_args], h_df.data_ptr(), h_f.data_ptr(),
                            [d.data_ptr() for d in h_dargs], staging.data_ptr(), staging.numel(), stream)
         host_step()
-        barrier()
+        replicas.barrier(distributed)
         t0 = time.perf_counter()
         for _ in range(e2e_steps):
             host_step()
@@ -275,50 +325,53 @@ def run_ours(opts):
         d2h = h_f.numel() * 4 + sum(d.numel() * 4 for d in h_dargs)
         e2e = {"value": world * elements_per_step(expr) / e2e_s, "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * e2e_s}
-        del staging
+        del staging, h_args, h_df, h_f, h_dargs
     except RuntimeError as exc:                       # e.g. not enough pinned memory
         e2e = {"value": None, "unit": UNIT, "error": str(exc)[:200]}
 
     if rank == 0:
         peaks = load_peaks()
         sms = torch.cuda.get_device_properties(dev).multi_processor_count
-        fp32_peak_tflops = 2 * 128 * sms * peaks["sm_max_mhz"] * 1e6 / 1e12
-        stats = [plan.kernel_stats(-1)]
-        first_access = {}
-        for q, a in enumerate(expr.accesses):
-            first_access.setdefault(a.arg, []).append(q)
-        per_part = []
-        launches = 0
-        for i, name in enumerate(parts):
-            if name == "forward":
-                qs = [-1]
-            elif name == "stage":
-                qs = [-2 - st for st in range(n_stages)]
-            else:
-                qs = first_access.get(expr.arg_names.index(name[1:]), [])
-            flops = sum(plan.kernel_stats(q).alg_flops for q in qs)
-            byts = sum(plan.kernel_stats(q).alg_bytes for q in qs)
-            nl = sum(plan.kernel_stats(q).n_launches for q in qs)
-            launches += nl
-            ms = part_ms[i]
-            t_alu = flops / (fp32_peak_tflops * 1e12)
-            t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
-            per_part.append({"part": name, "ms": ms, "alg_gflop": flops / 1e9, "alg_gb": byts / 1e9,
-                             "bound": "alu" if t_alu >= t_hbm else "hbm",
-                             "frac": max(t_alu, t_hbm) / (ms * 1e-3) if ms > 0 else None})
-        dom = max(range(len(parts)), key=lambda i: part_ms[i])
+        fp32_clock = 2 * 128 * sms * peaks["sm_max_mhz"] * 1e6 / 1e12
+        try:
+            fp32_measured = measure_fp32_rate(stream)
+        except Exception:                              # noqa: BLE001 - the fraction against it is then left out
+            fp32_measured = None
+        per_part, launches = part_records(run, peaks, fp32_clock, fp32_measured)
+        # the roofline object describes the slowest backward part (the target is on the backward kernels)
+        backward = [i for i, p in enumerate(per_part) if p["part"] not in ("forward",)]
+        dom = max(backward or range(len(per_part)), key=lambda i: per_part[i]["ms"])
         d = per_part[dom]
         if d["bound"] == "alu":
             achieved = d["alg_gflop"] / 1e3 / (d["ms"] * 1e-3)
-            roof = {"bound": "alu", "achieved": achieved, "peak": fp32_peak_tflops, "unit": "TFLOP/s",
-                    "frac": achieved / fp32_peak_tflops, "traffic": None,
-                    "peak_source": f"2 x 128 lanes x {sms} SMs x {peaks['sm_max_mhz']:.0f} MHz ({peaks['source']} clock)"}
+            roof = {"bound": "alu", "achieved": achieved, "peak": fp32_clock, "unit": "TFLOP/s",
+                    "frac": achieved / fp32_clock, "traffic": None,
+                    "peak_source": f"2 x 128 lanes x {sms} SMs x {peaks['sm_max_mhz']:.0f} MHz ({peaks['source']} clock)",
+                    "peak_measured_fma": fp32_measured,
+                    "frac_measured_fma": achieved / fp32_measured if fp32_measured else None}
         else:
             achieved = d["alg_gb"] / (d["ms"] * 1e-3)
             roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                    "frac_contract": achieved / CONTRACT_HBM_GBS}
         roof["kernel"] = d["part"]
         roof["traffic"] = recorded_traffic(expr.name, d["part"])
+        # the other workloads: same timing, parts only (cfg1 is a launch-latency case: times, no fractions)
+        others = {}
+        if opts.all_workloads and not distributed and not opts.rows:
+            run = None
+            torch.cuda.empty_cache()
+            for key in ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"]:
+                if key == opts.config:
+                    continue
+                r = time_workload(key, opts, dev, distributed, replicas, steps=max(opts.steps, 20), warmup=max(opts.warmup, 3))
+                recs, nl = part_records(r, peaks, fp32_clock, fp32_measured)
+                if key == "cfg1":
+                    recs = [{"part": p["part"], "us": 1e3 * p["ms"]} for p in recs]
+                others[key] = {"workload": r["expr"].name, "ms_per_step": r["ms_per_step"], "steps": r["steps"],
+                               "gpu_launches_per_step": nl, "l2": L2_NOTE[key], "parts": recs}
+                del r
+                torch.cuda.empty_cache()
         cpu = None
         if not distributed and not opts.no_cpu_baseline and not opts.rows:
             from oracle.oracle import build as build_oracle, max_threads
@@ -327,7 +380,6 @@ def run_ours(opts):
             dt, elems, sample = oracle_sample(opts.config, expr, args, df, cores)
             cpu = {"value": elems / dt, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
                    "seconds": dt}
-        ms_per_step = total_ms / opts.steps
         line = {"metric": METRIC, "value": world * elements_per_step(expr) / (ms_per_step * 1e-3), "unit": UNIT,
                 "n_gpus": world, "steps": opts.steps, "warmup": opts.warmup, "ms_per_step": ms_per_step,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
@@ -336,7 +388,10 @@ def run_ours(opts):
                            "l2": L2_NOTE[opts.config],
                            "saved_forward": bool(opts.saved_forward),
                            "parallelism": "replicas" if world > 1 else "single"},
-                "roofline": roof, "parts": per_part, "cpu_baseline": cpu, "e2e": e2e,
+                "roofline": roof, "parts": per_part,
+                "fp32_peak": {"by_clock_tflops": fp32_clock, "measured_fma_tflops": fp32_measured,
+                              "contract_hbm_gbs": CONTRACT_HBM_GBS, "measured_hbm_gbs": peaks["hbm_gbs"]},
+                "workloads": others, "cpu_baseline": cpu, "e2e": e2e,
                 "gpu_launches": launches * opts.steps, "clocks": clocks}
         print(json.dumps(line), flush=True)
     replicas.finish(distributed)
@@ -351,6 +406,8 @@ def main():
     ap.add_argument("--config", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--single", dest="all_workloads", action="store_false",
+                    help="time only the workload of --config (the default run also times the parts of the other four)")
     ap.add_argument("--saved-forward", action="store_true",
                     help="compile the plan with saved_forward: the backward kernels read f of the same step")
     ap.add_argument("--rows", type=int, default=0,

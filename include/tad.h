@@ -240,6 +240,15 @@ tad_status tad_step_host(const tad_plan *plan, const float *const *h_args, const
 /* Text of the last non-OK status on the calling thread ("" if none). */
 const char *tad_last_error(void);
 
+/*
+ * Measures the rate at which the current device retires FP32 multiply-adds from registers (a short kernel of
+ * independent multiply-add chains, well under 100 ms, timed with events on the given stream; the call
+ * synchronises).  The benchmark divides the algorithmic flops of ALU-bound kernels by this rate next to the
+ * clock-derived peak.  No counterpart in the paper: a measurement aid.  Allocates four bytes for the duration
+ * of the call.  *tflops is written only on TAD_OK.
+ */
+tad_status tad_measure_fp32_rate(void *cuda_stream, double *tflops);
+
 /* debug_bounds plans: reads back (and clears) the debug word in `workspace` after
  * synchronising the stream.  TAD_ERR_OUT_OF_RANGE if a kernel skipped an out-of-range
  * access since the last query, TAD_OK otherwise. */

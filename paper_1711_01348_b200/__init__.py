@@ -2,4 +2,4 @@
 expressions (Urban & van der Smagt, 2017).  Everything runs in libtad.so; this package is the
 ctypes binding."""
 from .binding import (AccessInfo, KernelStats, Plan, TadError, extended_euclid,  # noqa: F401
-                      fourier_motzkin, smith_normal_form, lib, EXPORTS)
+                      fourier_motzkin, measure_fp32_rate, smith_normal_form, lib, EXPORTS)

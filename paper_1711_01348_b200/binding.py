@@ -26,7 +26,8 @@ EXPORTS = ["tad_compile", "tad_destroy", "tad_workspace_bytes", "tad_forward", "
            "tad_backward_stage", "tad_backward_arg", "tad_plan_num_stages", "tad_backward_noalloc",
            "tad_staging_bytes", "tad_step_host", "tad_last_error", "tad_debug_status",
            "tad_plan_access_info", "tad_plan_bound_row", "tad_plan_enumerate", "tad_plan_kernel_stats",
-           "tad_plan_disassemble", "tad_extended_euclid", "tad_smith_normal_form", "tad_fourier_motzkin"]
+           "tad_plan_disassemble", "tad_extended_euclid", "tad_smith_normal_form", "tad_fourier_motzkin",
+           "tad_measure_fp32_rate"]
 
 
 class TadError(RuntimeError):
@@ -268,6 +269,13 @@ class Plan:
 
 
 # ---- host-only pieces of the integer algebra (for tests) ----
+
+def measure_fp32_rate(stream: int = 0) -> float:
+    """TFLOP/s of FP32 multiply-adds from registers on the current device (tad_measure_fp32_rate)."""
+    out = C.c_double(0.0)
+    _check(lib.tad_measure_fp32_rate(stream or None, C.byref(out)))
+    return out.value
+
 
 def extended_euclid(a: int, b: int):
     g, x, y = C.c_int64(), C.c_int64(), C.c_int64()

@@ -342,7 +342,10 @@ void finish_stats(Gen &g, Kernel &k, bool backward, int64_t outputs, int64_t ter
         case I_EXP: case I_LOG: case I_SIN: case I_COS: case I_TANH: case I_SINH: case I_COSH:
             s.alg_flops += n; s.alg_trans += n; break;
         case I_POWI: s.alg_flops += n * std::max(1, std::abs(in.ipow) - 1); break;
-        case I_SUM: s.alg_flops += bindings(g.inst[in.a].adeps | (1u << (16 + in.var))); break;   // one add per summand
+        case I_SUM:
+            // one add per summand; a sum whose summand is a sum adds nothing of its own (they share one accumulator)
+            if (g.inst[in.a].op != I_SUM) s.alg_flops += bindings(g.inst[in.a].adeps | (1u << (16 + in.var)));
+            break;
         default: s.alg_flops += n; break;
         }
     }

@@ -65,6 +65,24 @@ tad_reduce_partials(const __grid_constant__ TadpProgram P, float *out, const flo
     }
 }
 
+// Sixteen independent multiply-add chains per thread, operands in registers only: the rate at which this GPU
+// retires FP32 multiply-adds under its own clocks (the denominator of the ALU-bound roofline fractions).
+__global__ void __launch_bounds__(256)
+tad_fma_rate_kernel(float *sink, int iters, float m)
+{
+    float a[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) a[i] = (float)(threadIdx.x + i) * 1e-3f;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) a[i] = fmaf(a[i], m, 1e-7f);
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) s += a[i];
+    if (s == 12345.678f) *sink = s;             // never true: keeps the chains alive
+}
+
 __global__ void tad_fill_zero(float *out, unsigned n)
 {
     const unsigned stride = gridDim.x * blockDim.x;
@@ -473,6 +491,35 @@ tad_status tad_backward_noalloc(const tad_plan *plan, const float *const *args, 
         if (e != cudaSuccess) { tad::set_error(std::string("clearing the debug word: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
     }
     return tad_backward(plan, args, df, dargs, scratch, TAD_NOALLOC_SCRATCH_BYTES, cuda_stream);
+}
+
+tad_status tad_measure_fp32_rate(void *cuda_stream, double *tflops)
+{
+    if (!tflops) { tad::set_error("NULL argument"); return TAD_ERR_INVALID_ARG; }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    float *sink = nullptr;
+    const unsigned blocks = (unsigned)sm_count() * 8u, threads = 256u;
+    const int iters = 4096;
+    cudaError_t e = cudaMalloc(&sink, sizeof(float));
+    if (e == cudaSuccess) e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) {
+        tad_fma_rate_kernel<<<blocks, threads, 0, stream>>>(sink, iters, 1.0001f);           // warm-up
+        e = cudaEventRecord(e0, stream);
+        if (e == cudaSuccess) { tad_fma_rate_kernel<<<blocks, threads, 0, stream>>>(sink, iters, 1.0001f); e = cudaGetLastError(); }
+        if (e == cudaSuccess) e = cudaEventRecord(e1, stream);
+        if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    }
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    if (sink) cudaFree(sink);
+    if (e != cudaSuccess || ms <= 0.f) { tad::set_error(std::string("measuring the multiply-add rate: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
+    const double flops = 2.0 * 16.0 * (double)iters * (double)blocks * (double)threads;
+    *tflops = flops / (ms * 1e-3) / 1e12;
+    return TAD_OK;
 }
 
 tad_status tad_debug_status(const tad_plan *plan, void *workspace, void *cuda_stream)
