@@ -54,8 +54,9 @@ typedef enum {
     TAD_ERR_NOMEM = 8
 } tad_status;
 
-/* Elementary functions of the scalar expression fbar (Sec. 2: "addition, subtraction,
- * multiplication, division, trigonometric function, the exponential function, the logarithm"). */
+/* Node operations of the scalar expression fbar: the elementary functions Sec. 2 builds its
+ * computational graphs from (arithmetic, integer powers, exponential, logarithm, circular and
+ * hyperbolic functions) and the sum over an index with a constant range of Sec. 5.2. */
 typedef enum {
     TAD_OP_CONST = 0,   /* imm */
     TAD_OP_LOAD = 1,    /* element of an argument, through access[access] */
@@ -200,7 +201,8 @@ tad_status tad_backward_arg(const tad_plan *plan, const float *const *args, cons
  * a host application's own memory pool, a callback that runs while allocation is forbidden,
  * or a process whose device-memory budget is fixed at start-up.  (The paper has no
  * counterpart: it evaluates derivatives without temporary memory, Sec. 7; this library
- * stages shared adjoints and therefore needs scratch.)
+ * stages shared adjoints, keeps partial sums of split summations and the auxiliary tensors
+ * of its expression optimisation in scratch.)
  *
  * The scratch is a fixed array of TAD_NOALLOC_SCRATCH_BYTES inside the library image; every
  * GPU that loads the library holds that much memory until the process exits.  A plan whose
@@ -224,7 +226,8 @@ tad_status tad_backward_noalloc(const tad_plan *plan, const float *const *args, 
  * tad_step_host: one forward and one backward pass with HOST buffers (same meaning as
  * tad_forward followed by tad_backward).  Inputs are copied to the device staging area,
  * results copied back.  The kernels run on the given stream, after whatever it already
- * holds; the copies run on two streams the call creates and destroys, ordered by events so
+ * holds; the copies run on two streams of the plan's own (created by the first call, released
+ * by tad_destroy; calls on one plan must not run concurrently), ordered by events so
  * that df goes up during the forward pass and f and each gradient come down while the next
  * kernels run.  The call returns after all of it has drained.  Host buffers should be pinned for the copies to
  * be asynchronous.  staging is a DEVICE buffer of at least tad_staging_bytes() bytes,
@@ -251,7 +254,9 @@ tad_status tad_measure_fp32_rate(void *cuda_stream, double *tflops);
 
 /* debug_bounds plans: reads back (and clears) the debug word in `workspace` after
  * synchronising the stream.  TAD_ERR_OUT_OF_RANGE if a kernel skipped an out-of-range
- * access since the last query, TAD_OK otherwise. */
+ * access since the last query, TAD_OK otherwise.  workspace == NULL asks about the scratch
+ * of tad_backward_noalloc on the current device (query it before the next call of that
+ * entry point, which clears the word). */
 tad_status tad_debug_status(const tad_plan *plan, void *workspace, void *cuda_stream);
 
 /* ------------------------------------------------------------------------- */

@@ -54,7 +54,7 @@ tad_status tad_compile(const tad_expr *expr, const tad_options *opt, tad_plan **
     return TAD_OK;
 }
 
-void tad_destroy(tad_plan *plan) { delete plan; }
+void tad_destroy(tad_plan *plan) { if (plan) tad_release_host_step(plan); delete plan; }
 
 int32_t tad_plan_num_stages(const tad_plan *plan) { return plan ? (int32_t)plan->stages.size() : 0; }
 

@@ -5,6 +5,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <mutex>
+#include <new>
 #include <string>
 
 #include "plan.h"
@@ -188,6 +189,20 @@ tad_status zero_fill(float *out, int64_t n, cudaStream_t stream)
 
 }  // namespace
 
+// streams and events of tad_step_host, owned by a plan
+struct HostStep {
+    static constexpr int N_EVENTS = 4 + TADP_MAX_PTRS;
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t ev[N_EVENTS] = {};
+    void release()
+    {
+        for (cudaEvent_t &e : ev) if (e) { cudaEventDestroy(e); e = nullptr; }
+        if (in) cudaStreamDestroy(in);
+        if (out) cudaStreamDestroy(out);
+        in = out = nullptr;
+    }
+};
+
 // Scratch of tad_backward_noalloc: lives in the library image, one copy per GPU that loads it.
 static __device__ __align__(256) unsigned char tad_noalloc_scratch[TAD_NOALLOC_SCRATCH_BYTES];
 
@@ -249,6 +264,15 @@ bool fill_inputs(const tad_plan *plan, const float *const *args, const float *df
 }
 
 }  // namespace
+
+void tad_release_host_step(const tad_plan *plan)
+{
+    if (!plan || !plan->host_step) return;
+    HostStep *hs = static_cast<HostStep *>(plan->host_step);
+    hs->release();
+    delete hs;
+    plan->host_step = nullptr;
+}
 
 extern "C" {
 
@@ -371,27 +395,23 @@ tad_status tad_step_host(const tad_plan *plan, const float *const *h_args, const
     float *d_df = reinterpret_cast<float *>(cur); cur += pad(fbytes);
 
     // Copies run on two streams of their own so that they overlap the kernels: df goes up while the
-    // forward pass runs, f and every gradient come down while the next kernels run.
+    // forward pass runs, f and every gradient come down while the next kernels run.  The streams and
+    // events belong to the plan: made by the first call, reused by every later one.
+    if (!plan->host_step) {
+        HostStep *hs = new (std::nothrow) HostStep();
+        if (!hs) { tad::set_error("out of host memory"); return TAD_ERR_NOMEM; }
+        bool ok = cudaStreamCreateWithFlags(&hs->in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&hs->out, cudaStreamNonBlocking) == cudaSuccess;
+        for (int i = 0; ok && i < HostStep::N_EVENTS; ++i) ok = cudaEventCreateWithFlags(&hs->ev[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) { hs->release(); delete hs; tad::set_error("creating the copy streams and events failed"); return TAD_ERR_CUDA; }
+        plan->host_step = hs;
+    }
     struct Side {
-        cudaStream_t in = nullptr, out = nullptr;
-        cudaEvent_t ev[4 + TADP_MAX_PTRS] = {};
-        int n_ev = 0;
-        ~Side()
-        {
-            for (int i = 0; i < n_ev; ++i) if (ev[i]) cudaEventDestroy(ev[i]);
-            if (in) cudaStreamDestroy(in);
-            if (out) cudaStreamDestroy(out);
-        }
-        cudaEvent_t event()
-        {
-            cudaEvent_t e = nullptr;
-            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-            ev[n_ev++] = e;
-            return e;
-        }
-    } side;
-    if (!check(cudaStreamCreateWithFlags(&side.in, cudaStreamNonBlocking), "stream for the copies in") ||
-        !check(cudaStreamCreateWithFlags(&side.out, cudaStreamNonBlocking), "stream for the copies out")) return TAD_ERR_CUDA;
+        HostStep *hs; int used = 0;
+        cudaStream_t in, out;
+        cudaEvent_t event() { return used < HostStep::N_EVENTS ? hs->ev[used++] : nullptr; }
+    } side{static_cast<HostStep *>(plan->host_step)};
+    side.in = side.hs->in; side.out = side.hs->out;
     cudaEvent_t ev_start = side.event(), ev_args = side.event(), ev_df = side.event(), ev_f = side.event();
     if (!ev_start || !ev_args || !ev_df || !ev_f) { tad::set_error("event creation failed"); return TAD_ERR_CUDA; }
     // whatever the caller queued on its stream comes first
@@ -526,7 +546,14 @@ tad_status tad_debug_status(const tad_plan *plan, void *workspace, void *cuda_st
 {
     if (!plan) { tad::set_error("NULL plan"); return TAD_ERR_INVALID_ARG; }
     if (!plan->opt.debug_bounds) return TAD_OK;
-    if (!workspace) { tad::set_error("NULL workspace"); return TAD_ERR_INVALID_ARG; }
+    if (!workspace) {
+        // the scratch of tad_backward_noalloc on the current device, if that entry point has run here
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) { tad::set_error("no current device"); return TAD_ERR_CUDA; }
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        workspace = g_noalloc_ptr[dev];
+        if (!workspace) { tad::set_error("NULL workspace (and tad_backward_noalloc has not run on this device)"); return TAD_ERR_INVALID_ARG; }
+    }
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     int32_t word = 0;
     cudaError_t e = cudaMemcpyAsync(&word, workspace, sizeof word, cudaMemcpyDeviceToHost, stream);

@@ -350,3 +350,50 @@ def test_masked_fused_loops_get_the_register_rich_build():
     # the forward pass has no loops: sin over the elements of x once (a function table), then an element-wise program
     fwd = plan.disassemble(-1)
     assert "; function table" in fwd and fwd.count("; element-wise program") == 2
+
+
+# --------------------------------------------------------------------------- #
+# argument checks that return before anything is launched (no GPU needed)
+# --------------------------------------------------------------------------- #
+
+def _many_args(n_args):
+    """f_i = x0_i + x1_i + ... : one index expression per argument."""
+    from workloads.expr import Builder, unit
+    b = Builder(f"sum_of_{n_args}", [8], 0, [f"x{k}" for k in range(n_args)], [[8]] * n_args)
+    acc = b.load("x0", [unit(1, (0, 1))])
+    for k in range(1, n_args):
+        acc = b.bin("add", acc, b.load(f"x{k}", [unit(1, (0, 1))]))
+    return b.done()
+
+
+def test_pointer_slots_count_the_saved_forward_output():
+    """Arguments, df and (for saved_forward plans) f share 16 pointer slots: 15 arguments fit without the saved
+    output and are refused with it, instead of letting f overwrite the slot of df."""
+    Plan(_many_args(15))
+    Plan(_many_args(14), saved_forward=True)
+    with pytest.raises(TadError) as ei:
+        Plan(_many_args(15), saved_forward=True)
+    assert ei.value.code == "TAD_ERR_UNSUPPORTED"
+    with pytest.raises(TadError):
+        Plan(_many_args(16))
+
+
+def test_workspace_too_small_or_misaligned_is_refused_before_any_launch():
+    from workloads import configs as W
+    e = W.REDUCED["cfg2"]()
+    plan = Plan(e)
+    need = plan.workspace_bytes()
+    assert need > 0
+    fake = 1 << 20                                   # never dereferenced: the checks come first
+    args = [fake] * len(e.arg_shapes)
+    for ws_ptr, ws_bytes in ((fake, need - 1), (fake + 8, need + 256), (0, 0)):
+        with pytest.raises(TadError) as ei:
+            plan.backward(args, fake, [fake] * len(args), ws_ptr, ws_bytes)
+        assert ei.value.code == "TAD_ERR_WORKSPACE", (ws_ptr, ws_bytes)
+    # the forward pass of the full-size workload keeps auxiliary tensors in the workspace
+    big = Plan(W.FULL["cfg2"]())
+    need = big.workspace_bytes()
+    for ws_ptr, ws_bytes in ((fake, need - 1), (fake + 8, need + 256), (0, 0)):
+        with pytest.raises(TadError) as ei:
+            big.forward(args, fake, 0, ws_ptr, ws_bytes)
+        assert ei.value.code == "TAD_ERR_WORKSPACE", (ws_ptr, ws_bytes)
