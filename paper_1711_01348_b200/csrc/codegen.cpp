@@ -560,10 +560,11 @@ int body_fetch_kind(const TadpLoad &L, int ta, int ub)
 
 // A program without loops and temporaries whose pending values never exceed two becomes an element-wise program
 // (ew.h); a thread owns four consecutive values of the lane variable.
-bool try_elementwise(Gen &g, Kernel &k, const Emitter &em)
+bool try_elementwise(Gen &g, Kernel &k, const Emitter &em, const std::vector<TadpRow> &guards)
 {
     const TadpProgram &prog = k.prog;
-    if (g.kappa != 0 || g.p.opt.debug_bounds || prog.n_guards || prog.write_only_live) return false;
+    // (elements that a guard or a mask excludes are not evaluated by the interpreter: such kernels stay there)
+    if (g.kappa != 0 || g.p.opt.debug_bounds || !guards.empty() || prog.write_only_live) return false;
     if (g.lane_var < 0 || g.lane_var >= g.n_outer) return false;
     if ((int)g.loads.size() > TADE_MAX_LOADS) return false;
     const std::vector<TadpInsn> &code = em.code;
@@ -605,6 +606,18 @@ bool try_elementwise(Gen &g, Kernel &k, const Emitter &em)
     if (term_op == P_MACC) { if (vd != 2) return false; push_step(E_MULY); }
     else if (vd != 1) return false;
     if ((int)steps.size() > TADE_MAX_STEPS) return false;
+    // every offset the kernel can form must lie inside its tensor (interval check over the outer box)
+    auto inside = [&](const int32_t *coef, int64_t base, int64_t limit) {
+        int64_t lo = base, hi = base;
+        for (int v = 0; v < g.n_outer; ++v) {
+            const int64_t a = (int64_t)coef[v] * prog.outer_lo[v], b = (int64_t)coef[v] * (prog.outer_lo[v] + std::max(1, prog.outer_ext[v]) - 1);
+            lo += std::min(a, b); hi += std::max(a, b);
+        }
+        return lo >= 0 && hi < limit;
+    };
+    for (const TadeStep &s : steps)
+        if (s.op == E_LD && !inside(g.loads[s.a].coef, g.loads[s.a].base, g.loads[s.a].limit)) return false;
+    if (!inside(prog.out_coef, prog.out_base, prog.out_limit)) return false;
     TadeProgram E{};
     E.n_outer = g.n_outer; E.lane_var = g.lane_var;
     for (int v = 0; v < g.n_outer; ++v) {
@@ -750,7 +763,7 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     if (scale >= 0) { em.expr(scale); em.emit(P_SCALE, 0, 0, 0, -1); }
     em.emit(P_END);
     if (em.depth != 0) throw BadExpr("internal: unbalanced operand stack");
-    if (n_temps == 0 && try_elementwise(g, k, em)) return;
+    if (n_temps == 0 && try_elementwise(g, k, em, guards)) return;
     // rows
     std::vector<TadpRow> rows;
     for (TadpLoop &L : em.loops) {

@@ -487,6 +487,157 @@ tad_rowsum_kernel(const __grid_constant__ TadcProgram P, const __grid_constant__
     }
 }
 
+// Narrow contractions that stream a big operand: out[m, n] = sum_k A[m, k] B[n, k] with at most 36 columns n,
+// one digit each for m, n and k, and B[k][n] rows of consecutive elements (the column blocks the optimisation
+// pass lays out, or an argument read along its rows).  Every element of A is used by exactly one thread, so A
+// goes from global memory straight into registers; only B is staged: 128 summation indices x 36 columns at a
+// time in shared memory (16-byte asynchronous copies, two buffers), read with 128-bit loads.
+//   A along k (A[m, k] consecutive in k): a warp owns two rows m, its lanes walk k four at a time (coalesced
+//   128-bit loads), every lane keeps the sums of all columns for both rows and the warp adds them up at the end.
+//   A along m (A[m, k] consecutive in m): a lane owns two rows m (32 apart) and walks all k of the block's slice;
+//   the B values of a k are the same for the whole warp (broadcast loads).
+// A summation split over blocks (grid.y) writes planes of partial sums like the tile kernel.
+constexpr int SK_COLS = 36;        // columns held per row (9 groups of four)
+constexpr int SK_KC = 128;         // summation indices per stage of B
+
+__global__ void __launch_bounds__(256, 2)
+tad_skinny_kernel(const __grid_constant__ TadcProgram P, const __grid_constant__ TadpPointers ptrs)
+{
+    __shared__ __align__(16) float bs[2][SK_KC * SK_COLS];
+    const unsigned tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const float *__restrict__ A = ptrs.in[P.ptrA];
+    const float *__restrict__ B = ptrs.in[P.ptrB];
+    const unsigned Mext = (unsigned)P.M.extent, Next = (unsigned)P.N.extent, Kext = (unsigned)P.K.extent;
+    const int sAm = P.M.n_digits ? P.M.sA[0] : 0, sAk = P.K.n_digits ? P.K.sA[0] : 0, sBk = P.K.n_digits ? P.K.sB[0] : 0;
+    const unsigned ksplit = (unsigned)max(1, P.ksplit);
+    const unsigned ks = blockIdx.y;
+    const unsigned kbeg = ks * (unsigned)P.kchunk, kend = min(Kext, kbeg + (unsigned)P.kchunk);
+    const int n_chunks = (int)((kend - kbeg + SK_KC - 1) / SK_KC);
+    const bool along_k = P.modeA == TG_K;
+    // rows of this thread
+    unsigned m0, m1;
+    if (along_k) { m0 = (blockIdx.x * 8u + warp) * 2u; m1 = m0 + 1u; }
+    else { m0 = (blockIdx.x * 8u + warp) * 64u + lane; m1 = m0 + 32u; }
+    const bool live0 = m0 < Mext, live1 = m1 < Mext;
+    const unsigned a0 = (unsigned)(P.baseA + (int)(live0 ? m0 : 0u) * sAm), a1 = (unsigned)(P.baseA + (int)(live1 ? m1 : 0u) * sAm);
+    float acc0[SK_COLS], acc1[SK_COLS];
+#pragma unroll
+    for (int n = 0; n < SK_COLS; ++n) { acc0[n] = 0.f; acc1[n] = 0.f; }
+    // B chunk: rows of Next consecutive floats at B + baseB + k * sBk, copied as 16-byte pieces; columns beyond
+    // Next and rows beyond the slice are zero
+    const unsigned pieces = (Next + 3u) / 4u;                    // 16-byte pieces per row
+    auto issue = [&](int chunk) {
+        if (chunk < n_chunks) {
+            float *dst = bs[chunk & 1];
+            const unsigned k0 = kbeg + (unsigned)chunk * SK_KC;
+            for (unsigned e = tid; e < SK_KC * (SK_COLS / 4); e += 256u) {
+                const unsigned kl = e / (SK_COLS / 4), pc = e % (SK_COLS / 4);
+                const bool ok = pc < pieces && k0 + kl < kend;
+                // a row's last piece may reach past Next: the pass pads its rows to whole pieces, an argument read
+                // along rows of a length that is no multiple of four does not take this kernel
+                cp_async16(dst + kl * SK_COLS + pc * 4, B + (ok ? (unsigned)(P.baseB + (int)(k0 + kl) * sBk + (int)pc * 4) : 0u), ok);
+            }
+        }
+        cp_async_commit();
+    };
+    issue(0);
+    for (int ch = 0; ch < n_chunks; ++ch) {
+        issue(ch + 1);
+        cp_async_wait<1>();
+        __syncthreads();
+        const float *bsc = bs[ch & 1];
+        const unsigned k0 = kbeg + (unsigned)ch * SK_KC;
+        if (along_k) {
+            // lanes along k: this lane's four summation indices of the chunk, both rows
+            const unsigned k = k0 + lane * 4u;
+            float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0;
+            if (k < kend) {          // (slices are multiples of four long)
+                if (live0) g0 = __ldg(reinterpret_cast<const float4 *>(A + a0 + k));
+                if (live1) g1 = __ldg(reinterpret_cast<const float4 *>(A + a1 + k));
+            }
+            const float ga[4] = {g0.x, g0.y, g0.z, g0.w}, gb[4] = {g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const float *row = bsc + (lane * 4u + kk) * SK_COLS;
+#pragma unroll
+                for (int q = 0; q < SK_COLS / 4; ++q) {
+                    const float4 b4 = *reinterpret_cast<const float4 *>(row + 4 * q);
+                    acc0[4 * q] = fmaf(ga[kk], b4.x, acc0[4 * q]); acc0[4 * q + 1] = fmaf(ga[kk], b4.y, acc0[4 * q + 1]);
+                    acc0[4 * q + 2] = fmaf(ga[kk], b4.z, acc0[4 * q + 2]); acc0[4 * q + 3] = fmaf(ga[kk], b4.w, acc0[4 * q + 3]);
+                    acc1[4 * q] = fmaf(gb[kk], b4.x, acc1[4 * q]); acc1[4 * q + 1] = fmaf(gb[kk], b4.y, acc1[4 * q + 1]);
+                    acc1[4 * q + 2] = fmaf(gb[kk], b4.z, acc1[4 * q + 2]); acc1[4 * q + 3] = fmaf(gb[kk], b4.w, acc1[4 * q + 3]);
+                }
+            }
+        } else {
+            // lanes along m: every k of the chunk, the loads of A eight indices ahead of their use
+            const int kn = (int)min((unsigned)SK_KC, kend - k0);
+            for (int kb = 0; kb < kn; kb += 8) {
+                float ga[8], gb[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const bool ok = kb + u < kn;
+                    const unsigned ko = (unsigned)((int)(k0 + kb + u) * sAk);
+                    ga[u] = ok && live0 ? __ldg(A + a0 + ko) : 0.f;
+                    gb[u] = ok && live1 ? __ldg(A + a1 + ko) : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const float *row = bsc + (kb + u) * SK_COLS;      // rows past the slice are zero
+#pragma unroll
+                    for (int q = 0; q < SK_COLS / 4; ++q) {
+                        const float4 b4 = *reinterpret_cast<const float4 *>(row + 4 * q);
+                        acc0[4 * q] = fmaf(ga[u], b4.x, acc0[4 * q]); acc0[4 * q + 1] = fmaf(ga[u], b4.y, acc0[4 * q + 1]);
+                        acc0[4 * q + 2] = fmaf(ga[u], b4.z, acc0[4 * q + 2]); acc0[4 * q + 3] = fmaf(ga[u], b4.w, acc0[4 * q + 3]);
+                        acc1[4 * q] = fmaf(gb[u], b4.x, acc1[4 * q]); acc1[4 * q + 1] = fmaf(gb[u], b4.y, acc1[4 * q + 1]);
+                        acc1[4 * q + 2] = fmaf(gb[u], b4.z, acc1[4 * q + 2]); acc1[4 * q + 3] = fmaf(gb[u], b4.w, acc1[4 * q + 3]);
+                    }
+                }
+            }
+        }
+        __syncthreads();
+    }
+    cp_async_wait<0>();
+    // ---- results ----
+    const bool partial = ksplit > 1;
+    float *__restrict__ out = partial ? ptrs.part : ptrs.out;
+    const int sOm = P.M.n_digits ? P.M.sO[0] : 0, sOn = P.N.n_digits ? P.N.sO[0] : 0;
+    auto store = [&](unsigned m, int n, float v) {
+        if (partial) out[((size_t)ks * Mext + m) * Next + (unsigned)n] = v;
+        else {
+            const unsigned off = (unsigned)(P.baseO + (int)m * sOm + n * sOn);
+            float r = epilogue(P, ptrs, v * P.scale, off);
+            if (P.accumulate) r += out[off];
+            out[off] = r;
+        }
+    };
+    if (along_k) {
+        // fixed-order butterfly over the lanes, then lane n stores column n
+#pragma unroll
+        for (int n = 0; n < SK_COLS; ++n) {
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) {
+                acc0[n] += __shfl_xor_sync(0xffffffffu, acc0[n], d);
+                acc1[n] += __shfl_xor_sync(0xffffffffu, acc1[n], d);
+            }
+        }
+#pragma unroll
+        for (int n = 0; n < SK_COLS; ++n) {
+            if ((unsigned)n < Next && (lane == (unsigned)(n & 31))) {
+                if (live0) store(m0, n, acc0[n]);
+                if (live1) store(m1, n, acc1[n]);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int n = 0; n < SK_COLS; ++n) {
+            if ((unsigned)n < Next) {
+                if (live0) store(m0, n, acc0[n]);
+                if (live1) store(m1, n, acc1[n]);
+            }
+        }
+    }
+}
+
 template <int BM, int BN, int TM, int TN>
 cudaError_t launch_shape(const TadcProgram &P, const TadpPointers &ptrs, cudaStream_t stream)
 {
@@ -512,6 +663,19 @@ cudaError_t launch_shape(const TadcProgram &P, const TadpPointers &ptrs, cudaStr
 cudaError_t tad_launch_contract(const TadcProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream)
 {
     if (P.M.extent <= 0 || P.N.extent <= 0 || P.Z.extent <= 0) return cudaSuccess;
+    if (P.shape == 5) {
+        const unsigned rows_per_block = P.modeA == TG_K ? 16u : 512u;
+        dim3 grid(((unsigned)P.M.extent + rows_per_block - 1u) / rows_per_block, (unsigned)std::max(1, P.ksplit), 1u);
+        tad_skinny_kernel<<<grid, 256, 0, stream>>>(P, ptrs);
+        cudaError_t e = cudaGetLastError();
+        if (e == cudaSuccess && P.ksplit > 1) {
+            const unsigned long long cells = (unsigned long long)P.M.extent * P.N.extent;
+            const unsigned blocks = (unsigned)std::min<unsigned long long>((cells + 255) / 256, (unsigned long long)sms * 8);
+            tad_contract_reduce<<<blocks, 256, 0, stream>>>(P, ptrs);
+            e = cudaGetLastError();
+        }
+        return e;
+    }
     if (P.shape == 4) {
         const unsigned warps = (unsigned)P.M.extent;
         const unsigned blocks = std::min((warps + 7u) / 8u, sms * 16u);

@@ -194,11 +194,35 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
         }
     }
     if (row_sums) { P.shape = 4; split = 1; }
+    // the streaming kernel for narrow contractions (see tad_skinny_kernel): one digit per group, B rows of consecutive,
+    // 16-byte aligned elements, A consecutive along k (128-bit loads) or along m
+    if (!row_sums && s.B.ptr >= 0 && !ga && !gb && P.Z.extent == 1 && P.N.extent >= 2 && P.N.extent <= 36 && P.M.n_digits == 1 &&
+        P.K.n_digits == 1 && P.N.n_digits == 1 && P.N.sB[0] == 1 && P.M.extent >= 512 && P.K.extent >= 512) {
+        const int64_t sBk = P.K.sB[0], sAk = P.K.sA[0], sAm = P.M.sA[0];
+        const bool b_ok = sBk > 0 && sBk % 4 == 0 && s.B.base % 4 == 0 && (P.N.extent % 4 == 0 || sBk >= (P.N.extent + 3) / 4 * 4);
+        const bool along_k = sAk == 1 && sAm % 4 == 0 && s.A.base % 4 == 0 && P.K.extent % 4 == 0;
+        const bool along_m = sAm == 1;
+        if (b_ok && (along_k || along_m)) {
+            P.shape = 5;
+            P.modeA = along_k ? TG_K : TG_ROW;
+            const int64_t row_blocks = along_k ? (P.M.extent + 15) / 16 : (P.M.extent + 511) / 512;
+            split = 1;
+            if (allow_split && row_blocks < 222) split = std::max<int64_t>(1, std::min<int64_t>(296 / row_blocks, P.K.extent / 512));
+            const int64_t cells = (int64_t)P.M.extent * P.N.extent;
+            while (split > 1 && split * cells > (int64_t(1) << 25)) --split;
+            const int64_t per128 = ((P.K.extent + split - 1) / split + 127) / 128 * 128;
+            P.kchunk = fit(per128);
+            P.ksplit = fit((P.K.extent + per128 - 1) / per128);
+        }
+    }
+    if (P.shape != 5) {
     split = std::max<int64_t>(1, split);
     const int64_t per = ((kstages + split - 1) / split) * TADC_BK;
     P.kchunk = fit(std::max<int64_t>(per, TADC_BK));
     P.ksplit = fit(std::max<int64_t>(1, (P.K.extent + P.kchunk - 1) / P.kchunk));
     if (P.ksplit <= 1) { P.ksplit = 1; P.kchunk = fit(std::max<int64_t>(kstages, 1) * TADC_BK); }
+    }
+    if (P.shape == 5 && P.ksplit <= 1) { P.ksplit = 1; P.kchunk = fit((P.K.extent + 127) / 128 * 128); }
     char line[320];
     auto group_text = [&](const char *name, const TadcGroup &G) {
         std::string t = std::string("  ") + name + ":";
@@ -210,7 +234,7 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     };
     std::snprintf(line, sizeof line, "; contraction %d x %d x %d (batch %d): A=ptr %d mode %d guard %d, B=ptr %d mode %d guard %d, tile %s, ksplit %d x %d, vec4 %d, scale %g, accumulate %d\n",
                   P.M.extent, P.N.extent, P.K.extent, P.Z.extent, P.ptrA, P.modeA, P.guardA, P.ptrB, P.modeB, P.guardB,
-                  P.shape == 4 ? "row sums" : P.shape == 3 ? "128x36" : P.shape == 2 ? "128x64" : "128x128", P.ksplit, P.kchunk, P.out_vec4, (double)P.scale, P.accumulate);
+                  P.shape == 5 ? "streamed" : P.shape == 4 ? "row sums" : P.shape == 3 ? "128x36" : P.shape == 2 ? "128x64" : "128x128", P.ksplit, P.kchunk, P.out_vec4, (double)P.scale, P.accumulate);
     text += line;
     text += group_text("m", P.M) + group_text("n", P.N) + group_text("k", P.K) + group_text("z", P.Z);
     return true;

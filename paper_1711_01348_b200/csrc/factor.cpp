@@ -54,6 +54,7 @@ struct Group {
     int a_inst = -1; uint32_t kmask = 0;
     std::vector<Request> reqs;
     int t_tensor = -1, x_tensor = -1;
+    int64_t cols = 0;                 // merged: columns in use (the tensors' rows are padded to whole 16-byte pieces)
     bool u_trick = false;             // single request on ones with the output indexed by the operand's own row
     int64_t u_g = 1, u0 = 0, u_ext = 0;
 };
@@ -771,8 +772,10 @@ static bool factor_kernel(Gen &g, Kernel &k, int root, int scale, bool allow_spl
             continue;
         }
         // merged: X[summed variables, column], T[row variables, column]
-        G.x_tensor = F.new_tensor(F.vars_of(G.kmask), cols);
-        G.t_tensor = F.new_tensor(F.vars_of(mmask), cols);
+        G.cols = cols;
+        const int64_t padded = (cols + 3) / 4 * 4;          // rows of whole 16-byte pieces (copied as such by the kernels)
+        G.x_tensor = F.new_tensor(F.vars_of(G.kmask), padded);
+        G.t_tensor = F.new_tensor(F.vars_of(mmask), padded);
         for (Request &r : G.reqs) {
             // the block's own variables index its columns, last variable fastest
             std::vector<int> nvars = F.vars_of(r.nmask);
@@ -968,7 +971,7 @@ static bool factor_kernel(Gen &g, Kernel &k, int root, int scale, bool allow_spl
                     const Tensor &X = F.tensors[G.x_tensor];
                     s.B.ptr = slot_of[G.x_tensor]; s.B.limit = X.elems; s.B.base = 0;
                     for (size_t d = 0; d < X.vars.size(); ++d) s.B.coef[X.vars[d]] = X.stride[d];
-                    s.vars[nv - 1] = AVar{X.cols, false};
+                    s.vars[nv - 1] = AVar{G.cols, false};
                     s.B.coef[nv - 1] = 1; s.O.coef[nv - 1] = 1;
                 } else if (G.reqs[0].b_atoms.empty()) s.B.ptr = -1;
                 else {
