@@ -348,6 +348,7 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
     const int n_epi = partial ? 0 : P.n_epi;
     const int obase = P.baseO + z.o;
     const bool vec_ok = partial ? (Next & 3u) == 0 : P.out_vec4 != 0;
+#pragma unroll 2
     for (unsigned e = tid; e < (unsigned)(BM * BN / 4); e += NT) {
         const unsigned rl = e / (BN / 4), cl = (e % (BN / 4)) * 4;
         const unsigned m = tile_m * BM + rl, n = tile_n * BN + cl;
@@ -361,8 +362,14 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
             for (int j = 0; j < 4; ++j) off[j] = o0 + j;
         } else {
             const int ob = obase + outM[rl];
+            if (vec_ok) {
+                const unsigned o0 = (unsigned)(ob + outN[cl]);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) { off[j] = (unsigned)(ob + outN[cl + j]); v[j] *= scale; }
+                for (int j = 0; j < 4; ++j) { off[j] = o0 + j; v[j] *= scale; }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { off[j] = (unsigned)(ob + outN[cl + j]); v[j] *= scale; }
+            }
         }
         const int live = (int)min(4u, Next - n);
         for (int s = 0; s < n_epi; ++s) {
@@ -540,25 +547,38 @@ tad_skinny_kernel(const __grid_constant__ TadcProgram P, const __grid_constant__
         }
         cp_async_commit();
     };
+    // A along k: the values of the next chunk are loaded while the current one is multiplied
+    float na[4] = {0.f, 0.f, 0.f, 0.f}, nb[4] = {0.f, 0.f, 0.f, 0.f};
+    auto load_a = [&](int chunk) {
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+            const unsigned k = kbeg + (unsigned)chunk * SK_KC + lane + 32u * kk;
+            const bool ok = chunk < n_chunks && k < kend;
+            na[kk] = (ok && live0) ? __ldg(A + a0 + k) : 0.f;
+            nb[kk] = (ok && live1) ? __ldg(A + a1 + k) : 0.f;
+        }
+    };
     issue(0);
+    if (along_k) load_a(0);
     for (int ch = 0; ch < n_chunks; ++ch) {
         issue(ch + 1);
+        float ga[4], gb[4];
+        if (along_k) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) { ga[kk] = na[kk]; gb[kk] = nb[kk]; }
+            load_a(ch + 1);
+        }
         cp_async_wait<1>();
         __syncthreads();
         const float *bsc = bs[ch & 1];
         const unsigned k0 = kbeg + (unsigned)ch * SK_KC;
         if (along_k) {
-            // lanes along k: this lane's four summation indices of the chunk, both rows
-            const unsigned k = k0 + lane * 4u;
-            float4 g0 = make_float4(0.f, 0.f, 0.f, 0.f), g1 = g0;
-            if (k < kend) {          // (slices are multiples of four long)
-                if (live0) g0 = __ldg(reinterpret_cast<const float4 *>(A + a0 + k));
-                if (live1) g1 = __ldg(reinterpret_cast<const float4 *>(A + a1 + k));
-            }
-            const float ga[4] = {g0.x, g0.y, g0.z, g0.w}, gb[4] = {g1.x, g1.y, g1.z, g1.w};
+            // lanes along k: lane l takes the summation indices l, l + 32, l + 64, l + 96 of the chunk for both rows
+            // (coalesced loads of A; the rows of B a warp reads at a time are consecutive, 36 words apart: no bank
+            // conflicts for its 128-bit loads)
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
-                const float *row = bsc + (lane * 4u + kk) * SK_COLS;
+                const float *row = bsc + (lane + 32u * kk) * SK_COLS;
 #pragma unroll
                 for (int q = 0; q < SK_COLS / 4; ++q) {
                     const float4 b4 = *reinterpret_cast<const float4 *>(row + 4 * q);
@@ -572,13 +592,13 @@ tad_skinny_kernel(const __grid_constant__ TadcProgram P, const __grid_constant__
             // lanes along m: every k of the chunk, the loads of A eight indices ahead of their use
             const int kn = (int)min((unsigned)SK_KC, kend - k0);
             for (int kb = 0; kb < kn; kb += 8) {
-                float ga[8], gb[8];
+                float ha[8], hb[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     const bool ok = kb + u < kn;
                     const unsigned ko = (unsigned)((int)(k0 + kb + u) * sAk);
-                    ga[u] = ok && live0 ? __ldg(A + a0 + ko) : 0.f;
-                    gb[u] = ok && live1 ? __ldg(A + a1 + ko) : 0.f;
+                    ha[u] = ok && live0 ? __ldg(A + a0 + ko) : 0.f;
+                    hb[u] = ok && live1 ? __ldg(A + a1 + ko) : 0.f;
                 }
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
@@ -586,10 +606,10 @@ tad_skinny_kernel(const __grid_constant__ TadcProgram P, const __grid_constant__
 #pragma unroll
                     for (int q = 0; q < SK_COLS / 4; ++q) {
                         const float4 b4 = *reinterpret_cast<const float4 *>(row + 4 * q);
-                        acc0[4 * q] = fmaf(ga[u], b4.x, acc0[4 * q]); acc0[4 * q + 1] = fmaf(ga[u], b4.y, acc0[4 * q + 1]);
-                        acc0[4 * q + 2] = fmaf(ga[u], b4.z, acc0[4 * q + 2]); acc0[4 * q + 3] = fmaf(ga[u], b4.w, acc0[4 * q + 3]);
-                        acc1[4 * q] = fmaf(gb[u], b4.x, acc1[4 * q]); acc1[4 * q + 1] = fmaf(gb[u], b4.y, acc1[4 * q + 1]);
-                        acc1[4 * q + 2] = fmaf(gb[u], b4.z, acc1[4 * q + 2]); acc1[4 * q + 3] = fmaf(gb[u], b4.w, acc1[4 * q + 3]);
+                        acc0[4 * q] = fmaf(ha[u], b4.x, acc0[4 * q]); acc0[4 * q + 1] = fmaf(ha[u], b4.y, acc0[4 * q + 1]);
+                        acc0[4 * q + 2] = fmaf(ha[u], b4.z, acc0[4 * q + 2]); acc0[4 * q + 3] = fmaf(ha[u], b4.w, acc0[4 * q + 3]);
+                        acc1[4 * q] = fmaf(hb[u], b4.x, acc1[4 * q]); acc1[4 * q + 1] = fmaf(hb[u], b4.y, acc1[4 * q + 1]);
+                        acc1[4 * q + 2] = fmaf(hb[u], b4.z, acc1[4 * q + 2]); acc1[4 * q + 3] = fmaf(hb[u], b4.w, acc1[4 * q + 3]);
                     }
                 }
             }

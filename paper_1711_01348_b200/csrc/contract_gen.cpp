@@ -200,7 +200,7 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
         P.K.n_digits == 1 && P.N.n_digits == 1 && P.N.sB[0] == 1 && P.M.extent >= 512 && P.K.extent >= 512) {
         const int64_t sBk = P.K.sB[0], sAk = P.K.sA[0], sAm = P.M.sA[0];
         const bool b_ok = sBk > 0 && sBk % 4 == 0 && s.B.base % 4 == 0 && (P.N.extent % 4 == 0 || sBk >= (P.N.extent + 3) / 4 * 4);
-        const bool along_k = sAk == 1 && sAm % 4 == 0 && s.A.base % 4 == 0 && P.K.extent % 4 == 0;
+        const bool along_k = sAk == 1;
         const bool along_m = sAm == 1;
         if (b_ok && (along_k || along_m)) {
             P.shape = 5;

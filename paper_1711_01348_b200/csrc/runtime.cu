@@ -122,8 +122,8 @@ tad_status launch_contractions(const tad::Kernel &k, const TadpPointers &ptrs, c
         if (P.modeA == TG_ROW16 && misaligned(ptrs.in[P.ptrA])) P.modeA = TG_ROW;
         if (P.ptrB >= 0 && P.modeB == TG_ROW16 && misaligned(ptrs.in[P.ptrB])) P.modeB = TG_ROW;
         if (P.out_vec4 && misaligned(ptrs.out)) P.out_vec4 = 0;
-        // the streaming kernel copies B in 16-byte pieces and, with A along k, loads A 16 bytes at a time
-        if (P.shape == 5 && (misaligned(ptrs.in[P.ptrB]) || (P.modeA == TG_K && misaligned(ptrs.in[P.ptrA])))) P.shape = 3;
+        // the streaming kernel copies B in 16-byte pieces
+        if (P.shape == 5 && misaligned(ptrs.in[P.ptrB])) P.shape = 3;
         const cudaError_t e = tad_launch_contract(P, ptrs, (unsigned)sm_count(), stream);
         if (e != cudaSuccess) { tad::set_error(std::string("contraction launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
     }
