@@ -348,85 +348,84 @@ tad_contract_kernel(const __grid_constant__ TadcProgram P, const __grid_constant
     const int n_epi = partial ? 0 : P.n_epi;
     const int obase = P.baseO + z.o;
     const bool vec_ok = partial ? (Next & 3u) == 0 : P.out_vec4 != 0;
-#pragma unroll 2
-    for (unsigned e = tid; e < (unsigned)(BM * BN / 4); e += NT) {
-        const unsigned rl = e / (BN / 4), cl = (e % (BN / 4)) * 4;
-        const unsigned m = tile_m * BM + rl, n = tile_n * BN + cl;
-        if (m >= Mext || n >= Next) continue;
-        const float4 s4 = *reinterpret_cast<const float4 *>(cs + rl * LDC + cl);
-        float v[4] = {s4.x, s4.y, s4.z, s4.w};
-        unsigned off[4];
-        if (partial) {
-            const unsigned o0 = (unsigned)(((zb * (unsigned)P.ksplit + ks) * Mext + m) * Next + n);     // < 2^25 cells per plane set
+    // four pieces of four columns per pass: every epilogue step is dispatched once for 16 values and the loads of a
+    // step (a tensor laid out like the output) are issued together
+    constexpr int EU = 4;
+    for (unsigned e0 = tid; e0 < (unsigned)(BM * BN / 4); e0 += NT * EU) {
+        float v[EU][4];
+        unsigned off[EU][4];
+        int live[EU];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) off[j] = o0 + j;
-        } else {
-            const int ob = obase + outM[rl];
-            if (vec_ok) {
-                const unsigned o0 = (unsigned)(ob + outN[cl]);
+        for (int u = 0; u < EU; ++u) {
+            const unsigned e = e0 + (unsigned)u * NT;
+            const unsigned rl = e / (BN / 4), cl = (e % (BN / 4)) * 4;
+            const unsigned m = tile_m * BM + rl, n = tile_n * BN + cl;
+            const bool in = e < (unsigned)(BM * BN / 4) && m < Mext && n < Next;
+            live[u] = in ? (int)min(4u, Next - n) : 0;
+            const float4 s4 = in ? *reinterpret_cast<const float4 *>(cs + rl * LDC + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
+            v[u][0] = s4.x; v[u][1] = s4.y; v[u][2] = s4.z; v[u][3] = s4.w;
+            if (partial) {
+                const unsigned o0 = (unsigned)(((zb * (unsigned)P.ksplit + ks) * Mext + m) * Next + n);     // < 2^25 cells per plane set
 #pragma unroll
-                for (int j = 0; j < 4; ++j) { off[j] = o0 + j; v[j] *= scale; }
+                for (int j = 0; j < 4; ++j) off[u][j] = in ? o0 + j : 0u;
             } else {
+                const int ob = obase + outM[in ? rl : 0];
+                if (vec_ok) {
+                    const unsigned o0 = (unsigned)(ob + outN[in ? cl : 0]);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) { off[j] = (unsigned)(ob + outN[cl + j]); v[j] *= scale; }
+                    for (int j = 0; j < 4; ++j) { off[u][j] = o0 + j; v[u][j] *= scale; }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) { off[u][j] = (unsigned)(ob + outN[in && j < live[u] ? cl + j : 0]); v[u][j] *= scale; }
+                }
             }
         }
-        const int live = (int)min(4u, Next - n);
+#define TAD_EPI_ALL(expr)                                               \
+    _Pragma("unroll") for (int u = 0; u < EU; ++u)                       \
+        _Pragma("unroll") for (int j = 0; j < 4; ++j) { expr; }
         for (int s = 0; s < n_epi; ++s) {
             const int op = P.epi_op[s];
             const float imm = P.epi_imm[s];
             const float *src = (op == TE_MUL_LOAD || op == TE_ADD_LOAD) ? ptrs.in[P.epi_ptr[s]] : nullptr;
             const int sb = P.epi_base[s];
             switch (op) {
-            case TE_NEG:
+            case TE_NEG: TAD_EPI_ALL(v[u][j] = -v[u][j]) break;
+            case TE_EXP: TAD_EPI_ALL(v[u][j] = __expf(v[u][j])) break;
+            case TE_MULC: TAD_EPI_ALL(v[u][j] *= imm) break;
+            case TE_ADDC: TAD_EPI_ALL(v[u][j] += imm) break;
+            case TE_SQR: TAD_EPI_ALL(v[u][j] *= v[u][j]) break;
+            case TE_TANH: TAD_EPI_ALL(v[u][j] = own_tanh(v[u][j])) break;
+            case TE_MUL_LOAD: case TE_ADD_LOAD: {
+                float w[EU][4];
+                if (vec_ok && ((sb & 3) == 0) && ((reinterpret_cast<uintptr_t>(src) & 15u) == 0)) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) v[j] = -v[j];
-                break;
-            case TE_EXP:
-#pragma unroll
-                for (int j = 0; j < 4; ++j) v[j] = __expf(v[j]);
-                break;
-            case TE_MULC:
-#pragma unroll
-                for (int j = 0; j < 4; ++j) v[j] *= imm;
-                break;
-            case TE_ADDC:
-#pragma unroll
-                for (int j = 0; j < 4; ++j) v[j] += imm;
-                break;
-            case TE_SQR:
-#pragma unroll
-                for (int j = 0; j < 4; ++j) v[j] *= v[j];
-                break;
-            case TE_TANH:
-#pragma unroll
-                for (int j = 0; j < 4; ++j) v[j] = own_tanh(v[j]);
-                break;
-            case TE_MUL_LOAD:
-                if (vec_ok && ((sb & 3) == 0)) {
-                    const float4 w4 = __ldg(reinterpret_cast<const float4 *>(src + (unsigned)(sb + (int)off[0])));
-                    v[0] *= w4.x; v[1] *= w4.y; v[2] *= w4.z; v[3] *= w4.w;
+                    for (int u = 0; u < EU; ++u) {
+                        const float4 w4 = live[u] ? __ldg(reinterpret_cast<const float4 *>(src + (unsigned)(sb + (int)off[u][0]))) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        w[u][0] = w4.x; w[u][1] = w4.y; w[u][2] = w4.z; w[u][3] = w4.w;
+                    }
                 } else {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) if (j < live) v[j] *= __ldg(src + (unsigned)(sb + (int)off[j]));
+                    TAD_EPI_ALL(w[u][j] = j < live[u] ? __ldg(src + (unsigned)(sb + (int)off[u][j])) : 0.f)
                 }
+                if (op == TE_MUL_LOAD) { TAD_EPI_ALL(v[u][j] *= w[u][j]) } else { TAD_EPI_ALL(v[u][j] += w[u][j]) }
                 break;
-            case TE_ADD_LOAD:
-#pragma unroll
-                for (int j = 0; j < 4; ++j) if (j < live) v[j] += __ldg(src + (unsigned)(sb + (int)off[j]));
-                break;
+            }
             default: break;
             }
         }
-        if (vec_ok) {
-            float4 *dst = reinterpret_cast<float4 *>(out + off[0]);
-            float4 r = make_float4(v[0], v[1], v[2], v[3]);
-            if (!partial && P.accumulate) { const float4 o = *dst; r.x += o.x; r.y += o.y; r.z += o.z; r.w += o.w; }
-            *dst = r;
-        } else {
+#undef TAD_EPI_ALL
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (j < live) out[off[j]] = (!partial && P.accumulate) ? v[j] + out[off[j]] : v[j];
+        for (int u = 0; u < EU; ++u) {
+            if (!live[u]) continue;
+            if (vec_ok) {
+                float4 *dst = reinterpret_cast<float4 *>(out + off[u][0]);
+                float4 r = make_float4(v[u][0], v[u][1], v[u][2], v[u][3]);
+                if (!partial && P.accumulate) { const float4 o = *dst; r.x += o.x; r.y += o.y; r.z += o.z; r.w += o.w; }
+                *dst = r;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (j < live[u]) out[off[u][j]] = (!partial && P.accumulate) ? v[u][j] + out[off[u][j]] : v[u][j];
+            }
         }
     }
 }
@@ -462,13 +461,39 @@ tad_rowsum_kernel(const __grid_constant__ TadcProgram P, const __grid_constant__
     const unsigned lane = threadIdx.x & 31u;
     const unsigned warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, n_warps = (gridDim.x * blockDim.x) >> 5;
     const float *__restrict__ A = ptrs.in[P.ptrA];
+    const bool weighted = P.ptrB >= 0;                   // B[k]: one weight per summation index
+    const float *__restrict__ B = weighted ? ptrs.in[P.ptrB] : A;
+    const int kb = P.K.n_digits ? P.K.sB[0] : 0;
     const unsigned K = (unsigned)P.K.extent;
     const int ks = P.K.n_digits ? P.K.sA[0] : 0;
     for (unsigned m = warp; m < (unsigned)P.M.extent; m += n_warps) {
         const Parts p = decode(P.M, m);
         const int base = P.baseA + p.a;
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-        if (ks == 1 && ((base & 3) == 0) && ((reinterpret_cast<uintptr_t>(A) & 15u) == 0)) {
+        if (weighted && ks == 1 && kb == 1 && ((base & 3) == 0) && ((P.baseB & 3) == 0) &&
+            (((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B)) & 15u) == 0)) {
+            const float4 *row = reinterpret_cast<const float4 *>(A + (unsigned)base);
+            const float4 *wts = reinterpret_cast<const float4 *>(B + (unsigned)P.baseB);
+            const unsigned K4 = K / 4;
+            unsigned k = lane;
+            for (; k + 96 < K4; k += 128) {
+                const float4 a = __ldg(row + k), b = __ldg(row + k + 32), c = __ldg(row + k + 64), d = __ldg(row + k + 96);
+                const float4 wa = __ldg(wts + k), wb = __ldg(wts + k + 32), wc = __ldg(wts + k + 64), wd = __ldg(wts + k + 96);
+                s0 += (a.x * wa.x + a.y * wa.y) + (a.z * wa.z + a.w * wa.w); s1 += (b.x * wb.x + b.y * wb.y) + (b.z * wb.z + b.w * wb.w);
+                s2 += (c.x * wc.x + c.y * wc.y) + (c.z * wc.z + c.w * wc.w); s3 += (d.x * wd.x + d.y * wd.y) + (d.z * wd.z + d.w * wd.w);
+            }
+            for (; k < K4; k += 32) { const float4 a = __ldg(row + k), wa = __ldg(wts + k); s0 += (a.x * wa.x + a.y * wa.y) + (a.z * wa.z + a.w * wa.w); }
+            for (unsigned t = K4 * 4 + lane; t < K; t += 32) s1 = fmaf(__ldg(A + (unsigned)(base + (int)t)), __ldg(B + (unsigned)(P.baseB + (int)t)), s1);
+        } else if (weighted) {
+            unsigned k = lane;
+            for (; k + 96 < K; k += 128) {
+                s0 = fmaf(__ldg(A + (unsigned)(base + (int)k * ks)), __ldg(B + (unsigned)(P.baseB + (int)k * kb)), s0);
+                s1 = fmaf(__ldg(A + (unsigned)(base + (int)(k + 32) * ks)), __ldg(B + (unsigned)(P.baseB + (int)(k + 32) * kb)), s1);
+                s2 = fmaf(__ldg(A + (unsigned)(base + (int)(k + 64) * ks)), __ldg(B + (unsigned)(P.baseB + (int)(k + 64) * kb)), s2);
+                s3 = fmaf(__ldg(A + (unsigned)(base + (int)(k + 96) * ks)), __ldg(B + (unsigned)(P.baseB + (int)(k + 96) * kb)), s3);
+            }
+            for (; k < K; k += 32) s0 = fmaf(__ldg(A + (unsigned)(base + (int)k * ks)), __ldg(B + (unsigned)(P.baseB + (int)k * kb)), s0);
+        } else if (ks == 1 && ((base & 3) == 0) && ((reinterpret_cast<uintptr_t>(A) & 15u) == 0)) {
             const float4 *row = reinterpret_cast<const float4 *>(A + (unsigned)base);
             const unsigned K4 = K / 4;
             unsigned k = lane;
@@ -658,6 +683,48 @@ tad_skinny_kernel(const __grid_constant__ TadcProgram P, const __grid_constant__
     }
 }
 
+// Plain or weighted sums of an operand that is consecutive along its row index:
+//     out[m] = sum_k A[m + k * stride] (* B[k]),   a thread per m, a slice of k per block row (grid.y);
+// consecutive threads read consecutive elements, four loads in flight per thread.  Slices write planes of
+// partial sums that tad_contract_reduce adds in order.
+__global__ void __launch_bounds__(256)
+tad_colsum_kernel(const __grid_constant__ TadcProgram P, const __grid_constant__ TadpPointers ptrs)
+{
+    const unsigned m = blockIdx.x * 256u + threadIdx.x;
+    const unsigned Mext = (unsigned)P.M.extent, K = (unsigned)P.K.extent;
+    if (m >= Mext) return;
+    const float *__restrict__ A = ptrs.in[P.ptrA];
+    const bool weighted = P.ptrB >= 0;
+    const float *__restrict__ B = weighted ? ptrs.in[P.ptrB] : A;
+    const int ks = P.K.sA[0], kb = P.K.sB[0];
+    const unsigned kbeg = blockIdx.y * (unsigned)P.kchunk, kend = min(K, kbeg + (unsigned)P.kchunk);
+    const int base = P.baseA + (int)m * P.M.sA[0];
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    unsigned k = kbeg;
+    for (; k + 7 < kend; k += 8) {
+        float a[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) a[u] = __ldg(A + (unsigned)(base + (int)(k + u) * ks));
+        if (weighted) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) a[u] *= __ldg(B + (unsigned)(P.baseB + (int)(k + u) * kb));
+        }
+        s0 += a[0] + a[4]; s1 += a[1] + a[5]; s2 += a[2] + a[6]; s3 += a[3] + a[7];
+    }
+    for (; k < kend; ++k) {
+        const float a0 = __ldg(A + (unsigned)(base + (int)k * ks));
+        s0 = weighted ? fmaf(a0, __ldg(B + (unsigned)(P.baseB + (int)k * kb)), s0) : s0 + a0;
+    }
+    const float s = (s0 + s1) + (s2 + s3);
+    if (P.ksplit > 1) ptrs.part[(size_t)blockIdx.y * Mext + m] = s;
+    else {
+        const unsigned off = (unsigned)(P.baseO + (int)m * P.M.sO[0]);
+        float v = s * P.scale;
+        if (P.accumulate) v += ptrs.out[off];
+        ptrs.out[off] = v;
+    }
+}
+
 template <int BM, int BN, int TM, int TN>
 cudaError_t launch_shape(const TadcProgram &P, const TadpPointers &ptrs, cudaStream_t stream)
 {
@@ -696,13 +763,25 @@ cudaError_t tad_launch_contract(const TadcProgram &P, const TadpPointers &ptrs, 
         }
         return e;
     }
+    if (P.shape == 6) {
+        dim3 grid(((unsigned)P.M.extent + 255u) / 256u, (unsigned)std::max(1, P.ksplit), 1u);
+        tad_colsum_kernel<<<grid, 256, 0, stream>>>(P, ptrs);
+        cudaError_t e = cudaGetLastError();
+        if (e == cudaSuccess && P.ksplit > 1) {
+            const unsigned blocks = (unsigned)std::min<unsigned long long>(((unsigned long long)P.M.extent + 255) / 256, (unsigned long long)sms * 8);
+            tad_contract_reduce<<<blocks, 256, 0, stream>>>(P, ptrs);
+            e = cudaGetLastError();
+        }
+        return e;
+    }
     if (P.shape == 4) {
         const unsigned warps = (unsigned)P.M.extent;
         const unsigned blocks = std::min((warps + 7u) / 8u, sms * 16u);
         tad_rowsum_kernel<<<blocks, 256, 0, stream>>>(P, ptrs);
         return cudaGetLastError();
     }
-    cudaError_t e = P.shape == 3 ? launch_shape<128, 36, 8, 4>(P, ptrs, stream)
+    cudaError_t e = P.shape == 1 ? launch_shape<128, 32, 8, 4>(P, ptrs, stream)
+                  : P.shape == 3 ? launch_shape<128, 36, 8, 4>(P, ptrs, stream)
                   : P.shape == 2 ? launch_shape<128, 64, 8, 4>(P, ptrs, stream) : launch_shape<128, 128, 8, 8>(P, ptrs, stream);
     if (e != cudaSuccess) return e;
     if (P.ksplit > 1) {

@@ -49,7 +49,8 @@ struct alignas(16) TadcProgram {
     int32_t kchunk;                // summation indices per chunk (a multiple of TADC_BK)
     int32_t accumulate;            // 1: out += result
     int32_t out_vec4;              // 1: four consecutive n are four consecutive, 16-byte aligned output elements
-    int32_t shape;                 // 0 = 128 x 128 tile (8 x 8 per thread), 2 = 128 x 64 (8 x 4), 3 = 128 x 36 (8 x 4), 4 = plain row sums (one warp per output)
+    int32_t shape;                 // tiles: 0 = 128 x 128 (8 x 8 per thread), 1 = 128 x 32, 2 = 128 x 64, 3 = 128 x 36 (8 x 4 per thread);
+                                   // 4 = sums of rows (a warp per output), 5 = streamed narrow contraction, 6 = sums of columns (a thread per output)
     float scale;
     int32_t n_epi;
     int32_t epi_op[TADC_MAX_EPI];

@@ -60,7 +60,9 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     for (int v = 0; v < nv; ++v)
         if (!s.vars[v].reduce && s.O.coef[v] != 0 && s.vars[v].ext > 1 &&
             (contiguous < 0 || std::llabs(s.O.coef[v]) < std::llabs(s.O.coef[contiguous]))) contiguous = v;
-    if (contiguous >= 0 && s.A.coef[contiguous] != 0 && s.B.coef[contiguous] == 0 && s.B.ptr >= 0) std::swap(s.A, s.B);
+    bool b_has_rows = false;                               // B reads some variable that is not summed
+    for (int v = 0; v < nv; ++v) if (!s.vars[v].reduce && s.vars[v].ext > 1 && s.B.coef[v] != 0) b_has_rows = true;
+    if (contiguous >= 0 && s.A.coef[contiguous] != 0 && s.B.coef[contiguous] == 0 && s.B.ptr >= 0 && b_has_rows) std::swap(s.A, s.B);
     std::vector<Digit> dm, dn, dk, dz;
     for (int v = 0; v < nv; ++v) {
         if (s.vars[v].ext == 1) continue;                  // a single value: nothing to index
@@ -126,12 +128,16 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     P.guardB = gb ? 1 : 0; P.guardB_c0 = gb ? fit(gb->c0) : 0; P.guardB_ext = gb ? fit(gb->ext) : 1;
     P.scale = scale; P.accumulate = accumulate;
     // tile shape: narrow column tiles for narrow outputs
-    P.shape = P.N.extent <= 36 ? 3 : P.N.extent <= 64 ? 2 : 0;
-    const int64_t BM = 128, BN = P.shape == 3 ? 36 : P.shape == 2 ? 64 : 128;
+    P.shape = P.N.extent <= 32 ? 1 : P.N.extent <= 36 ? 3 : P.N.extent <= 64 ? 2 : 0;
+    const int64_t BM = 128, BN = P.shape == 1 ? 32 : P.shape == 3 ? 36 : P.shape == 2 ? 64 : 128;
     const int64_t tiles_m = (P.M.extent + BM - 1) / BM, tiles_n = (P.N.extent + BN - 1) / BN;
     const double fill = (double)P.M.extent * P.N.extent / ((double)tiles_m * BM * tiles_n * BN);
-    const bool row_sums = s.B.ptr < 0 && P.N.extent == 1 && P.Z.extent == 1 && P.K.n_digits <= 1 && !P.guardA && P.M.extent >= 1024;
-    if (!row_sums && fill < (strict_fill ? 0.15 : 0.05)) return false;    // mostly empty tiles: the interpreter's schedules do better
+    // one output column: plain or weighted sums of A (B is ones or a vector over k), run at memory speed by a warp
+    // per row (A along k) or a thread per row (A along m)
+    const bool one_column = P.N.extent == 1 && P.Z.extent == 1 && P.K.n_digits <= 1 && !P.guardA && !P.guardB && P.M.extent >= 1024;
+    const bool col_sums = one_column && P.M.n_digits == 1 && P.M.sA[0] == 1 && P.K.n_digits == 1 && std::llabs((int64_t)P.K.sA[0]) != 1;
+    const bool row_sums = one_column && !col_sums;
+    if (!one_column && fill < (strict_fill ? 0.15 : 0.05)) return false;    // mostly empty tiles: the interpreter's schedules do better
     // gather modes: the one whose warp-wide copy touches fewer 128-byte lines (lanes along the row index:
     // 32 rows at one summation index; lanes along the summation index: 2 rows x 16 indices)
     auto mode_of = [&](const std::vector<Digit> &rows, bool second, const AGuard *gd, int64_t base) {
@@ -194,13 +200,26 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
         }
     }
     if (row_sums) { P.shape = 4; split = 1; }
+    if (col_sums) {
+        // a thread per row, blocks of 256 rows: the summation is split to fill the GPU
+        P.shape = 6;
+        const int64_t row_blocks = (P.M.extent + 255) / 256;
+        split = allow_split ? std::max<int64_t>(1, std::min<int64_t>((592 + row_blocks - 1) / row_blocks, P.K.extent / 64)) : 1;
+        const int64_t cells = (int64_t)P.M.extent;
+        while (split > 1 && split * cells > (int64_t(1) << 25)) --split;
+        const int64_t per = (P.K.extent + split - 1) / split;
+        P.kchunk = fit(std::max<int64_t>(per, 1));
+        P.ksplit = fit((P.K.extent + P.kchunk - 1) / P.kchunk);
+    }
     // the streaming kernel for narrow contractions (see tad_skinny_kernel): one digit per group, B rows of consecutive,
     // 16-byte aligned elements, A consecutive along k (128-bit loads) or along m
-    if (!row_sums && s.B.ptr >= 0 && !ga && !gb && P.Z.extent == 1 && P.N.extent >= 2 && P.N.extent <= 36 && P.M.n_digits == 1 &&
+    if (!one_column && s.B.ptr >= 0 && !ga && !gb && P.Z.extent == 1 && P.N.extent >= 2 && P.N.extent <= 36 && P.M.n_digits == 1 &&
         P.K.n_digits == 1 && P.N.n_digits == 1 && P.N.sB[0] == 1 && P.M.extent >= 512 && P.K.extent >= 512) {
         const int64_t sBk = P.K.sB[0], sAk = P.K.sA[0], sAm = P.M.sA[0];
         const bool b_ok = sBk > 0 && sBk % 4 == 0 && s.B.base % 4 == 0 && (P.N.extent % 4 == 0 || sBk >= (P.N.extent + 3) / 4 * 4);
-        const bool along_k = sAk == 1;
+        // (A along k is left to the tiles: with the lanes along k every lane reads its own rows of B from shared
+        // memory, which that memory cannot deliver at the rate of the multiply-adds; the kernel keeps the path)
+        const bool along_k = false && sAk == 1;
         const bool along_m = sAm == 1;
         if (b_ok && (along_k || along_m)) {
             P.shape = 5;
@@ -215,7 +234,7 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
             P.ksplit = fit((P.K.extent + per128 - 1) / per128);
         }
     }
-    if (P.shape != 5) {
+    if (P.shape != 5 && P.shape != 6) {
     split = std::max<int64_t>(1, split);
     const int64_t per = ((kstages + split - 1) / split) * TADC_BK;
     P.kchunk = fit(std::max<int64_t>(per, TADC_BK));
@@ -234,7 +253,7 @@ bool emit_program(const System &s0, float scale, int accumulate, bool allow_spli
     };
     std::snprintf(line, sizeof line, "; contraction %d x %d x %d (batch %d): A=ptr %d mode %d guard %d, B=ptr %d mode %d guard %d, tile %s, ksplit %d x %d, vec4 %d, scale %g, accumulate %d\n",
                   P.M.extent, P.N.extent, P.K.extent, P.Z.extent, P.ptrA, P.modeA, P.guardA, P.ptrB, P.modeB, P.guardB,
-                  P.shape == 5 ? "streamed" : P.shape == 4 ? "row sums" : P.shape == 3 ? "128x36" : P.shape == 2 ? "128x64" : "128x128", P.ksplit, P.kchunk, P.out_vec4, (double)P.scale, P.accumulate);
+                  P.shape == 6 ? "column sums" : P.shape == 5 ? "streamed" : P.shape == 4 ? "row sums" : P.shape == 1 ? "128x32" : P.shape == 3 ? "128x36" : P.shape == 2 ? "128x64" : "128x128", P.ksplit, P.kchunk, P.out_vec4, (double)P.scale, P.accumulate);
     text += line;
     text += group_text("m", P.M) + group_text("n", P.N) + group_text("k", P.K) + group_text("z", P.Z);
     return true;

@@ -706,6 +706,31 @@ static bool factor_kernel(Gen &g, Kernel &k, int root, int scale, bool allow_spl
     }
 
     // ---- layouts of the merged contractions ----
+    // A group a few columns wider than 32 gives its single columns (plain and weighted sums of the streamed
+    // operand) to passes of their own: those run at memory speed, and the rest fits the 32-column tile exactly
+    // instead of padding every tile to the next width.
+    for (size_t gi = 0, n_groups = F.groups.size(); gi < n_groups; ++gi) {
+        auto width = [&](const Request &r) { int64_t wd = 1; for (int v = 0; v < TADP_MAX_VARS; ++v) if (r.nmask & (1u << v)) wd *= F.vext[v]; return wd; };
+        int64_t total = 0;
+        for (const Request &r : F.groups[gi].reqs) total += width(r);
+        if (total <= 32 || total > 40) continue;
+        // (an operand that is consecutive along its rows takes the streaming kernel, which holds 36 columns)
+        {
+            const TadpLoad &LA = w.loads[w.inst[F.groups[gi].a_inst].load];
+            bool along_rows = false;
+            for (int v = 0; v < TADP_MAX_VARS; ++v) if (!(F.groups[gi].kmask & (1u << v)) && std::abs(LA.coef[v]) == 1 && F.vext[v] > 1) along_rows = true;
+            if (along_rows && total <= 36) continue;
+        }
+        for (size_t ri = 0; ri < F.groups[gi].reqs.size() && total > 32;) {
+            const Request r = F.groups[gi].reqs[ri];
+            const bool single = width(r) == 1 && (r.b_atoms.empty() || (r.b_atoms.size() == 1 && F.is_plain_load(r.b_atoms[0])));
+            if (!single) { ++ri; continue; }
+            Group G; G.a_inst = F.groups[gi].a_inst; G.kmask = F.groups[gi].kmask; G.reqs.push_back(r);
+            F.groups[gi].reqs.erase(F.groups[gi].reqs.begin() + ri);
+            F.groups.push_back(G);
+            total -= 1;
+        }
+    }
     const int slot0 = p.n_args + 1 + (int)p.stages.size();
     const int max_aux = (p.opt.saved_forward ? TADP_F_SLOT : TADP_MAX_PTRS) - slot0;
     for (size_t gi = 0; gi < F.groups.size(); ++gi) {

@@ -253,7 +253,9 @@ def test_kernel_stats_and_listing():
     # factored gradient: its contractions stream the staged adjoint once (three column blocks of one matrix)
     assert st.terms == 8192 * 8192 * 32 and st.n_launches >= 4
     dc = plan.disassemble(q["c"])
-    assert dc.count("; contraction") == 1 and "8192 x 34 x 8192" in dc
+    # one 32-column contraction with b, and the two single columns (plain row sums and row sums weighted by
+    # sum_k b_jk^2) as passes of their own at memory speed
+    assert dc.count("; contraction") == 3 and "8192 x 32 x 8192" in dc and dc.count("row sums") == 2
     # dd: the sum over j of the staged adjoint is a row sum, indexed by the row and not by (beta, z)
     dd = plan.disassemble(q["d"])
     assert "; contraction 8192 x 1 x 8192" in dd and "ZLOOP" in dd
