@@ -693,6 +693,8 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     if (try_contraction(g, k, root, scale, allow_split, lower, upper, guards)) return;
     // sums that can be pushed inside the term (Sec. 6's missing clean-up step): auxiliary kernels + a smaller kernel
     if (may_factor && try_factoring(g, k, root, scale, allow_split, lower, upper, guards)) return;
+    // sums of products of index expressions (most derivative terms once the functions are tabulated)
+    if (try_line(g, k, root, scale, allow_split, lower, upper, guards)) return;
     // a short loop whose range shifts from lane to lane will be walked relative to every element's own
     // start, which needs the elements of a thread to lie along the lane variable only
     bool relative_candidate = false;
@@ -1014,7 +1016,7 @@ void emit_plain_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vecto
 static void account(tad_plan &p, Kernel &k)
 {
     std::function<void(const Kernel &)> walk = [&](const Kernel &x) {
-        if (x.ew.empty() && x.contract.empty() && x.prog.zsplit > 1)
+        if (x.ew.empty() && x.contract.empty() && x.prog.zsplit > 1)   // (line-sum kernels keep their shares in prog too)
             p.partial_bytes = std::max(p.partial_bytes, (size_t(x.prog.zsplit) + 1) * size_t(x.prog.part_limit) * 4);
         for (const TadcProgram &cp : x.contract)
             if (cp.ksplit > 1)
@@ -1026,7 +1028,7 @@ static void account(tad_plan &p, Kernel &k)
     std::function<int(const Kernel &)> launches = [&](const Kernel &x) {
         int n = 0;
         if (!x.ew.empty()) n = 1;
-        else if (x.contract.empty()) n = 1 + (x.prog.zsplit > 1 ? 1 + (x.prog.write_only_live ? 1 : 0) : 0);
+        else if (x.contract.empty()) n = 1 + (x.prog.zsplit > 1 ? 1 + (x.prog.write_only_live && x.line.empty() ? 1 : 0) : 0);
         for (const TadcProgram &cp : x.contract) n += 1 + (cp.ksplit > 1 ? 1 : 0);
         for (const Kernel &y : x.pre) n += launches(y);
         return n;

@@ -73,6 +73,7 @@ struct Factorizer {
     bool changed = false;
     bool allow_sums = true;                           // false: only function tables (kernels with guards)
     int n_outer_vars = 0;
+    bool has_loops = false;                           // the kernel has summation loops around its term
     std::map<int, int> table_memo;                    // instance -> load of its table
 
     Factorizer(Gen &gen, Kernel &kern) : w(gen), k(kern), nv0((int)gen.vars.size()), vlo(TADP_MAX_VARS, 0), vext(TADP_MAX_VARS, 1), can_sum(TADP_MAX_VARS, false) {}
@@ -392,7 +393,10 @@ struct Factorizer {
         // evaluated again for every output that runs the loop
         uint32_t reach = w.inst[i].deps;
         if (reach >> n_outer_vars) reach |= (1u << n_outer_vars) - 1u;
-        if (L.limit <= 0 || (double)L.limit * 8.0 > space(reach) || L.limit > (1 << 26)) return -1;
+        // a kernel with summation loops also tabulates the factors outside its sums when the table is not much
+        // larger than the number of outputs: its terms are then products of index expressions (line sums)
+        const double worth = (has_loops && !(w.inst[i].deps >> n_outer_vars)) ? 0.5 : 8.0;
+        if (L.limit <= 0 || (double)L.limit * worth > space(reach) || L.limit > (1 << 26)) return -1;
         Tensor T; T.cols = 1; T.elems = L.limit;
         tensors.push_back(T);
         const int t = (int)tensors.size() - 1;
@@ -528,6 +532,7 @@ static bool factor_kernel(Gen &g, Kernel &k, int root, int scale, bool allow_spl
     Factorizer F(w, k);
     F.allow_sums = guards.empty();
     F.n_outer_vars = g.n_outer;
+    F.has_loops = g.kappa >= 1;
     const TadpProgram &prog = k.prog;
     for (int v = 0; v < g.n_outer; ++v) { F.vlo[v] = prog.outer_lo[v]; F.vext[v] = prog.outer_ext[v]; }
     // kernel-coordinate loops with fixed ranges that no other loop's bounds read can be summed away
@@ -1085,9 +1090,9 @@ static bool factor_kernel(Gen &g, Kernel &k, int root, int scale, bool allow_spl
     }
     g3.lane_var = lane;
     Kernel main = k;
-    main.pre.clear(); main.contract.clear(); main.ew.clear();
+    main.pre.clear(); main.contract.clear(); main.ew.clear(); main.line.clear();
     emit_plain_kernel(g3, main, root3, lower3, upper3, guards3, allow_split);
-    k.prog = main.prog; k.vec = main.vec; k.vec_u = main.vec_u; k.rich = main.rich; k.contract = main.contract; k.ew = main.ew;
+    k.prog = main.prog; k.vec = main.vec; k.vec_u = main.vec_u; k.rich = main.rich; k.contract = main.contract; k.ew = main.ew; k.line = main.line;
     k.listing = text + main.listing;
     k.pre = pre;
     return true;

@@ -343,6 +343,9 @@ bool emit_program(const System &s, float scale, int accumulate, bool allow_split
 bool try_contraction(Gen &g, Kernel &k, int root, int scale, bool allow_split, const std::vector<std::vector<TadpRow>> &lower,
                      const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards);
 
+// line_gen.cpp: a gradient kernel whose term is a product of index expressions becomes a line-sum program
+bool try_line(Gen &g, Kernel &k, int root, int scale, bool allow_split, const std::vector<std::vector<TadpRow>> &lower,
+              const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards);
 // factor.cpp: the expression optimisation pass; fills k.pre / k.aux and emits the kernel itself when it
 // finds summations worth pushing inside the term, returns false (k untouched) otherwise
 bool try_factoring(Gen &g, Kernel &k, int root, int scale, bool allow_split, const std::vector<std::vector<TadpRow>> &lower,

@@ -10,6 +10,7 @@
 #include "program.h"
 #include "contract.h"
 #include "ew.h"
+#include "line.h"
 
 namespace tad {
 
@@ -72,6 +73,7 @@ struct Kernel {
     std::vector<TadcProgram> contract;   // non-empty: the kernel is a contraction, run by the tile kernel (one launch per
                                          // program) instead of the interpreter
     std::vector<TadeProgram> ew;         // non-empty: a kernel without loops, run by the element-wise kernel
+    std::vector<TadlProgram> line;       // non-empty: sums of products of index expressions, run by the line-sum kernel
     // Expression optimisation: tensors in the auxiliary area of the workspace and the kernels that fill them
     // (launched in this order before the kernel itself, each writing the tensor out_aux)
     struct Aux { size_t offset = 0, bytes = 0; int slot = 0; };

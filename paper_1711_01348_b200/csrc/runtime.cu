@@ -22,6 +22,7 @@ TAD_VM_SHAPES(TAD_DECLARE_VM)
 void tad_launch_vm_16_1_rich(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream);
 cudaError_t tad_launch_contract(const TadcProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream);
 cudaError_t tad_launch_ew(const TadeProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream);
+cudaError_t tad_launch_line(const TadlProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream);
 
 namespace {
 
@@ -147,6 +148,19 @@ tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStrea
     if (!k.ew.empty()) {
         const cudaError_t e = tad_launch_ew(k.ew[0], ptrs, (unsigned)sm_count(), stream);
         if (e != cudaSuccess) { tad::set_error(std::string("element-wise launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
+        return TAD_OK;
+    }
+    if (!k.line.empty()) {
+        const TadlProgram &L = k.line[0];
+        if (L.zsplit > 1 && !ptrs.part) { tad::set_error("internal: partial-sum buffer missing"); return TAD_ERR_WORKSPACE; }
+        cudaError_t e = tad_launch_line(L, ptrs, (unsigned)sm_count(), stream);
+        if (e == cudaSuccess && L.zsplit > 1) {
+            const unsigned n = (unsigned)k.prog.part_limit;
+            const unsigned rblocks = std::min((n + 31u) / 32u, (unsigned)sm_count() * 8u);
+            tad_reduce_partials<<<rblocks, REDUCE_WARPS * 32, 0, stream>>>(k.prog, ptrs.out, ptrs.part);
+            e = cudaGetLastError();
+        }
+        if (e != cudaSuccess) { tad::set_error(std::string("line-sum launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
         return TAD_OK;
     }
     const int zsplit = k.prog.zsplit > 1 ? k.prog.zsplit : 1;
