@@ -154,6 +154,216 @@ tad_ew_kernel(const __grid_constant__ TadeProgram P, const __grid_constant__ Tad
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------------------
+// Products of loads.  Most element-wise kernels that remain after the function tables are
+//     out = c * L_1^e1 * L_2^e2 * ...        (e in 1..3),
+// and at one multiplication per load the index arithmetic of the general program dominates.  Here a thread
+// owns four outputs of a row and walks a run of consecutive rows along another outer variable, so the
+// variables are decoded once per run and every offset advances by a constant per row.  Two layouts:
+//   vector:      the four outputs are consecutive; every load that moves along the row is a 128-bit load
+//                (forward, or reversed for offsets that step by -1), which the host has proven aligned in every row;
+//   interleaved: output j of a thread lies j * (threads per row) further, so that plain loads of neighbouring
+//                threads fall into the same lines whatever the load's step.
+// Loads that do not change from row to row are read once per run, loads that do not move along the row once per row.
+// ---------------------------------------------------------------------------------------------------------
+enum ProdKind : int { PK_HOIST = 0, PK_BCAST, PK_FWD, PK_REV, PK_GEN };
+
+struct ProdLoad { int32_t load, kind, exp; };
+struct ProdPlan {
+    int32_t n_loads, row_var, run, vec;      // run: rows per thread along row_var (row_var < 0: single rows)
+    float c;
+    ProdLoad ld[4];
+};
+
+__device__ __forceinline__ float powe(float v, int e) { return e == 1 ? v : e == 2 ? v * v : v * v * v; }
+
+template <bool VEC>
+__global__ void __launch_bounds__(256)
+tad_prod_kernel(const __grid_constant__ TadeProgram P, const __grid_constant__ ProdPlan Q, const __grid_constant__ TadpPointers ptrs,
+                const unsigned n_items, const unsigned cols, const unsigned lane_blocks, const unsigned n_runs, const unsigned runs_per_line)
+{
+    const unsigned tid = threadIdx.x;
+    const unsigned rows_per_block = 256u / cols;
+    const unsigned tc = tid % cols, tr = tid / cols;
+    const int lane_var = P.lane_var, row_var = Q.row_var;
+    const unsigned lane_ext = (unsigned)P.outer_ext[lane_var];
+    const unsigned es = VEC ? 1u : cols;                       // distance between two outputs of a thread
+    float *__restrict__ out = ptrs.out;
+    for (unsigned item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const unsigned lb = item % lane_blocks, rb = item / lane_blocks;
+        const unsigned run = rb * rows_per_block + tr;
+        const unsigned lane0 = lb * cols * 4u + (VEC ? tc * 4u : tc);
+        if (run >= n_runs || lane0 >= lane_ext) continue;
+        int live;                                              // outputs of this thread inside the row
+        if (VEC) live = (int)min(4u, lane_ext - lane0);
+        else live = (int)min(4u, (lane_ext - lane0 + cols - 1u) / cols);
+        // the run: its position along row_var, then the other outer variables
+        const unsigned piece = run % runs_per_line;
+        unsigned rem = run / runs_per_line;
+        int var[TADP_MAX_VARS];
+#pragma unroll
+        for (int v = TADP_MAX_VARS - 1; v >= 0; --v) {
+            var[v] = 0;
+            if (v < P.n_outer) {
+                if (v == lane_var) var[v] = P.outer_lo[v] + (int)lane0;
+                else if (v == row_var) var[v] = P.outer_lo[v] + (int)(piece * (unsigned)Q.run);
+                else {
+                    const unsigned q = (unsigned)(((unsigned long long)rem * (unsigned)P.div_mul[v]) >> P.div_shift[v]);
+                    var[v] = P.outer_lo[v] + (int)(rem - q * (unsigned)P.outer_ext[v]);
+                    rem = q;
+                }
+            }
+        }
+        const int n_rows = row_var < 0 ? 1 : min(Q.run, P.outer_ext[row_var] - (int)(piece * (unsigned)Q.run));
+        int off[4], step[4], adv[4];
+        float held[4][4];
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+            off[l] = 0; step[l] = 0; adv[l] = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) held[l][j] = 1.f;
+            if (l < Q.n_loads) {
+                const TadpLoad &L = P.loads[Q.ld[l].load];
+                int o = L.base;
+#pragma unroll
+                for (int v = 0; v < TADP_MAX_VARS; ++v) o += L.coef[v] * var[v];
+                off[l] = o; step[l] = L.coef[lane_var] * (int)es; adv[l] = row_var < 0 ? 0 : L.coef[row_var];
+                if (Q.ld[l].kind == PK_HOIST) {
+                    const float *__restrict__ src = ptrs.in[L.ptr];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) if (j < live) held[l][j] = powe(__ldg(src + (unsigned)(o + j * step[l])), Q.ld[l].exp);
+                }
+            }
+        }
+        int oo = P.out_base;
+#pragma unroll
+        for (int v = 0; v < TADP_MAX_VARS; ++v) oo += P.out_coef[v] * var[v];
+        const int ostep = P.out_coef[lane_var] * (int)es, oadv = row_var < 0 ? 0 : P.out_coef[row_var];
+        for (int r = 0; r < n_rows; ++r) {
+            float p[4] = {Q.c, Q.c, Q.c, Q.c};
+#pragma unroll
+            for (int l = 0; l < 4; ++l) {
+                if (l >= Q.n_loads) continue;
+                const int kind = Q.ld[l].kind, e = Q.ld[l].exp;
+                if (kind == PK_HOIST) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) p[j] *= held[l][j];
+                    continue;
+                }
+                const float *__restrict__ src = ptrs.in[P.loads[Q.ld[l].load].ptr];
+                float v4[4];
+                if (kind == PK_BCAST) {
+                    const float s = __ldg(src + (unsigned)off[l]);
+                    v4[0] = v4[1] = v4[2] = v4[3] = s;
+                } else if (VEC && kind == PK_FWD && live == 4) {
+                    const float4 q = __ldg(reinterpret_cast<const float4 *>(src + (unsigned)off[l]));
+                    v4[0] = q.x; v4[1] = q.y; v4[2] = q.z; v4[3] = q.w;
+                } else if (VEC && kind == PK_REV && live == 4) {
+                    const float4 q = __ldg(reinterpret_cast<const float4 *>(src + (unsigned)(off[l] - 3)));
+                    v4[0] = q.w; v4[1] = q.z; v4[2] = q.y; v4[3] = q.x;
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) v4[j] = j < live ? __ldg(src + (unsigned)(off[l] + j * step[l])) : 0.f;
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) p[j] *= powe(v4[j], e);
+                off[l] += adv[l];
+            }
+            if (VEC && live == 4) {
+                float4 *dst = reinterpret_cast<float4 *>(out + (unsigned)oo);
+                float4 q = make_float4(p[0], p[1], p[2], p[3]);
+                if (P.accumulate) { const float4 o = *dst; q.x += o.x; q.y += o.y; q.z += o.z; q.w += o.w; }
+                *dst = q;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (j < live) { const unsigned o = (unsigned)(oo + j * ostep); out[o] = P.accumulate ? out[o] + p[j] : p[j]; }
+            }
+            oo += oadv;
+        }
+    }
+}
+
+// c * product of powers of loads, read off the accumulator program; false when the program is anything else
+bool product_form(const TadeProgram &P, ProdPlan &Q)
+{
+    struct Group { float c; int exp[TADE_MAX_LOADS]; bool any; };
+    Group x{}, y{};
+    bool have_x = false, have_y = false;
+    auto raise = [](Group &g, int k) {
+        for (int l = 0; l < TADE_MAX_LOADS; ++l) { g.exp[l] *= k; if (g.exp[l] > 3) return false; }
+        g.c = k == 2 ? g.c * g.c : g.c * g.c * g.c;
+        return true;
+    };
+    for (int s = 0; s < P.n_steps; ++s) {
+        const TadeStep &st = P.steps[s];
+        switch (st.op) {
+        case E_LD:
+            if (st.a < 0 || st.a >= TADE_MAX_LOADS) return false;
+            if (st.b == 0) { x = Group{}; x.c = 1.f; x.exp[st.a] = 1; have_x = true; }
+            else if (st.b == 2 && have_x) { if (++x.exp[st.a] > 3) return false; }
+            else return false;
+            break;
+        case E_PUSH: if (!have_x || have_y) return false; y = x; have_y = true; have_x = false; break;
+        case E_NEG: if (!have_x) return false; x.c = -x.c; break;
+        case E_MULC: if (!have_x) return false; x.c *= st.imm; break;
+        case E_SQR: if (!have_x || !raise(x, 2)) return false; break;
+        case E_CUBE: if (!have_x || !raise(x, 3)) return false; break;
+        case E_MULY:
+            if (!have_x || !have_y) return false;
+            x.c *= y.c;
+            for (int l = 0; l < TADE_MAX_LOADS; ++l) { x.exp[l] += y.exp[l]; if (x.exp[l] > 3) return false; }
+            have_y = false;
+            break;
+        default: return false;
+        }
+    }
+    if (!have_x || have_y) return false;
+    Q = ProdPlan{};
+    Q.c = x.c;
+    for (int l = 0; l < TADE_MAX_LOADS; ++l)
+        if (x.exp[l] > 0) {
+            if (Q.n_loads == 4 || l >= P.n_loads) return false;
+            Q.ld[Q.n_loads].load = l; Q.ld[Q.n_loads].exp = x.exp[l]; ++Q.n_loads;
+        }
+    return Q.n_loads > 0;
+}
+
+// layout and load kinds of a product program; the row variable is the innermost outer variable besides the lane variable
+void plan_product(const TadeProgram &P, const TadpPointers &ptrs, unsigned sms, ProdPlan &Q)
+{
+    const int lane = P.lane_var;
+    Q.row_var = -1;
+    for (int v = P.n_outer - 1; v >= 0; --v) if (v != lane && P.outer_ext[v] > 1) { Q.row_var = v; break; }
+    double elems = 1;
+    for (int v = 0; v < P.n_outer; ++v) elems *= (double)P.outer_ext[v];
+    // rows per thread: as many as leave every SM a few thousand threads
+    int run = 1;
+    while (run < 16 && elems / (4.0 * run * 2) >= (double)sms * 2048.0 * 2.0) run *= 2;
+    Q.run = Q.row_var < 0 ? 1 : std::min(run, P.outer_ext[Q.row_var]);
+    // offset of the first element, and whether it stays a multiple of four in every row
+    auto aligned = [&](const int32_t *coef, int64_t base, int shift) {
+        int64_t o = base - shift;
+        for (int v = 0; v < P.n_outer; ++v) { o += (int64_t)coef[v] * P.outer_lo[v]; if (v != lane && coef[v] % 4 != 0) return false; }
+        return o % 4 == 0;
+    };
+    bool vec = P.out_coef[lane] == 1 && aligned(P.out_coef, P.out_base, 0) && (reinterpret_cast<uintptr_t>(ptrs.out) & 15u) == 0;
+    for (int i = 0; i < Q.n_loads; ++i) {
+        const TadpLoad &L = P.loads[Q.ld[i].load];
+        const int step = L.coef[lane], adv = Q.row_var < 0 ? 0 : L.coef[Q.row_var];
+        const bool base16 = (reinterpret_cast<uintptr_t>(ptrs.in[L.ptr]) & 15u) == 0;
+        int kind = PK_GEN;
+        if (adv == 0 || Q.run == 1) kind = PK_HOIST;
+        else if (step == 0) kind = PK_BCAST;
+        else if (step == 1 && base16 && aligned(L.coef, L.base, 0)) kind = PK_FWD;
+        else if (step == -1 && base16 && aligned(L.coef, L.base, 3)) kind = PK_REV;
+        if (kind == PK_GEN) vec = false;
+        Q.ld[i].kind = kind;
+    }
+    Q.vec = vec ? 1 : 0;
+}
+
 }  // namespace
 
 cudaError_t tad_launch_ew(const TadeProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream)
@@ -162,6 +372,24 @@ cudaError_t tad_launch_ew(const TadeProgram &P, const TadpPointers &ptrs, unsign
     unsigned long long rows = 1;
     for (int v = 0; v < P.n_outer; ++v) if (v != P.lane_var) rows *= (unsigned long long)P.outer_ext[v];
     if (lane_ext == 0 || rows == 0) return cudaSuccess;
+    ProdPlan Q;
+    if (product_form(P, Q)) {
+        plan_product(P, ptrs, sms, Q);
+        unsigned pc = 1;
+        while (pc < 256u && pc * 4u < lane_ext) pc *= 2u;
+        if (!Q.vec && pc < 32u) pc = 32u;                      // interleaved outputs: a warp covers a run of 32 columns
+        const unsigned per_block = 256u / pc;
+        const unsigned lblocks = (lane_ext + pc * 4u - 1u) / (pc * 4u);
+        const unsigned long long row_ext = Q.row_var < 0 ? 1ull : (unsigned long long)P.outer_ext[Q.row_var];
+        const unsigned long long per_line = (row_ext + Q.run - 1) / Q.run;
+        const unsigned long long runs = rows / row_ext * per_line;
+        const unsigned long long its = ((runs + per_block - 1) / per_block) * lblocks;
+        if (its >= (1ull << 32) || runs >= (1ull << 31)) return cudaErrorInvalidValue;
+        const unsigned g = (unsigned)std::min<unsigned long long>(its, (unsigned long long)sms * 32ull);
+        if (Q.vec) tad_prod_kernel<true><<<g, 256, 0, stream>>>(P, Q, ptrs, (unsigned)its, pc, lblocks, (unsigned)runs, (unsigned)per_line);
+        else tad_prod_kernel<false><<<g, 256, 0, stream>>>(P, Q, ptrs, (unsigned)its, pc, lblocks, (unsigned)runs, (unsigned)per_line);
+        return cudaGetLastError();
+    }
     unsigned cols = 1;
     while (cols < 256u && cols * 4u * EG < lane_ext) cols *= 2u;
     const unsigned rows_per_block = 256u / cols;

@@ -32,9 +32,52 @@ __device__ __forceinline__ void range(const TadlProgram &P, int l, const int (&v
 
 constexpr int V = 4;     // outer variables a line-sum program may have
 
+// One run of the innermost loop: sum over z = z0, z0 + step, ... <= hi of the product of NL loads, every offset advancing
+// by its own constant.  U terms are in flight at once (their loads are issued before the first multiplication), each
+// with its own accumulator; the accumulators are added in a fixed order at the end.  Where load 0 (the largest
+// operand) is consecutive along the lanes every line of it is used once: it then streams through the cache (evict-first)
+// and leaves the lines of the smaller operands alone.
+template <int NL, int U, bool STREAM>
+__device__ __forceinline__ float walk(const float *const (&src)[4], const int (&sq)[4], int (&o)[4], const int (&d)[4], int z, const int hi, const int step)
+{
+    float s[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) s[u] = 0.f;
+    for (; z + (U - 1) * step <= hi; z += U * step) {
+        float v[U][NL];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int l = 0; l < NL; ++l) v[u][l] = (l == 0 && STREAM) ? __ldcs(src[l] + (unsigned)(o[l] + u * d[l])) : __ldg(src[l] + (unsigned)(o[l] + u * d[l]));
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            float p = sq[0] ? v[u][0] * v[u][0] : v[u][0];
+#pragma unroll
+            for (int l = 1; l < NL; ++l) p *= sq[l] ? v[u][l] * v[u][l] : v[u][l];
+            s[u] += p;
+        }
+#pragma unroll
+        for (int l = 0; l < NL; ++l) o[l] += U * d[l];
+    }
+    for (; z <= hi; z += step) {
+        float p = STREAM ? __ldcs(src[0] + (unsigned)o[0]) : __ldg(src[0] + (unsigned)o[0]);
+        if (sq[0]) p *= p;
+#pragma unroll
+        for (int l = 1; l < NL; ++l) { const float x = __ldg(src[l] + (unsigned)o[l]); p *= sq[l] ? x * x : x; }
+        s[0] += p;
+#pragma unroll
+        for (int l = 0; l < NL; ++l) o[l] += d[l];
+    }
+    float total = 0.f;
+#pragma unroll
+    for (int u = 0; u < U; ++u) total += s[u];
+    return total;
+}
+
+template <bool STREAM>
 __global__ void __launch_bounds__(256)
 tad_line_kernel(const __grid_constant__ TadlProgram P, const __grid_constant__ TadpPointers ptrs, const unsigned n_items,
-                const unsigned cols, const unsigned lane_blocks, const unsigned n_rows)
+                const unsigned cols, const unsigned lane_blocks, const unsigned n_rows, const int unroll)
 {
     const unsigned tid = threadIdx.x, lane = tid & 31u;
     const bool by_warp = P.mode == 1;
@@ -45,6 +88,8 @@ tad_line_kernel(const __grid_constant__ TadlProgram P, const __grid_constant__ T
     const float *__restrict__ src2 = P.n_loads > 2 ? ptrs.in[P.loads[2].ptr] : src0;
     const float *__restrict__ src3 = P.n_loads > 3 ? ptrs.in[P.loads[3].ptr] : src0;
     const int n_loads = P.n_loads;
+    const float *const srcs[4] = {src0, src1, src2, src3};
+    const int sq[4] = {P.loads[0].sq, P.loads[1].sq, P.loads[2].sq, P.loads[3].sq};
     for (unsigned item = blockIdx.x; item < n_items; item += gridDim.x) {
         // the output of this thread (mode 0) or warp (mode 1)
         unsigned row, lane0;
@@ -87,11 +132,11 @@ tad_line_kernel(const __grid_constant__ TadlProgram P, const __grid_constant__ T
             }
             int lo0, hi0;
             range(P, 0, var, 0, lo0, hi0);
-            if (P.zsplit > 1 && hi0 >= lo0) {
-                // share s of the range: [lo + len * s / S, lo + len * (s + 1) / S)
-                const long long len = (long long)hi0 - lo0 + 1;
-                const int a = lo0 + (int)(len * share / P.zsplit), b = lo0 + (int)(len * (share + 1) / P.zsplit) - 1;
-                lo0 = a; hi0 = b;
+            if (P.n_share[0] > 1) {
+                // pieces of the loop's box, counted from the one this output's range starts in: every share is short
+                const int s0 = P.n_share[1] == 1 ? share : share / P.n_share[1];
+                const int a = P.zbox_lo[0] + ((((lo0 - P.zbox_lo[0]) >> P.chunk_shift[0]) + s0) << P.chunk_shift[0]);
+                lo0 = max(lo0, a); hi0 = min(hi0, a + (1 << P.chunk_shift[0]) - 1);
             }
             const bool two = P.n_loops == 2;
             const int step_in = by_warp ? 32 : 1, first_in = by_warp ? (int)lane : 0;
@@ -104,38 +149,24 @@ tad_line_kernel(const __grid_constant__ TadlProgram P, const __grid_constant__ T
                 int o0 = b0, o1 = b1, o2 = b2, o3 = b3;
                 if (two) {
                     range(P, 1, var, z0, lo, hi);
+                    if (P.n_share[1] > 1) {
+                        const int a = P.zbox_lo[1] + ((((lo - P.zbox_lo[1]) >> P.chunk_shift[1]) + share % P.n_share[1]) << P.chunk_shift[1]);
+                        lo = max(lo, a); hi = min(hi, a + (1 << P.chunk_shift[1]) - 1);
+                    }
                     o0 += P.loads[0].cz[0] * z0; o1 += P.loads[1].cz[0] * z0; o2 += P.loads[2].cz[0] * z0; o3 += P.loads[3].cz[0] * z0;
                 }
                 const int zs = lo + first_in;
                 o0 += P.loads[0].cz[l_in] * zs; o1 += P.loads[1].cz[l_in] * zs; o2 += P.loads[2].cz[l_in] * zs; o3 += P.loads[3].cz[l_in] * zs;
-                float s0 = 0.f, s1 = 0.f;
-                int z = zs;
-                if (n_loads == 1) {
-                    for (; z + step_in <= hi; z += 2 * step_in) { s0 += __ldg(src0 + (unsigned)o0); s1 += __ldg(src0 + (unsigned)(o0 + d0)); o0 += 2 * d0; }
-                    if (z <= hi) s0 += __ldg(src0 + (unsigned)o0);
-                } else if (n_loads == 2) {
-                    for (; z + step_in <= hi; z += 2 * step_in) {
-                        const float x0 = __ldg(src0 + (unsigned)o0), y0 = __ldg(src1 + (unsigned)o1);
-                        const float x1 = __ldg(src0 + (unsigned)(o0 + d0)), y1 = __ldg(src1 + (unsigned)(o1 + d1));
-                        s0 = fmaf(x0, y0, s0); s1 = fmaf(x1, y1, s1);
-                        o0 += 2 * d0; o1 += 2 * d1;
-                    }
-                    if (z <= hi) s0 = fmaf(__ldg(src0 + (unsigned)o0), __ldg(src1 + (unsigned)o1), s0);
-                } else if (n_loads == 3) {
-                    for (; z + step_in <= hi; z += 2 * step_in) {
-                        const float x0 = __ldg(src0 + (unsigned)o0), y0 = __ldg(src1 + (unsigned)o1), w0 = __ldg(src2 + (unsigned)o2);
-                        const float x1 = __ldg(src0 + (unsigned)(o0 + d0)), y1 = __ldg(src1 + (unsigned)(o1 + d1)), w1 = __ldg(src2 + (unsigned)(o2 + d2));
-                        s0 = fmaf(x0 * y0, w0, s0); s1 = fmaf(x1 * y1, w1, s1);
-                        o0 += 2 * d0; o1 += 2 * d1; o2 += 2 * d2;
-                    }
-                    if (z <= hi) s0 = fmaf(__ldg(src0 + (unsigned)o0) * __ldg(src1 + (unsigned)o1), __ldg(src2 + (unsigned)o2), s0);
-                } else {
-                    for (; z <= hi; z += step_in) {
-                        s0 = fmaf(__ldg(src0 + (unsigned)o0) * __ldg(src1 + (unsigned)o1), __ldg(src2 + (unsigned)o2) * __ldg(src3 + (unsigned)o3), s0);
-                        o0 += d0; o1 += d1; o2 += d2; o3 += d3;
-                    }
-                }
-                acc += s0 + s1;
+                int o[4] = {o0, o1, o2, o3};
+                const int d[4] = {d0, d1, d2, d3};
+                float part;
+#define TAD_WALK(NL) (unroll == 2 ? walk<NL, 2, STREAM>(srcs, sq, o, d, zs, hi, step_in) : unroll == 4 ? walk<NL, 4, STREAM>(srcs, sq, o, d, zs, hi, step_in) : walk<NL, 8, STREAM>(srcs, sq, o, d, zs, hi, step_in))
+                if (n_loads == 1) part = TAD_WALK(1);
+                else if (n_loads == 2) part = TAD_WALK(2);
+                else if (n_loads == 3) part = TAD_WALK(3);
+                else part = TAD_WALK(4);
+#undef TAD_WALK
+                acc += part;
             }
         }
         if (by_warp) {
@@ -187,6 +218,7 @@ cudaError_t tad_launch_line(const TadlProgram &P, const TadpPointers &ptrs, unsi
     if (items >= (1ull << 31) || rows >= (1ull << 31)) return cudaErrorInvalidValue;
     const unsigned gx = (unsigned)std::min<unsigned long long>(items, (unsigned long long)sms * 32ull);
     dim3 grid(gx, (unsigned)std::max(1, P.zsplit), 1u);
-    tad_line_kernel<<<grid, 256, 0, stream>>>(P, ptrs, (unsigned)items, cols, lane_blocks, (unsigned)rows);
+    if (P.stream) tad_line_kernel<true><<<grid, 256, 0, stream>>>(P, ptrs, (unsigned)items, cols, lane_blocks, (unsigned)rows, P.unroll);
+    else tad_line_kernel<false><<<grid, 256, 0, stream>>>(P, ptrs, (unsigned)items, cols, lane_blocks, (unsigned)rows, P.unroll);
     return cudaGetLastError();
 }

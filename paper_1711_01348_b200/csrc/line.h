@@ -11,7 +11,7 @@
 #define TADL_MAX_LOADS 4
 #define TADL_MAX_ROWS 6
 
-struct TadlLoad { int32_t ptr, base; int32_t coef[TADP_MAX_VARS]; int32_t cz[2]; };     // offset = base + coef . outer + cz . z
+struct TadlLoad { int32_t ptr, base; int32_t coef[TADP_MAX_VARS]; int32_t cz[2]; int32_t sq; };     // offset = base + coef . outer + cz . z; sq: the value enters squared
 struct TadlRow { int32_t den, c0; int32_t coef[TADP_MAX_VARS]; int32_t cz; };           // (c0 + coef . outer + cz * z0) / den
 
 struct alignas(16) TadlProgram {
@@ -27,7 +27,12 @@ struct alignas(16) TadlProgram {
     float cterm;
     int32_t n_scale; TadlLoad scale[2]; float cscale;                      // factor outside the sums: cscale * product
     int32_t out_base, out_coef[TADP_MAX_VARS], out_limit, accumulate;
-    int32_t zsplit;                        // > 1: the range of loop 0 is divided among grid.y shares, each writing a plane
+    int32_t zsplit;                        // > 1: grid.y shares, each writing a plane of partial sums; share = s0 * n_share[1] + s1
+    int32_t n_share[2], chunk_shift[2], zbox_lo[2];
+    // the box of loop l is cut into pieces of 2^chunk_shift values counted from zbox_lo; share s_l of an output walks the
+    // s_l-th piece counted from the one its range starts in (cut to the range), so that neighbouring outputs stay in step
     int32_t part_limit, part_coef[TADP_MAX_VARS];
+    int32_t stream;                        // load 0 is consecutive along the lanes: read with evict-first loads
+    int32_t unroll;                        // terms a thread keeps in flight: 2, 4 or 8
     int32_t live_plane;                    // share 0 also writes plane zsplit: 1 where the guards hold (outputs of masked gradients that exist)
 };

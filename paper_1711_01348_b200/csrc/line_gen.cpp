@@ -3,6 +3,9 @@
 // is again such a product.  After the function tables of the optimisation pass most derivative terms have this
 // form (df times pre-evaluated functions of the arguments), and the kernel runs them without interpretation.
 #include <algorithm>
+#include <climits>
+#include <cmath>
+#include <cstdint>
 #include <cstring>
 #include <functional>
 
@@ -68,13 +71,28 @@ bool try_line(Gen &g, Kernel &k, int root, int scale, bool allow_split, const st
     if (guards.size() > TADL_MAX_ROWS) LFAIL;
     P.n_guards = (int32_t)guards.size();
     for (size_t r = 0; r < guards.size(); ++r) if (!conv_row(guards[r], 0, P.guards[r]) || guards[r].den != 1) LFAIL;
-    P.n_loads = (int32_t)loads.size();
-    int big = 0;
-    for (size_t i = 0; i < loads.size(); ++i) {
-        if (!conv_load(g.loads[loads[i]], P.loads[i])) LFAIL;
-        if (g.loads[loads[i]].limit > g.loads[loads[big]].limit) big = (int)i;
+    // (a load that occurs twice is read once and squared)
+    {
+        std::vector<int> uniq, twice;
+        for (int l : loads) {
+            size_t at = 0;
+            while (at < uniq.size() && uniq[at] != l) ++at;
+            if (at == uniq.size()) { uniq.push_back(l); twice.push_back(0); }
+            else if (!twice[at]) twice[at] = 1;
+            else { uniq.push_back(l); twice.push_back(0); }
+        }
+        int big = 0;
+        for (size_t i = 0; i < uniq.size(); ++i) {
+            if (!conv_load(g.loads[uniq[i]], P.loads[i])) LFAIL;
+            P.loads[i].sq = twice[i];
+            // load 0 is the operand the kernel streams: the largest, among equals the one more variables move
+            auto moving = [&](int l) { int n = 0; for (int v = 0; v < TADP_MAX_VARS; ++v) n += g.loads[l].coef[v] != 0; return n; };
+            const int64_t a = g.loads[uniq[i]].limit, b = g.loads[uniq[big]].limit;
+            if (a > b || (a == b && moving(uniq[i]) > moving(uniq[big]))) big = (int)i;
+        }
+        P.n_loads = (int32_t)uniq.size();
+        std::swap(P.loads[0], P.loads[big]);                 // (order is free in a product)
     }
-    std::swap(P.loads[0], P.loads[big]);                     // (order is free in a product)
     P.n_scale = (int32_t)sloads.size();
     for (size_t i = 0; i < sloads.size(); ++i) {
         if (!conv_load(g.loads[sloads[i]], P.scale[i]) || P.scale[i].cz[0] || P.scale[i].cz[1]) LFAIL;
@@ -110,18 +128,79 @@ bool try_line(Gen &g, Kernel &k, int root, int scale, bool allow_split, const st
     int64_t cells = 1;
     for (int v = g.n_outer - 1; v >= 0; --v) { P.part_coef[v] = to_i32(cells); cells = mul_ck(cells, prog.outer_ext[v]); }
     P.part_limit = to_i32(cells);
-    const double ext0 = (double)std::max<int64_t>(1, g.vars[z_id[0]].ext);
-    const double want = P.mode == 1 ? 148.0 * 64 : 148.0 * 2048;          // warps / threads that fill the GPU
-    if (allow_split && outputs < want / 2 && cells <= (1 << 22)) {
-        double s = std::ceil(want / outputs);
-        // every share keeps enough terms: eight of a single loop (128 when a warp walks it), a whole run of the inner loop
-        s = std::min(s, std::max(1.0, std::floor(ext0 / (g.kappa == 2 ? 1.0 : P.mode == 1 ? 128.0 : 8.0))));
-        s = std::min(s, 1024.0);
-        while (s > 1 && (s + 1) * (double)cells > (double)(1 << 25)) s -= 1;
-        P.zsplit = (int32_t)std::max(1.0, s);
+    // the box of every loop variable: a row bounds the range of every output, so its extreme over the outer box
+    // (and over the box of loop 0 for the rows of loop 1) bounds them all
+    int64_t zlo[2] = {0, 0}, zhi[2] = {0, 0};
+    for (int l = 0; l < g.kappa; ++l) {
+        auto extreme = [&](const TadlRow &R, bool want_max) {
+            int64_t v = R.c0;
+            for (int o = 0; o < g.n_outer; ++o) {
+                const int64_t a = (int64_t)R.coef[o] * P.outer_lo[o], b = (int64_t)R.coef[o] * (P.outer_lo[o] + std::max(1, P.outer_ext[o]) - 1);
+                v += want_max ? std::max(a, b) : std::min(a, b);
+            }
+            if (l == 1) { const int64_t a = (int64_t)R.cz * zlo[0], b = (int64_t)R.cz * zhi[0]; v += want_max ? std::max(a, b) : std::min(a, b); }
+            return v;
+        };
+        auto floor_div = [](int64_t a, int64_t b) { int64_t q = a / b; return (a % b != 0 && a < 0) ? q - 1 : q; };
+        int64_t lo = INT64_MIN, hi = INT64_MAX;
+        for (int r = 0; r < P.n_lower[l]; ++r) lo = std::max(lo, -floor_div(-extreme(P.lower[l][r], false), P.lower[l][r].den));
+        for (int r = 0; r < P.n_upper[l]; ++r) hi = std::min(hi, floor_div(extreme(P.upper[l][r], true), P.upper[l][r].den));
+        if (lo < INT32_MIN / 2 || hi > INT32_MAX / 2) LFAIL;
+        zlo[l] = lo; zhi[l] = std::max(lo, hi);
+    }
+    // the longest range of every loop: hi - lo <= (an upper row) - (a lower row) for every pair of rows, an affine
+    // form over the outer box (and the box of loop 0) whose maximum interval arithmetic gives
+    int64_t longest[2] = {1, 1};
+    for (int l = 0; l < g.kappa; ++l) {
+        int64_t best = zhi[l] - zlo[l] + 1;
+        for (int u = 0; u < P.n_upper[l]; ++u)
+            for (int r = 0; r < P.n_lower[l]; ++r) {
+                const TadlRow &U = P.upper[l][u], &L = P.lower[l][r];
+                // U / du - L / dl = (U * dl - L * du) / (du * dl)
+                const int64_t du = U.den, dl = L.den;
+                int64_t top = (int64_t)U.c0 * dl - (int64_t)L.c0 * du;
+                auto add = [&](int64_t c, int64_t lo, int64_t hi) { top += std::max(c * lo, c * hi); };
+                for (int o = 0; o < g.n_outer; ++o)
+                    add((int64_t)U.coef[o] * dl - (int64_t)L.coef[o] * du, P.outer_lo[o], P.outer_lo[o] + std::max(1, P.outer_ext[o]) - 1);
+                if (l == 1) add((int64_t)U.cz * dl - (int64_t)L.cz * du, zlo[0], zhi[0]);
+                const int64_t den = du * dl;
+                int64_t q = top / den; if (top % den != 0 && top < 0) --q;       // floor
+                best = std::min(best, std::max<int64_t>(1, q + 1));
+            }
+        longest[l] = best;
+    }
+    P.n_share[0] = P.n_share[1] = 1;
+    // ---- shares: pieces of every range, short enough that no thread walks a long chain of dependent batches and
+    //      numerous enough to fill the GPU several times over ----
+    const double slots = P.mode == 1 ? 148.0 * 48 : 148.0 * 1536;          // warps / threads resident at once
+    const double piece = P.mode == 1 ? 1024.0 : 64.0;                       // terms of one thread (warp) per share
+    const double ext_in = (double)longest[l_in], ext_out = g.kappa == 2 ? (double)longest[0] : 1.0;
+    if (allow_split && outputs < slots * 4 && cells <= (1 << 22)) {
+        double room = std::floor((double)(1 << 25) / (double)cells) - 1;    // planes the workspace may hold
+        room = std::min(room, std::max(1.0, std::floor(slots * 16 / outputs)));   // and no more threads than sixteen rounds
+        room = std::min(room, 4096.0);
+        // pieces of 2^k values; a range of length n that starts anywhere inside a piece touches up to ceil(n / 2^k) + 1
+        // pieces, never more than the box has
+        auto cut = [&](int l, double length, double box, double want_shares) {
+            int shift = 0;
+            while ((double)(1 << shift) * want_shares < length && shift < 30) ++shift;
+            const double pieces = std::ceil(length / (double)(1 << shift)) + (length < box ? 1 : 0);
+            P.chunk_shift[l] = shift;
+            P.n_share[l] = (int32_t)std::max(1.0, std::min(pieces, std::ceil(box / (double)(1 << shift)) + 1));
+            P.zbox_lo[l] = to_i32(zlo[l]);
+        };
+        const double s_in = std::min(std::ceil(ext_in / piece), std::max(1.0, room));
+        if (s_in > 1) cut(l_in, ext_in, (double)(zhi[l_in] - zlo[l_in] + 1), s_in);
+        if (g.kappa == 2) {
+            const double s_out = std::min(ext_out, std::max(1.0, std::floor(room / P.n_share[1])));
+            if (s_out > 1) cut(0, ext_out, (double)(zhi[0] - zlo[0] + 1), s_out);
+        }
+        P.zsplit = P.n_share[0] * P.n_share[1];
     }
     // a masked gradient's box also holds positions that are no elements (their offsets may fall on real ones): the
     // reduction writes only where the guards held
+    P.unroll = 4;
+    P.stream = (P.mode == 1 ? std::abs(P.loads[0].cz[l_in]) == 1 : std::abs(P.loads[0].coef[P.lane_var]) == 1) ? 1 : 0;
     P.live_plane = (P.zsplit > 1 && prog.write_only_live) ? 1 : 0;
     if (P.zsplit <= 1) prog.write_only_live = 0;
     k.line = {P};

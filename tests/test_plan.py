@@ -288,7 +288,7 @@ def test_contractions_run_on_the_tile_kernel():
 def test_gradients_of_cfg3_and_cfg4_are_line_sums():
     """With exp, tanh, sin and cos tabulated over the elements of x, every gradient term of the shifted and the
     non-unimodular workload is a product of index expressions under one or two summation loops: line-sum
-    programs.  Few outputs with long summations share their outermost range out."""
+    programs.  Few outputs with long summations are cut into shares of about 64 terms (pieces of the loops' boxes)."""
     from workloads import configs as W
     p3 = Plan(W.FULL["cfg3"]())
     for q in (0, 1):                                  # dx through x[i + j] and through x[2i + 3j]
@@ -300,7 +300,8 @@ def test_gradients_of_cfg3_and_cfg4_are_line_sums():
     p4 = Plan(W.FULL["cfg4"]())
     dx, dy = p4.disassemble(0), p4.disassemble(1)
     assert "; line sums" in dx and " 1 shares" in dx and " 3 guards" in dx
-    assert "; line sums: 2 loads x 2 loops" in dy and " 512 shares" in dy               # 512 live outputs x 262 144 terms
+    assert "; line sums: 2 loads x 2 loops" in dy and " 4096 shares" in dy              # 512 live outputs x 262 144 terms: 512 x 8 pieces
+    assert " 64 shares" in p3.disassemble(0)                                             # ranges of up to 4 096 terms
 
 
 def test_split_summations_fill_whole_waves():
