@@ -171,15 +171,15 @@ enum ProdKind : int { PK_HOIST = 0, PK_BCAST, PK_FWD, PK_REV, PK_GEN };
 
 struct ProdLoad { int32_t load, kind, exp; };
 struct ProdPlan {
-    int32_t n_loads, row_var, run, vec;      // run: rows per thread along row_var (row_var < 0: single rows)
+    int32_t n_loads, n_moving, row_var, run, vec;      // run: rows per thread along row_var (row_var < 0: single rows); moving loads first
     float c;
     ProdLoad ld[4];
 };
 
 __device__ __forceinline__ float powe(float v, int e) { return e == 1 ? v : e == 2 ? v * v : v * v * v; }
 
-template <bool VEC>
-__global__ void __launch_bounds__(256)
+template <bool VEC, int M>
+__global__ void __launch_bounds__(256, 3)
 tad_prod_kernel(const __grid_constant__ TadeProgram P, const __grid_constant__ ProdPlan Q, const __grid_constant__ TadpPointers ptrs,
                 const unsigned n_items, const unsigned cols, const unsigned lane_blocks, const unsigned n_runs, const unsigned runs_per_line)
 {
@@ -216,23 +216,31 @@ tad_prod_kernel(const __grid_constant__ TadeProgram P, const __grid_constant__ P
             }
         }
         const int n_rows = row_var < 0 ? 1 : min(Q.run, P.outer_ext[row_var] - (int)(piece * (unsigned)Q.run));
-        int off[4], step[4], adv[4];
-        float held[4][4];
+        // loads that stay put from row to row are multiplied into one factor per output (with the constant); the
+        // others ("moving", Q.n_moving of them, first in Q.ld) keep an offset that advances by a constant per row
+        float held[4] = {Q.c, Q.c, Q.c, Q.c};
+        int off[3] = {0, 0, 0}, step[3] = {0, 0, 0}, adv[3] = {0, 0, 0}, kinds[3] = {0, 0, 0}, exps[3] = {1, 1, 1};
+        const float *__restrict__ srcs[3] = {nullptr, nullptr, nullptr};
+        constexpr int n_moving = M;
+        unsigned widths = 0x111u;                              // four bits per moving load: values per vector load in this run
 #pragma unroll
         for (int l = 0; l < 4; ++l) {
-            off[l] = 0; step[l] = 0; adv[l] = 0;
+            if (l >= Q.n_loads) continue;
+            const TadpLoad &L = P.loads[Q.ld[l].load];
+            int o = L.base;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) held[l][j] = 1.f;
-            if (l < Q.n_loads) {
-                const TadpLoad &L = P.loads[Q.ld[l].load];
-                int o = L.base;
+            for (int v = 0; v < TADP_MAX_VARS; ++v) o += L.coef[v] * var[v];
+            const int st = L.coef[lane_var] * (int)es;
+            if (l >= M) {
+                const float *__restrict__ src = ptrs.in[L.ptr];
 #pragma unroll
-                for (int v = 0; v < TADP_MAX_VARS; ++v) o += L.coef[v] * var[v];
-                off[l] = o; step[l] = L.coef[lane_var] * (int)es; adv[l] = row_var < 0 ? 0 : L.coef[row_var];
-                if (Q.ld[l].kind == PK_HOIST) {
-                    const float *__restrict__ src = ptrs.in[L.ptr];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) if (j < live) held[l][j] = powe(__ldg(src + (unsigned)(o + j * step[l])), Q.ld[l].exp);
+                for (int j = 0; j < 4; ++j) if (j < live) held[j] *= powe(__ldg(src + (unsigned)(o + j * st)), Q.ld[l].exp);
+            } else if (l < 3) {
+                off[l] = o; step[l] = st; adv[l] = L.coef[row_var];
+                kinds[l] = Q.ld[l].kind; exps[l] = Q.ld[l].exp; srcs[l] = ptrs.in[L.ptr];
+                if (VEC && live == 4 && (Q.ld[l].kind == PK_FWD || Q.ld[l].kind == PK_REV)) {
+                    const unsigned first = (unsigned)(Q.ld[l].kind == PK_FWD ? o : o - 3);
+                    widths += ((first & 3u) == 0 ? 3u : (first & 1u) == 0 ? 1u : 0u) << (4 * l);
                 }
             }
         }
@@ -240,36 +248,54 @@ tad_prod_kernel(const __grid_constant__ TadeProgram P, const __grid_constant__ P
 #pragma unroll
         for (int v = 0; v < TADP_MAX_VARS; ++v) oo += P.out_coef[v] * var[v];
         const int ostep = P.out_coef[lane_var] * (int)es, oadv = row_var < 0 ? 0 : P.out_coef[row_var];
-        for (int r = 0; r < n_rows; ++r) {
-            float p[4] = {Q.c, Q.c, Q.c, Q.c};
+        // the product of one row (offsets advance to the next row)
+        auto row = [&](float (&p)[4]) {
 #pragma unroll
-            for (int l = 0; l < 4; ++l) {
-                if (l >= Q.n_loads) continue;
-                const int kind = Q.ld[l].kind, e = Q.ld[l].exp;
-                if (kind == PK_HOIST) {
+            for (int j = 0; j < 4; ++j) p[j] = held[j];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) p[j] *= held[l][j];
-                    continue;
-                }
-                const float *__restrict__ src = ptrs.in[P.loads[Q.ld[l].load].ptr];
+            for (int l = 0; l < M; ++l) {
+                const int kind = kinds[l];
+                const unsigned w = (widths >> (4 * l)) & 15u;
+                const float *__restrict__ src = srcs[l];
                 float v4[4];
                 if (kind == PK_BCAST) {
                     const float s = __ldg(src + (unsigned)off[l]);
                     v4[0] = v4[1] = v4[2] = v4[3] = s;
-                } else if (VEC && kind == PK_FWD && live == 4) {
-                    const float4 q = __ldg(reinterpret_cast<const float4 *>(src + (unsigned)off[l]));
-                    v4[0] = q.x; v4[1] = q.y; v4[2] = q.z; v4[3] = q.w;
-                } else if (VEC && kind == PK_REV && live == 4) {
-                    const float4 q = __ldg(reinterpret_cast<const float4 *>(src + (unsigned)(off[l] - 3)));
-                    v4[0] = q.w; v4[1] = q.z; v4[2] = q.y; v4[3] = q.x;
+                } else if (VEC && w == 4u) {
+                    if (kind == PK_FWD) {
+                        const float4 q = __ldg(reinterpret_cast<const float4 *>(src + (unsigned)off[l]));
+                        v4[0] = q.x; v4[1] = q.y; v4[2] = q.z; v4[3] = q.w;
+                    } else {
+                        const float4 q = __ldg(reinterpret_cast<const float4 *>(src + (unsigned)(off[l] - 3)));
+                        v4[0] = q.w; v4[1] = q.z; v4[2] = q.y; v4[3] = q.x;
+                    }
+                } else if (VEC && w == 2u) {
+                    if (kind == PK_FWD) {
+                        const float2 q0 = __ldg(reinterpret_cast<const float2 *>(src + (unsigned)off[l]));
+                        const float2 q1 = __ldg(reinterpret_cast<const float2 *>(src + (unsigned)(off[l] + 2)));
+                        v4[0] = q0.x; v4[1] = q0.y; v4[2] = q1.x; v4[3] = q1.y;
+                    } else {
+                        const float2 q0 = __ldg(reinterpret_cast<const float2 *>(src + (unsigned)(off[l] - 1)));
+                        const float2 q1 = __ldg(reinterpret_cast<const float2 *>(src + (unsigned)(off[l] - 3)));
+                        v4[0] = q0.y; v4[1] = q0.x; v4[2] = q1.y; v4[3] = q1.x;
+                    }
+                } else if (live == 4) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) v4[j] = __ldg(src + (unsigned)(off[l] + j * step[l]));
                 } else {
 #pragma unroll
                     for (int j = 0; j < 4; ++j) v4[j] = j < live ? __ldg(src + (unsigned)(off[l] + j * step[l])) : 0.f;
                 }
+                if (exps[l] != 1) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) p[j] *= powe(v4[j], e);
+                    for (int j = 0; j < 4; ++j) v4[j] = powe(v4[j], exps[l]);
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) p[j] *= v4[j];
                 off[l] += adv[l];
             }
+        };
+        auto store = [&](const float (&p)[4]) {
             if (VEC && live == 4) {
                 float4 *dst = reinterpret_cast<float4 *>(out + (unsigned)oo);
                 float4 q = make_float4(p[0], p[1], p[2], p[3]);
@@ -281,7 +307,15 @@ tad_prod_kernel(const __grid_constant__ TadeProgram P, const __grid_constant__ P
                     if (j < live) { const unsigned o = (unsigned)(oo + j * ostep); out[o] = P.accumulate ? out[o] + p[j] : p[j]; }
             }
             oo += oadv;
+        };
+        // two rows in flight: the loads of the second are issued before the first is multiplied and stored
+        int r = 0;
+        for (; r + 2 <= n_rows; r += 2) {
+            float p0[4], p1[4];
+            row(p0); row(p1);
+            store(p0); store(p1);
         }
+        if (r < n_rows) { float p0[4]; row(p0); store(p0); }
     }
 }
 
@@ -331,7 +365,7 @@ bool product_form(const TadeProgram &P, ProdPlan &Q)
 }
 
 // layout and load kinds of a product program; the row variable is the innermost outer variable besides the lane variable
-void plan_product(const TadeProgram &P, const TadpPointers &ptrs, unsigned sms, ProdPlan &Q)
+bool plan_product(const TadeProgram &P, const TadpPointers &ptrs, unsigned sms, ProdPlan &Q)
 {
     const int lane = P.lane_var;
     Q.row_var = -1;
@@ -340,15 +374,16 @@ void plan_product(const TadeProgram &P, const TadpPointers &ptrs, unsigned sms, 
     for (int v = 0; v < P.n_outer; ++v) elems *= (double)P.outer_ext[v];
     // rows per thread: as many as leave every SM a few thousand threads
     int run = 1;
-    while (run < 16 && elems / (4.0 * run * 2) >= (double)sms * 2048.0 * 2.0) run *= 2;
+    while (run < 32 && elems / (4.0 * run * 2) >= (double)sms * 2048.0) run *= 2;
     Q.run = Q.row_var < 0 ? 1 : std::min(run, P.outer_ext[Q.row_var]);
-    // offset of the first element, and whether it stays a multiple of four in every row
-    auto aligned = [&](const int32_t *coef, int64_t base, int shift) {
-        int64_t o = base - shift;
+    // the output is stored in 128-bit pieces when its first element of every row is a multiple of four; a load needs
+    // only a row step that is one (the width of its vector loads is settled per run)
+    auto aligned = [&](const int32_t *coef, int64_t base) {
+        int64_t o = base;
         for (int v = 0; v < P.n_outer; ++v) { o += (int64_t)coef[v] * P.outer_lo[v]; if (v != lane && coef[v] % 4 != 0) return false; }
         return o % 4 == 0;
     };
-    bool vec = P.out_coef[lane] == 1 && aligned(P.out_coef, P.out_base, 0) && (reinterpret_cast<uintptr_t>(ptrs.out) & 15u) == 0;
+    bool vec = P.out_coef[lane] == 1 && aligned(P.out_coef, P.out_base) && (reinterpret_cast<uintptr_t>(ptrs.out) & 15u) == 0;
     for (int i = 0; i < Q.n_loads; ++i) {
         const TadpLoad &L = P.loads[Q.ld[i].load];
         const int step = L.coef[lane], adv = Q.row_var < 0 ? 0 : L.coef[Q.row_var];
@@ -356,12 +391,17 @@ void plan_product(const TadeProgram &P, const TadpPointers &ptrs, unsigned sms, 
         int kind = PK_GEN;
         if (adv == 0 || Q.run == 1) kind = PK_HOIST;
         else if (step == 0) kind = PK_BCAST;
-        else if (step == 1 && base16 && aligned(L.coef, L.base, 0)) kind = PK_FWD;
-        else if (step == -1 && base16 && aligned(L.coef, L.base, 3)) kind = PK_REV;
+        else if (step == 1 && base16 && adv % 4 == 0) kind = PK_FWD;
+        else if (step == -1 && base16 && adv % 4 == 0) kind = PK_REV;
         if (kind == PK_GEN) vec = false;
         Q.ld[i].kind = kind;
     }
+    // moving loads first
+    std::stable_sort(Q.ld, Q.ld + Q.n_loads, [](const ProdLoad &a, const ProdLoad &b) { return (a.kind != PK_HOIST) > (b.kind != PK_HOIST); });
+    Q.n_moving = 0;
+    for (int i = 0; i < Q.n_loads; ++i) Q.n_moving += Q.ld[i].kind != PK_HOIST;
     Q.vec = vec ? 1 : 0;
+    return Q.n_moving <= 3;
 }
 
 }  // namespace
@@ -373,8 +413,7 @@ cudaError_t tad_launch_ew(const TadeProgram &P, const TadpPointers &ptrs, unsign
     for (int v = 0; v < P.n_outer; ++v) if (v != P.lane_var) rows *= (unsigned long long)P.outer_ext[v];
     if (lane_ext == 0 || rows == 0) return cudaSuccess;
     ProdPlan Q;
-    if (product_form(P, Q)) {
-        plan_product(P, ptrs, sms, Q);
+    if (product_form(P, Q) && plan_product(P, ptrs, sms, Q)) {
         unsigned pc = 1;
         while (pc < 256u && pc * 4u < lane_ext) pc *= 2u;
         if (!Q.vec && pc < 32u) pc = 32u;                      // interleaved outputs: a warp covers a run of 32 columns
@@ -386,8 +425,18 @@ cudaError_t tad_launch_ew(const TadeProgram &P, const TadpPointers &ptrs, unsign
         const unsigned long long its = ((runs + per_block - 1) / per_block) * lblocks;
         if (its >= (1ull << 32) || runs >= (1ull << 31)) return cudaErrorInvalidValue;
         const unsigned g = (unsigned)std::min<unsigned long long>(its, (unsigned long long)sms * 32ull);
-        if (Q.vec) tad_prod_kernel<true><<<g, 256, 0, stream>>>(P, Q, ptrs, (unsigned)its, pc, lblocks, (unsigned)runs, (unsigned)per_line);
-        else tad_prod_kernel<false><<<g, 256, 0, stream>>>(P, Q, ptrs, (unsigned)its, pc, lblocks, (unsigned)runs, (unsigned)per_line);
+#define TAD_PROD_LAUNCH(V, MM) tad_prod_kernel<V, MM><<<g, 256, 0, stream>>>(P, Q, ptrs, (unsigned)its, pc, lblocks, (unsigned)runs, (unsigned)per_line)
+        switch ((Q.vec ? 4 : 0) + Q.n_moving) {
+        case 0: TAD_PROD_LAUNCH(false, 0); break;
+        case 1: TAD_PROD_LAUNCH(false, 1); break;
+        case 2: TAD_PROD_LAUNCH(false, 2); break;
+        case 3: TAD_PROD_LAUNCH(false, 3); break;
+        case 4: TAD_PROD_LAUNCH(true, 0); break;
+        case 5: TAD_PROD_LAUNCH(true, 1); break;
+        case 6: TAD_PROD_LAUNCH(true, 2); break;
+        default: TAD_PROD_LAUNCH(true, 3); break;
+        }
+#undef TAD_PROD_LAUNCH
         return cudaGetLastError();
     }
     unsigned cols = 1;
