@@ -560,11 +560,80 @@ int body_fetch_kind(const TadpLoad &L, int ta, int ub)
 
 // A program without loops and temporaries whose pending values never exceed two becomes an element-wise program
 // (ew.h); a thread owns four consecutive values of the lane variable.
-bool try_elementwise(Gen &g, Kernel &k, const Emitter &em, const std::vector<TadpRow> &guards)
+// Steps of an element-wise program read off the expression itself, the operand that needs the second value register
+// evaluated first (so that a * (b * c + d) needs no more than X and Y whatever the order it was written in).
+// need(i): value registers the evaluation of i occupies; a binary operation whose operands are both compound puts the
+// first into Y, which the second must then leave alone (need 1).
+bool elementwise_steps_of(const Gen &g, int root, std::vector<TadeStep> &steps)
+{
+    auto push_step = [&](int op, int a = 0, int b = 0, float imm = 0.f) { TadeStep s{}; s.op = (uint8_t)op; s.a = (int16_t)a; s.b = (uint8_t)b; s.imm = imm; steps.push_back(s); };
+    auto is_load = [&](int i) { return g.inst[i].op == I_LOAD; };
+    std::function<int(int)> need = [&](int i) -> int {
+        const Inst &in = g.inst[i];
+        switch (in.op) {
+        case I_CONST: case I_LOAD: return 1;
+        case I_SUM: return 99;
+        case I_ADD: case I_MUL:
+            if (is_load(in.a)) return need(in.b);
+            if (is_load(in.b)) return need(in.a);
+            return std::max(std::max(need(in.a), need(in.b)), std::min(need(in.a), need(in.b)) + 1);
+        case I_SUB: case I_DIV: return std::max(need(in.a), need(in.b) + 1);
+        default: return need(in.a);
+        }
+    };
+    std::function<bool(int)> emit = [&](int i) -> bool {
+        const Inst &in = g.inst[i];
+        if (in.temp >= 0) return false;
+        auto fn = [&](int f, int e = 0) { if (!emit(in.a)) return false; push_step(E_FN, e, f); return true; };
+        switch (in.op) {
+        case I_CONST: push_step(E_CONST, 0, 0, in.imm); return true;
+        case I_LOAD: push_step(E_LD, in.load, 0); return true;
+        case I_NEG: if (!emit(in.a)) return false; push_step(E_NEG); return true;
+        case I_SQR: if (!emit(in.a)) return false; push_step(E_SQR); return true;
+        case I_MULC: if (!emit(in.a)) return false; push_step(E_MULC, 0, 0, in.imm); return true;
+        case I_ADDC: if (!emit(in.a)) return false; push_step(E_ADDC, 0, 0, in.imm); return true;
+        case I_POWI:
+            if (in.ipow == 3) { if (!emit(in.a)) return false; push_step(E_CUBE); return true; }
+            return fn(F_POWI, in.ipow);
+        case I_EXP: return fn(F_EXP);
+        case I_LOG: return fn(F_LOG);
+        case I_SIN: return fn(F_SIN);
+        case I_COS: return fn(F_COS);
+        case I_TANH: return fn(F_TANH);
+        case I_SINH: return fn(F_SINH);
+        case I_COSH: return fn(F_COSH);
+        case I_ADD: case I_MUL: {
+            const int mode = in.op == I_ADD ? 1 : 2;
+            if (is_load(in.b) && !(is_load(in.a) && need(in.b) < need(in.a))) { if (!emit(in.a)) return false; push_step(E_LD, g.inst[in.b].load, mode); return true; }
+            if (is_load(in.a)) { if (!emit(in.b)) return false; push_step(E_LD, g.inst[in.a].load, mode); return true; }
+            const int first = need(in.a) >= need(in.b) ? in.a : in.b, second = first == in.a ? in.b : in.a;
+            if (need(first) > 2 || need(second) != 1) return false;
+            if (!emit(first)) return false;
+            push_step(E_PUSH);
+            if (!emit(second)) return false;
+            push_step(in.op == I_ADD ? E_ADDY : E_MULY);
+            return true;
+        }
+        case I_SUB: case I_DIV:
+            if (need(in.a) > 2 || need(in.b) != 1) return false;
+            if (!emit(in.a)) return false;
+            push_step(E_PUSH);
+            if (!emit(in.b)) return false;
+            push_step(in.op == I_SUB ? E_SUBY : E_DIVY);
+            return true;
+        default: return false;
+        }
+    };
+    if (need(root) > 2) return false;
+    return emit(root) && (int)steps.size() <= TADE_MAX_STEPS;
+}
+
+bool try_elementwise(Gen &g, Kernel &k, const Emitter &em, const std::vector<TadpRow> &guards, int root)
 {
     const TadpProgram &prog = k.prog;
     // (elements that a guard or a mask excludes are not evaluated by the interpreter: such kernels stay there)
-    if (g.kappa != 0 || g.p.opt.debug_bounds || !guards.empty() || prog.write_only_live) return false;
+    // (without guards and kernel coordinates every position of a masked gradient's box is an element)
+    if (g.kappa != 0 || g.p.opt.debug_bounds || !guards.empty()) return false;
     if (g.lane_var < 0 || g.lane_var >= g.n_outer) return false;
     if ((int)g.loads.size() > TADE_MAX_LOADS) return false;
     const std::vector<TadpInsn> &code = em.code;
@@ -574,8 +643,10 @@ bool try_elementwise(Gen &g, Kernel &k, const Emitter &em, const std::vector<Tad
     if (term_op != P_ACC && term_op != P_MACC) return false;
     std::vector<TadeStep> steps;
     auto push_step = [&](int op, int a = 0, int b = 0, float imm = 0.f) { TadeStep s{}; s.op = (uint8_t)op; s.a = (int16_t)a; s.b = (uint8_t)b; s.imm = imm; steps.push_back(s); };
+    const bool from_expression = root >= 0 && elementwise_steps_of(g, root, steps);
+    if (!from_expression) steps.clear();
     int vd = 0;                                  // pending values: 0, 1 (X) or 2 (Y below X)
-    for (int w = 0; w < n - 2; ++w) {
+    for (int w = 0; !from_expression && w < n - 2; ++w) {
         const TadpInsn &in = code[w];
         const int op = in.handler >> 3;
         float imm; std::memcpy(&imm, &in.imm, 4);
@@ -603,7 +674,8 @@ bool try_elementwise(Gen &g, Kernel &k, const Emitter &em, const std::vector<Tad
         default: return false;
         }
     }
-    if (term_op == P_MACC) { if (vd != 2) return false; push_step(E_MULY); }
+    if (from_expression) {}
+    else if (term_op == P_MACC) { if (vd != 2) return false; push_step(E_MULY); }
     else if (vd != 1) return false;
     if ((int)steps.size() > TADE_MAX_STEPS) return false;
     // every offset the kernel can form must lie inside its tensor (interval check over the outer box)
@@ -765,7 +837,7 @@ void emit_kernel(Gen &g, Kernel &k, int root, const std::vector<std::vector<Tadp
     if (scale >= 0) { em.expr(scale); em.emit(P_SCALE, 0, 0, 0, -1); }
     em.emit(P_END);
     if (em.depth != 0) throw BadExpr("internal: unbalanced operand stack");
-    if (n_temps == 0 && try_elementwise(g, k, em, guards)) return;
+    if (n_temps == 0 && try_elementwise(g, k, em, guards, scale < 0 ? root : -1)) return;
     // rows
     std::vector<TadpRow> rows;
     for (TadpLoop &L : em.loops) {

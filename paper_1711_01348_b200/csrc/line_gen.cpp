@@ -14,11 +14,29 @@
 
 namespace tad {
 
-bool try_line(Gen &g, Kernel &k, int root, int scale, bool allow_split, const std::vector<std::vector<TadpRow>> &lower,
-              const std::vector<std::vector<TadpRow>> &upper, const std::vector<TadpRow> &guards)
+bool try_line(Gen &g, Kernel &k, int root, int scale, bool allow_split, const std::vector<std::vector<TadpRow>> &lower_in,
+              const std::vector<std::vector<TadpRow>> &upper_in, const std::vector<TadpRow> &guards)
 {
-    if (g.p.opt.debug_bounds || root < 0 || g.kappa < 1 || g.kappa > 2 || g.n_outer < 1 || g.n_outer > 4) return false;
+    if (g.p.opt.debug_bounds || root < 0 || g.kappa > 2 || g.n_outer < 1 || g.n_outer > 4) return false;
     TadpProgram &prog = k.prog;
+    // a kernel without kernel coordinates whose value is one sum with constant bounds (a short sum the optimisation
+    // pass evaluates ahead of its kernel) is a line sum over that sum's variable
+    int n_loops = g.kappa, sum_var = -1;
+    std::vector<std::vector<TadpRow>> own_lower, own_upper;
+    if (g.kappa == 0) {
+        const Inst top = g.inst[root];
+        if (top.op != I_SUM || top.temp >= 0 || scale >= 0 || !guards.empty() || prog.write_only_live) return false;
+        if (top.lo < INT32_MIN / 2 || top.hi > INT32_MAX / 2 || top.hi < top.lo) return false;
+        TadpRow lo{}, hi{};
+        lo.den = hi.den = 1; lo.c0 = (int32_t)top.lo; hi.c0 = (int32_t)top.hi;
+        own_lower = {{lo}}; own_upper = {{hi}};
+        sum_var = top.var; n_loops = 1; root = top.a;
+        // (the outer variables must be the first n_outer ones: kernels the optimisation pass builds may order them otherwise)
+        if (sum_var < g.n_outer || sum_var >= TADP_MAX_VARS) return false;
+        for (int v = 0; v < g.n_outer; ++v) if (g.vars[v].kind != 0) return false;
+    }
+    const std::vector<std::vector<TadpRow>> &lower = g.kappa == 0 ? own_lower : lower_in;
+    const std::vector<std::vector<TadpRow>> &upper = g.kappa == 0 ? own_upper : upper_in;
     // ---- the term and the outer factor: products of loads and constants ----
     float cterm = 1.f, cscale = 1.f;
     std::vector<int> loads, sloads;
@@ -36,7 +54,7 @@ bool try_line(Gen &g, Kernel &k, int root, int scale, bool allow_split, const st
     };
     if (!flat(root, cterm, loads, TADL_MAX_LOADS) || loads.empty()) LFAIL;
     if (scale >= 0 && !flat(scale, cscale, sloads, 2)) LFAIL;
-    const int z_id[2] = {g.n_outer + g.zorder[0], g.kappa == 2 ? g.n_outer + g.zorder[1] : -1};
+    const int z_id[2] = {g.kappa == 0 ? sum_var : g.n_outer + g.zorder[0], g.kappa == 2 ? g.n_outer + g.zorder[1] : -1};
     auto conv_load = [&](const TadpLoad &L, TadlLoad &out) {
         out = TadlLoad{};
         out.ptr = L.ptr; out.base = L.base;
@@ -61,8 +79,8 @@ bool try_line(Gen &g, Kernel &k, int root, int scale, bool allow_split, const st
         return true;
     };
     TadlProgram P{};
-    P.n_outer = g.n_outer; P.n_loops = g.kappa;
-    for (int l = 0; l < g.kappa; ++l) {
+    P.n_outer = g.n_outer; P.n_loops = n_loops;
+    for (int l = 0; l < n_loops; ++l) {
         if (lower[l].empty() || upper[l].empty() || lower[l].size() > TADL_MAX_ROWS || upper[l].size() > TADL_MAX_ROWS) LFAIL;
         P.n_lower[l] = (int32_t)lower[l].size(); P.n_upper[l] = (int32_t)upper[l].size();
         for (size_t r = 0; r < lower[l].size(); ++r) if (!conv_row(lower[l][r], l, P.lower[l][r])) LFAIL;
@@ -111,7 +129,7 @@ bool try_line(Gen &g, Kernel &k, int root, int scale, bool allow_split, const st
     // ---- which way the lanes run: along an outer variable that makes the largest operand consecutive, else along
     //      the inner loop if that does (a warp per output), else along the longest outer variable ----
     const TadlLoad &B = P.loads[0];
-    const int l_in = g.kappa - 1;
+    const int l_in = n_loops - 1;
     int lane = -1;
     for (int v = 0; v < g.n_outer; ++v)
         if (std::abs(B.coef[v]) == 1 && prog.outer_ext[v] >= 32 && (lane < 0 || prog.outer_ext[v] > prog.outer_ext[lane])) lane = v;
@@ -131,7 +149,7 @@ bool try_line(Gen &g, Kernel &k, int root, int scale, bool allow_split, const st
     // the box of every loop variable: a row bounds the range of every output, so its extreme over the outer box
     // (and over the box of loop 0 for the rows of loop 1) bounds them all
     int64_t zlo[2] = {0, 0}, zhi[2] = {0, 0};
-    for (int l = 0; l < g.kappa; ++l) {
+    for (int l = 0; l < n_loops; ++l) {
         auto extreme = [&](const TadlRow &R, bool want_max) {
             int64_t v = R.c0;
             for (int o = 0; o < g.n_outer; ++o) {
@@ -151,7 +169,7 @@ bool try_line(Gen &g, Kernel &k, int root, int scale, bool allow_split, const st
     // the longest range of every loop: hi - lo <= (an upper row) - (a lower row) for every pair of rows, an affine
     // form over the outer box (and the box of loop 0) whose maximum interval arithmetic gives
     int64_t longest[2] = {1, 1};
-    for (int l = 0; l < g.kappa; ++l) {
+    for (int l = 0; l < n_loops; ++l) {
         int64_t best = zhi[l] - zlo[l] + 1;
         for (int u = 0; u < P.n_upper[l]; ++u)
             for (int r = 0; r < P.n_lower[l]; ++r) {
@@ -174,7 +192,7 @@ bool try_line(Gen &g, Kernel &k, int root, int scale, bool allow_split, const st
     //      numerous enough to fill the GPU several times over ----
     const double slots = P.mode == 1 ? 148.0 * 48 : 148.0 * 1536;          // warps / threads resident at once
     const double piece = P.mode == 1 ? 1024.0 : 64.0;                       // terms of one thread (warp) per share
-    const double ext_in = (double)longest[l_in], ext_out = g.kappa == 2 ? (double)longest[0] : 1.0;
+    const double ext_in = (double)longest[l_in], ext_out = n_loops == 2 ? (double)longest[0] : 1.0;
     if (allow_split && outputs < slots * 4 && cells <= (1 << 22)) {
         double room = std::floor((double)(1 << 25) / (double)cells) - 1;    // planes the workspace may hold
         room = std::min(room, std::max(1.0, std::floor(slots * 16 / outputs)));   // and no more threads than sixteen rounds
@@ -191,7 +209,7 @@ bool try_line(Gen &g, Kernel &k, int root, int scale, bool allow_split, const st
         };
         const double s_in = std::min(std::ceil(ext_in / piece), std::max(1.0, room));
         if (s_in > 1) cut(l_in, ext_in, (double)(zhi[l_in] - zlo[l_in] + 1), s_in);
-        if (g.kappa == 2) {
+        if (n_loops == 2) {
             const double s_out = std::min(ext_out, std::max(1.0, std::floor(room / P.n_share[1])));
             if (s_out > 1) cut(0, ext_out, (double)(zhi[0] - zlo[0] + 1), s_out);
         }
@@ -211,6 +229,18 @@ bool try_line(Gen &g, Kernel &k, int root, int scale, bool allow_split, const st
     std::snprintf(line, sizeof line, "; line sums: %d loads x %d loops, outer factor of %d loads, %s, lanes along variable %d, %d shares, %d guards\n",
                   P.n_loads, P.n_loops, P.n_scale, P.mode == 1 ? "a warp per output" : "a thread per output", P.lane_var, P.zsplit, P.n_guards);
     k.listing = line;
+    for (int i = 0; i < P.n_loads; ++i) {
+        std::snprintf(line, sizeof line, ";   load %d ptr=%d base=%d coef=[%d %d %d %d] step=[%d %d]%s\n", i, P.loads[i].ptr, P.loads[i].base, P.loads[i].coef[0],
+                      P.loads[i].coef[1], P.loads[i].coef[2], P.loads[i].coef[3], P.loads[i].cz[0], P.loads[i].cz[1], P.loads[i].sq ? " squared" : "");
+        k.listing += line;
+    }
+    for (int l = 0; l < P.n_loops; ++l) {
+        std::snprintf(line, sizeof line, ";   loop %d: %d lower rows, %d upper rows, first lower c0=%d den=%d, first upper c0=%d den=%d, %d pieces of 2^%d\n", l, P.n_lower[l], P.n_upper[l],
+                      P.lower[l][0].c0, P.lower[l][0].den, P.upper[l][0].c0, P.upper[l][0].den, P.n_share[l], P.chunk_shift[l]);
+        k.listing += line;
+    }
+    std::snprintf(line, sizeof line, ";   out base=%d coef=[%d %d %d %d] constant %g x %g\n", P.out_base, P.out_coef[0], P.out_coef[1], P.out_coef[2], P.out_coef[3], P.cterm, P.cscale);
+    k.listing += line;
     return true;
 }
 
