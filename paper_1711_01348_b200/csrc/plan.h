@@ -111,6 +111,7 @@ struct tad_plan {
     std::vector<bool> arg_zero_fill;            // the gradient is cleared before its kernels add into it
     size_t partial_bytes = 0;                   // workspace for the partial sums of split summations (largest kernel)
     size_t aux_bytes = 0;                       // workspace for auxiliary tensors (largest kernel)
+    mutable void *side = nullptr;               // second stream and its events (independent memory-bound passes run beside a contraction)
     mutable void *host_step = nullptr;          // streams and events of tad_step_host, created by its first call
 };
 

@@ -17,9 +17,9 @@ void set_error(const std::string &m);
 }
 
 // One build of the interpreter per vector shape, each in an object file of its own (vm_inst.cu).
-#define TAD_DECLARE_VM(TA, UB) void tad_launch_vm_##TA##_##UB(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream);
+#define TAD_DECLARE_VM(TA, UB) bool tad_launch_vm_##TA##_##UB(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream);
 TAD_VM_SHAPES(TAD_DECLARE_VM)
-void tad_launch_vm_16_1_rich(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream);
+bool tad_launch_vm_16_1_rich(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream);
 cudaError_t tad_launch_contract(const TadcProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream);
 cudaError_t tad_launch_ew(const TadeProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream);
 cudaError_t tad_launch_line(const TadlProgram &P, const TadpPointers &ptrs, unsigned sms, cudaStream_t stream);
@@ -113,10 +113,28 @@ unsigned long long item_count(const TadpProgram &P, int ta, int ub)
 
 tad_status zero_fill(float *out, int64_t n, cudaStream_t stream);
 
+// A second stream per plan.  Passes that only stream a tensor through memory (row and column sums, the zero fill of
+// a gradient) are independent of the contraction they accompany and bound by another unit: they run beside it,
+// forked from and joined to the caller's stream with events (which also works inside a stream capture).
+struct Side {
+    cudaStream_t s = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr, filled = nullptr;
+    void release()
+    {
+        if (fork) cudaEventDestroy(fork);
+        if (join) cudaEventDestroy(join);
+        if (filled) cudaEventDestroy(filled);
+        if (s) cudaStreamDestroy(s);
+        s = nullptr; fork = join = filled = nullptr;
+    }
+};
+
 // contraction kernels: one launch of the tile kernel per program
-tad_status launch_contractions(const tad::Kernel &k, const TadpPointers &ptrs, cudaStream_t stream)
+tad_status launch_contractions(const tad::Kernel &k, const TadpPointers &ptrs, cudaStream_t stream, Side *side)
 {
-    for (TadcProgram P : k.contract) {
+    bool forked = false;
+    for (size_t i = 0; i < k.contract.size(); ++i) {
+        TadcProgram P = k.contract[i];
         if (P.ksplit > 1 && !ptrs.part) { tad::set_error("internal: partial-sum buffer missing"); return TAD_ERR_WORKSPACE; }
         // 16-byte copies and stores need 16-byte aligned tensors: fall back to 4-byte accesses otherwise
         auto misaligned = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
@@ -125,26 +143,93 @@ tad_status launch_contractions(const tad::Kernel &k, const TadpPointers &ptrs, c
         if (P.out_vec4 && misaligned(ptrs.out)) P.out_vec4 = 0;
         // the streaming kernel copies B in 16-byte pieces
         if (P.shape == 5 && misaligned(ptrs.in[P.ptrB])) P.shape = 3;
-        const cudaError_t e = tad_launch_contract(P, ptrs, (unsigned)sm_count(), stream);
+        // single-column passes beside the tile kernel: no planes of partial sums, outputs of their own
+        const bool beside = side && k.contract.size() > 1 && i > 0 && P.ksplit == 1 && !P.accumulate && (P.shape == 4 || P.shape == 6);
+        cudaStream_t on = stream;
+        if (beside) {
+            if (!forked) {
+                if (cudaEventRecord(side->fork, stream) != cudaSuccess || cudaStreamWaitEvent(side->s, side->fork, 0) != cudaSuccess) {
+                    tad::set_error("event record / wait failed"); return TAD_ERR_CUDA;
+                }
+                forked = true;
+            }
+            on = side->s;
+        }
+        const cudaError_t e = tad_launch_contract(P, ptrs, (unsigned)sm_count(), on);
         if (e != cudaSuccess) { tad::set_error(std::string("contraction launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
+    }
+    if (forked && (cudaEventRecord(side->join, side->s) != cudaSuccess || cudaStreamWaitEvent(stream, side->join, 0) != cudaSuccess)) {
+        tad::set_error("event record / wait failed"); return TAD_ERR_CUDA;
     }
     return TAD_OK;
 }
 
-tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStream_t stream, char *aux_base = nullptr)
+// does the kernel (or one of the kernels that prepare its tensors) read through this pointer slot?
+bool reads_slot(const tad::Kernel &k, int slot)
+{
+    for (const tad::Kernel &pk : k.pre) if (reads_slot(pk, slot)) return true;
+    if (!k.contract.empty()) {
+        for (const TadcProgram &P : k.contract) {
+            if (P.ptrA == slot || P.ptrB == slot) return true;
+            for (int e = 0; e < P.n_epi; ++e) if ((P.epi_op[e] == TE_MUL_LOAD || P.epi_op[e] == TE_ADD_LOAD) && P.epi_ptr[e] == slot) return true;
+        }
+        return false;
+    }
+    if (!k.ew.empty()) {
+        for (int i = 0; i < k.ew[0].n_loads; ++i) if (k.ew[0].loads[i].ptr == slot) return true;
+        return false;
+    }
+    if (!k.line.empty()) {
+        for (int i = 0; i < k.line[0].n_loads; ++i) if (k.line[0].loads[i].ptr == slot) return true;
+        for (int i = 0; i < k.line[0].n_scale; ++i) if (k.line[0].scale[i].ptr == slot) return true;
+        return false;
+    }
+    for (int i = 0; i < k.prog.n_loads; ++i) if (k.prog.loads[i].ptr == slot) return true;
+    return false;
+}
+
+// a kernel that only streams one tensor through memory into a tensor of its own: a single row- or column-sum pass
+bool streams_only(const tad::Kernel &k)
+{
+    return k.pre.empty() && k.contract.size() == 1 && k.contract[0].ksplit == 1 && !k.contract[0].accumulate &&
+           (k.contract[0].shape == 4 || k.contract[0].shape == 6);
+}
+
+// pending: an event the kernel that writes the output must wait for (the zero fill of its tensor on the second stream)
+tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStream_t stream, char *aux_base = nullptr,
+                  Side *side = nullptr, cudaEvent_t pending = nullptr)
 {
     if (!k.aux.empty()) {
         // auxiliary tensors of this kernel, then the kernels that fill them, in order
         if (!aux_base) { tad::set_error("this plan needs a workspace (auxiliary tensors): pass one of tad_workspace_bytes() bytes"); return TAD_ERR_WORKSPACE; }
         for (const tad::Kernel::Aux &a : k.aux) ptrs.in[a.slot] = reinterpret_cast<const float *>(aux_base + a.offset);
+        // kernels that only stream a tensor run on the second stream, beside the kernels that do not read their result
+        std::vector<int> beside;                       // slots of tensors being written on the second stream
+        auto join = [&]() {
+            if (beside.empty()) return true;
+            beside.clear();
+            return cudaEventRecord(side->join, side->s) == cudaSuccess && cudaStreamWaitEvent(stream, side->join, 0) == cudaSuccess;
+        };
         for (const tad::Kernel &pk : k.pre) {
             TadpPointers pp = ptrs;
             pp.out = reinterpret_cast<float *>(aux_base + k.aux[pk.out_aux].offset);
-            const tad_status st = launch(pk, pp, debug, stream);
+            const bool on_side = side && k.pre.size() > 1 && streams_only(pk);
+            bool wait = false;
+            for (int slot : beside) wait = wait || reads_slot(pk, slot);
+            if (wait && !join()) { tad::set_error("event record / wait failed"); return TAD_ERR_CUDA; }
+            if (on_side) {
+                if (cudaEventRecord(side->fork, stream) != cudaSuccess || cudaStreamWaitEvent(side->s, side->fork, 0) != cudaSuccess) {
+                    tad::set_error("event record / wait failed"); return TAD_ERR_CUDA;
+                }
+                beside.push_back(k.aux[pk.out_aux].slot);
+            }
+            const tad_status st = launch(pk, pp, debug, on_side ? side->s : stream, nullptr, on_side ? nullptr : side);
             if (st != TAD_OK) return st;
         }
+        if (!join()) { tad::set_error("event record / wait failed"); return TAD_ERR_CUDA; }
     }
-    if (!k.contract.empty()) return launch_contractions(k, ptrs, stream);
+    if (pending && cudaStreamWaitEvent(stream, pending, 0) != cudaSuccess) { tad::set_error("event wait failed"); return TAD_ERR_CUDA; }
+    if (!k.contract.empty()) return launch_contractions(k, ptrs, stream, side);
     if (!k.ew.empty()) {
         const cudaError_t e = tad_launch_ew(k.ew[0], ptrs, (unsigned)sm_count(), stream);
         if (e != cudaSuccess) { tad::set_error(std::string("element-wise launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
@@ -176,12 +261,14 @@ tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStrea
     if (items64 == 0) return TAD_OK;
     if (items64 >= (1ull << 32)) { tad::set_error("too many work items"); return TAD_ERR_UNSUPPORTED; }
     const unsigned items = (unsigned)items64;
-    if (k.rich && !debug && k.vec == 16 && k.vec_u == 1) tad_launch_vm_16_1_rich(k.prog, ptrs, debug, items, (unsigned)sm_count(), stream);
+    bool launched = true;
+    if (k.rich && !debug && k.vec == 16 && k.vec_u == 1) launched = tad_launch_vm_16_1_rich(k.prog, ptrs, debug, items, (unsigned)sm_count(), stream);
     else switch (k.vec * 100 + k.vec_u) {
-#define TAD_CASE_VM(TA, UB) case TA * 100 + UB: tad_launch_vm_##TA##_##UB(k.prog, ptrs, debug, items, (unsigned)sm_count(), stream); break;
+#define TAD_CASE_VM(TA, UB) case TA * 100 + UB: launched = tad_launch_vm_##TA##_##UB(k.prog, ptrs, debug, items, (unsigned)sm_count(), stream); break;
     TAD_VM_SHAPES(TAD_CASE_VM)
     default: tad::set_error("internal: no kernel for this vector shape"); return TAD_ERR_UNSUPPORTED;
     }
+    if (!launched) { tad::set_error("internal: this vector shape has no kernel build for the program (bounds checks or a relative loop)"); return TAD_ERR_UNSUPPORTED; }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { tad::set_error(std::string("kernel launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
     if (zsplit > 1) {
@@ -281,8 +368,36 @@ bool fill_inputs(const tad_plan *plan, const float *const *args, const float *df
 
 }  // namespace
 
+namespace {
+std::mutex g_side_mutex;
+thread_local bool t_create_nothing = false;       // set while tad_backward_noalloc runs
+
+// the plan's second stream, created by the first call that can use it (nullptr: run everything on the caller's stream)
+Side *side_of(const tad_plan *plan)
+{
+    std::lock_guard<std::mutex> lock(g_side_mutex);
+    if (plan->side) return static_cast<Side *>(plan->side);
+    if (t_create_nothing) return nullptr;
+    Side *sd = new (std::nothrow) Side();
+    if (!sd) return nullptr;
+    bool ok = cudaStreamCreateWithFlags(&sd->s, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&sd->fork, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&sd->join, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&sd->filled, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { sd->release(); delete sd; cudaGetLastError(); return nullptr; }
+    plan->side = sd;
+    return sd;
+}
+}  // namespace
+
 void tad_release_host_step(const tad_plan *plan)
 {
+    if (plan && plan->side) {
+        Side *sd = static_cast<Side *>(plan->side);
+        sd->release();
+        delete sd;
+        plan->side = nullptr;
+    }
     if (!plan || !plan->host_step) return;
     HostStep *hs = static_cast<HostStep *>(plan->host_step);
     hs->release();
@@ -317,7 +432,7 @@ tad_status tad_forward(const tad_plan *plan, const float *const *args, float *f,
             ? reinterpret_cast<float *>(static_cast<char *>(workspace) + stage_offset(plan, (int)plan->stages.size())) : nullptr;
         aux_base = static_cast<char *>(workspace) + aux_offset(plan);
     }
-    return launch(plan->forward, ptrs, false, (cudaStream_t)cuda_stream, aux_base);
+    return launch(plan->forward, ptrs, false, (cudaStream_t)cuda_stream, aux_base, side_of(plan));
 }
 
 tad_status tad_backward_stage(const tad_plan *plan, const float *const *args, const float *df,
@@ -330,7 +445,7 @@ tad_status tad_backward_stage(const tad_plan *plan, const float *const *args, co
     for (int s = 0; s < (int)plan->stages.size(); ++s) {
         ptrs.out = reinterpret_cast<float *>(static_cast<char *>(workspace) + stage_offset(plan, s));
         tad_status st = launch(plan->stages[s], ptrs, plan->opt.debug_bounds != 0, (cudaStream_t)cuda_stream,
-                               workspace ? static_cast<char *>(workspace) + aux_offset(plan) : nullptr);
+                               workspace ? static_cast<char *>(workspace) + aux_offset(plan) : nullptr, side_of(plan));
         if (st != TAD_OK) return st;
     }
     return TAD_OK;
@@ -345,14 +460,28 @@ tad_status tad_backward_arg(const tad_plan *plan, const float *const *args, cons
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     TadpPointers ptrs{};
     if (!fill_inputs(plan, args, df, workspace, ptrs)) return TAD_ERR_INVALID_ARG;
+    Side *side = side_of(plan);
+    cudaEvent_t pending = nullptr;
     if (plan->arg_kernels[arg].empty() || plan->arg_zero_fill[arg]) {
-        tad_status st = zero_fill(darg, plan->arg_elems[arg], stream);
+        // the fill of a gradient whose first kernel prepares auxiliary tensors runs beside that preparation
+        const bool beside = side && !plan->arg_kernels[arg].empty() && !plan->backward[plan->arg_kernels[arg][0]].pre.empty();
+        if (beside) {
+            if (cudaEventRecord(side->fork, stream) != cudaSuccess || cudaStreamWaitEvent(side->s, side->fork, 0) != cudaSuccess) {
+                tad::set_error("event record / wait failed"); return TAD_ERR_CUDA;
+            }
+        }
+        tad_status st = zero_fill(darg, plan->arg_elems[arg], beside ? side->s : stream);
         if (st != TAD_OK) return st;
+        if (beside) {
+            if (cudaEventRecord(side->filled, side->s) != cudaSuccess) { tad::set_error("event record failed"); return TAD_ERR_CUDA; }
+            pending = side->filled;
+        }
     }
     ptrs.out = darg;
     for (int ki : plan->arg_kernels[arg]) {
         tad_status st = launch(plan->backward[ki], ptrs, plan->opt.debug_bounds != 0, stream,
-                               workspace ? static_cast<char *>(workspace) + aux_offset(plan) : nullptr);
+                               workspace ? static_cast<char *>(workspace) + aux_offset(plan) : nullptr, side, pending);
+        pending = nullptr;
         if (st != TAD_OK) return st;
     }
     return TAD_OK;
@@ -526,7 +655,11 @@ tad_status tad_backward_noalloc(const tad_plan *plan, const float *const *args, 
         e = cudaMemsetAsync(scratch, 0, 256, (cudaStream_t)cuda_stream);
         if (e != cudaSuccess) { tad::set_error(std::string("clearing the debug word: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
     }
-    return tad_backward(plan, args, df, dargs, scratch, TAD_NOALLOC_SCRATCH_BYTES, cuda_stream);
+    // (this entry point creates nothing: the second stream is used only if an earlier call of another entry point made it)
+    t_create_nothing = true;
+    const tad_status st = tad_backward(plan, args, df, dargs, scratch, TAD_NOALLOC_SCRATCH_BYTES, cuda_stream);
+    t_create_nothing = false;
+    return st;
 }
 
 tad_status tad_measure_fp32_rate(void *cuda_stream, double *tflops)

@@ -184,14 +184,19 @@ tad_vm_kernel(const __grid_constant__ TadpProgram P, const __grid_constant__ Tad
 #endif
 
 // Builds per shape: plain, with the relative-loop support (no element variable) and, for narrow
-// shapes, with bounds checks.
-void TAD_LAUNCH_NAME(TAD_TA, TAD_UB)(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream)
+// shapes, with bounds checks.  False when the shape has no build for what the program asks: nothing was launched.
+bool TAD_LAUNCH_NAME(TAD_TA, TAD_UB)(const TadpProgram &prog, const TadpPointers &ptrs, bool debug, unsigned items, unsigned sms, cudaStream_t stream)
 {
     constexpr int TA = TAD_TA, UB = TAD_UB;
     constexpr unsigned WPB = VmCfg<TA, UB>::WARPS;
     // one warp per work item, grid-stride; at most 128 warps' worth of blocks per SM
     const unsigned blocks = std::min((items + WPB - 1) / WPB, sms * (128u / WPB));
-    if (debug) { if constexpr (TA <= 4 && UB == 1) tad_vm_kernel<TA, UB, true, true><<<blocks, WPB * 32, 0, stream>>>(prog, ptrs, items); }
-    else if (prog.rel_var >= 0) { if constexpr (UB == 1) tad_vm_kernel<TA, UB, false, true><<<blocks, WPB * 32, 0, stream>>>(prog, ptrs, items); }
-    else tad_vm_kernel<TA, UB, false, false><<<blocks, WPB * 32, 0, stream>>>(prog, ptrs, items);
+    if (debug) {
+        if constexpr (TA <= 4 && UB == 1) tad_vm_kernel<TA, UB, true, true><<<blocks, WPB * 32, 0, stream>>>(prog, ptrs, items);
+        else return false;
+    } else if (prog.rel_var >= 0) {
+        if constexpr (UB == 1) tad_vm_kernel<TA, UB, false, true><<<blocks, WPB * 32, 0, stream>>>(prog, ptrs, items);
+        else return false;
+    } else tad_vm_kernel<TA, UB, false, false><<<blocks, WPB * 32, 0, stream>>>(prog, ptrs, items);
+    return true;
 }
