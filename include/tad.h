@@ -26,8 +26,14 @@
  *   - tad_compile / tad_plan_* are host-only and touch no GPU;
  *   - tad_forward / tad_backward take DEVICE pointers, enqueue work on the given
  *     CUDA stream (a cudaStream_t passed as void*, NULL = default stream), do not
- *     synchronise and allocate nothing;
- *   - the caller owns every buffer; a plan is immutable and may be shared;
+ *     synchronise and allocate no device memory.  Passes of a call that are independent
+ *     of each other (the zero fill of a gradient, a row or column sum beside a contraction)
+ *     may run on a second stream that the plan owns (created by the first launch, released
+ *     by tad_destroy); it is forked from and joined to the given stream with events, so
+ *     the call is complete in the given stream's order and may be captured into a graph;
+ *   - the caller owns every buffer; a plan's programs are immutable and the plan may be
+ *     shared, but two host threads must not launch from the same plan at the same time
+ *     (they would share that second stream's events);
  *   - every function returns a status; tad_last_error() gives a thread-local text.
  */
 #ifndef TAD_INCLUDE_TAD_H
