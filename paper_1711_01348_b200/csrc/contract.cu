@@ -1,6 +1,6 @@
 // Tile kernel for contraction programs (contract.h): a thread block owns a BM x BN tile of
 // outputs, gathers BK summation indices of both operands at a time into shared memory with
-// asynchronous copies (three stages in flight), and every thread keeps a TM x TN tile of sums in
+// asynchronous copies (two stages), and every thread keeps a TM x TN tile of sums in
 // registers that it feeds from shared memory with 128-bit loads.  Operand elements outside a
 // guard, past the end of the summation range or in the ragged edge of a tile arrive as zeros
 // (zero-fill copies), so the multiply-add loop has no tests.  No atomics: a summation split over
