@@ -326,6 +326,24 @@ tad_status tad_plan_kernel_stats(const tad_plan *plan, int32_t which, tad_kernel
 /* Human-readable listing of the compiled program (`which` as above); returns bytes needed. */
 size_t tad_plan_disassemble(const tad_plan *plan, int32_t which, char *buf, size_t cap);
 
+/*
+ * The expression (which = -1) or the derived derivative through index expression `which` as text in the
+ * notation of the listing in Sec. 6:
+ *     f[i; j] = exp (-sum{k}_0^4 (...))
+ *     dx[dx_0; dx_1] = if {conditions} then (sum{dx_z1}_lo^hi (sum{dx_z0}_lo^hi (term))) else (0)
+ * Index positions of the term are written as their affine forms alpha = I beta + K z (Sec. 5.1); kernel
+ * coordinates are named by kernel column (dx_z0, dx_z1, ...) and nested in the plan's loop order; ranges are the
+ * bound rows of Sec. 4.2 (max [..] / min [..], with ceil / floor where a row does not divide); conditions are the
+ * cokernel rows (= 0), divisibility by an invariant factor (mod n = 0, which the paper's listing never needs) and
+ * guards (<= 0).  The kernel basis, and with it names and signs of the z, is the plan's: any unimodular
+ * recombination describes the same set.  The text describes the derivative as derived, before the expression
+ * clean-up that the kernels run.
+ *   arg_names  n_args strings or NULL (x0, x1, ...);  idx_names  n_out_dims + n_sum_idx strings or NULL (i, j, k, ...)
+ * Host only.  Returns the bytes needed including the terminator (0: no such expression); writes at most cap.
+ */
+size_t tad_plan_print(const tad_plan *plan, int32_t which, const char *const *arg_names, const char *const *idx_names,
+                      char *buf, size_t cap);
+
 /* Host-only pieces of Sec. 4, exported for tests.  Matrices are row-major int64. */
 tad_status tad_extended_euclid(int64_t a, int64_t b, int64_t *gcd, int64_t *x, int64_t *y);
 tad_status tad_smith_normal_form(const int64_t *A, int32_t n_rows, int32_t n_cols,

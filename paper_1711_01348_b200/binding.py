@@ -26,7 +26,7 @@ EXPORTS = ["tad_compile", "tad_destroy", "tad_workspace_bytes", "tad_forward", "
            "tad_backward_stage", "tad_backward_arg", "tad_plan_num_stages", "tad_backward_noalloc",
            "tad_staging_bytes", "tad_step_host", "tad_last_error", "tad_debug_status",
            "tad_plan_access_info", "tad_plan_bound_row", "tad_plan_enumerate", "tad_plan_kernel_stats",
-           "tad_plan_disassemble", "tad_extended_euclid", "tad_smith_normal_form", "tad_fourier_motzkin",
+           "tad_plan_disassemble", "tad_plan_print", "tad_extended_euclid", "tad_smith_normal_form", "tad_fourier_motzkin",
            "tad_measure_fp32_rate"]
 
 
@@ -101,6 +101,8 @@ def _load() -> C.CDLL:
     lib.tad_plan_kernel_stats.argtypes = [vp, C.c_int32, C.POINTER(KernelStats)]
     lib.tad_plan_disassemble.argtypes = [vp, C.c_int32, C.c_char_p, C.c_size_t]
     lib.tad_plan_disassemble.restype = C.c_size_t
+    lib.tad_plan_print.argtypes = [vp, C.c_int32, C.POINTER(C.c_char_p), C.POINTER(C.c_char_p), C.c_char_p, C.c_size_t]
+    lib.tad_plan_print.restype = C.c_size_t
     lib.tad_extended_euclid.argtypes = [C.c_int64, C.c_int64, i64p, i64p, i64p]
     lib.tad_smith_normal_form.argtypes = [i64p, C.c_int32, C.c_int32, i64p, i64p, i64p, i32p]
     lib.tad_fourier_motzkin.argtypes = [i64p, C.c_int32, C.c_int32, C.c_int32, i32p, i32p,
@@ -265,6 +267,20 @@ class Plan:
         n = lib.tad_plan_disassemble(self._h, which, None, 0)
         buf = C.create_string_buffer(n)
         lib.tad_plan_disassemble(self._h, which, buf, n)
+        return buf.value.decode()
+
+    def print(self, which: int, arg_names=None, idx_names=None) -> str:
+        """tad_plan_print: the expression (which = -1) or the derivative through index expression `which`."""
+        def strings(names):
+            if names is None:
+                return None
+            return (C.c_char_p * len(names))(*[n.encode() for n in names])
+        a, i = strings(arg_names), strings(idx_names)
+        n = lib.tad_plan_print(self._h, which, a, i, None, 0)
+        if n == 0:
+            return ""
+        buf = C.create_string_buffer(n)
+        lib.tad_plan_print(self._h, which, a, i, buf, n)
         return buf.value.decode()
 
 

@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libtad.so")
-SOURCES = ["intalg.cpp", "plan.cpp", "codegen.cpp", "contract_gen.cpp", "factor.cpp", "line_gen.cpp", "api.cpp", "runtime.cu", "contract.cu", "ew.cu", "line.cu"]
+SOURCES = ["intalg.cpp", "plan.cpp", "codegen.cpp", "contract_gen.cpp", "factor.cpp", "line_gen.cpp", "print.cpp", "api.cpp", "runtime.cu", "contract.cu", "ew.cu", "line.cu"]
 HEADERS = ["intalg.h", "plan.h", "gen.h", "program.h", "contract.h", "ew.h", "line.h", "vm.cuh", "vm_shapes.h", "vm_inst.cu",
            os.path.join("..", "..", "include", "tad.h")]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]

@@ -147,6 +147,20 @@ size_t tad_plan_disassemble(const tad_plan *plan, int32_t which, char *buf, size
     return k->listing.size() + 1;
 }
 
+size_t tad_plan_print(const tad_plan *plan, int32_t which, const char *const *arg_names, const char *const *idx_names,
+                      char *buf, size_t cap)
+{
+    if (!plan) return 0;
+    std::string text;
+    if (guarded([&] { text = print_expression(*plan, which, arg_names, idx_names); }) != TAD_OK || text.empty()) return 0;
+    if (buf && cap) {
+        size_t n = std::min(cap - 1, text.size());
+        std::memcpy(buf, text.data(), n);
+        buf[n] = 0;
+    }
+    return text.size() + 1;
+}
+
 tad_status tad_extended_euclid(int64_t a, int64_t b, int64_t *g, int64_t *x, int64_t *y)
 {
     return guarded([&] {

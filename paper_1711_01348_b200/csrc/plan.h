@@ -132,4 +132,7 @@ void generate_forward(tad_plan &p);
 void generate_stages(tad_plan &p);
 void generate_backward(tad_plan &p, int q);
 
+// print.cpp: the expression (which = -1) or the derivative through index expression `which` in the notation of Sec. 6
+std::string print_expression(const tad_plan &p, int which, const char *const *arg_names, const char *const *idx_names);
+
 }  // namespace tad
