@@ -210,13 +210,25 @@ tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStrea
             beside.clear();
             return cudaEventRecord(side->join, side->s) == cudaSuccess && cudaStreamWaitEvent(stream, side->join, 0) == cudaSuccess;
         };
-        for (const tad::Kernel &pk : k.pre) {
+        // Launch order: the streaming passes move up to right behind the last kernel whose result they read, so that
+        // they are issued before the long kernels they run beside (every tensor has one writer: moving a kernel up
+        // past kernels that neither feed it nor read it changes nothing)
+        const bool use_side = side && k.pre.size() > 1;
+        std::vector<int> order;
+        for (int i = 0; i < (int)k.pre.size(); ++i) {
+            if (!(use_side && streams_only(k.pre[i]))) { order.push_back(i); continue; }
+            size_t at = order.size();
+            while (at > 0 && !reads_slot(k.pre[i], k.aux[k.pre[order[at - 1]].out_aux].slot)) --at;
+            order.insert(order.begin() + at, i);
+        }
+        for (int i : order) {
+            const tad::Kernel &pk = k.pre[i];
             TadpPointers pp = ptrs;
             pp.out = reinterpret_cast<float *>(aux_base + k.aux[pk.out_aux].offset);
-            const bool on_side = side && k.pre.size() > 1 && streams_only(pk);
+            const bool on_side = use_side && streams_only(pk);
             bool wait = false;
             for (int slot : beside) wait = wait || reads_slot(pk, slot);
-            if (wait && !join()) { tad::set_error("event record / wait failed"); return TAD_ERR_CUDA; }
+            if (wait && !on_side && !join()) { tad::set_error("event record / wait failed"); return TAD_ERR_CUDA; }
             if (on_side) {
                 if (cudaEventRecord(side->fork, stream) != cudaSuccess || cudaStreamWaitEvent(side->s, side->fork, 0) != cudaSuccess) {
                     tad::set_error("event record / wait failed"); return TAD_ERR_CUDA;
