@@ -410,3 +410,47 @@ def test_workspace_too_small_or_misaligned_is_refused_before_any_launch():
         with pytest.raises(TadError) as ei:
             big.forward(args, fake, 0, ws_ptr, ws_bytes)
         assert ei.value.code == "TAD_ERR_WORKSPACE", (ws_ptr, ws_bytes)
+
+
+def test_interpreter_shapes_asked_for_have_a_kernel_build():
+    """The interpreter is built with bounds checks for the narrow shapes only (up to 4 values per thread, no
+    element variable) and with relative loops only without an element variable; a launcher asked for anything
+    else launches nothing and reports it.  The code generator must therefore never ask: every kernel header of
+    debug plans and of plans with a relative loop is checked, over the reduced workloads and random expressions
+    of every level."""
+    from paper_1711_01348_b200 import TadError
+    from workloads import configs as W
+    from workloads.random_expr import random_expression
+
+    def kernels(plan, n_access):
+        for which in [-1] + list(range(n_access)) + [-2 - s for s in range(plan.num_stages())]:
+            try:
+                text = plan.disassemble(which)
+            except TadError:
+                continue
+            head = None
+            for line in text.splitlines():
+                if line.startswith("; vars="):
+                    head = dict(item.split("=") for item in line.lstrip("; ").split())
+                    yield head, False
+                elif line.startswith("; loop ") and " relative=1" in line and head is not None:
+                    yield head, True
+
+    exprs = [W.REDUCED[k]() for k in sorted(W.REDUCED)]
+    exprs += [random_expression(seed, large=lv) for lv in (0, 1, 3, 4, 5) for seed in range(6)]
+    seen_debug = seen_relative = 0
+    for e in exprs:
+        for debug in (False, True):
+            try:
+                plan = Plan(e, debug_bounds=debug)
+            except TadError:
+                continue
+            for head, relative in kernels(plan, len(e.accesses)):
+                ta, ub = (int(v.rstrip("r")) for v in head["vec"].split("x"))
+                if debug:
+                    assert ta <= 4 and ub == 1, head
+                    seen_debug += 1
+                if relative:
+                    assert ub == 1, head
+                    seen_relative += 1
+    assert seen_debug > 50
