@@ -29,10 +29,11 @@ namespace {
 
 // Adds the zsplit planes of partial sums up and writes the gradient elements: compact index
 // c -> outer variables -> output offset.  A block takes 32 consecutive cells (one per lane,
-// so that every plane is read in full sectors); its warp w adds planes w, w + 32, ... in that
+// so that every plane is read in full sectors); its warp w adds planes w, w + W, ... in that
 // order and the warps' subtotals are added in warp order: the same association every run.
+// W = 8 warps per block for up to 128 planes (many small blocks, all resident at once), 32 beyond.
 // Masked gradients write only outputs whose flag says that some term was accumulated.
-constexpr int REDUCE_WARPS = 32;
+template <int REDUCE_WARPS>
 __global__ void __launch_bounds__(REDUCE_WARPS * 32)
 tad_reduce_partials(const __grid_constant__ TadpProgram P, float *out, const float *part)
 {
@@ -65,6 +66,12 @@ tad_reduce_partials(const __grid_constant__ TadpProgram P, float *out, const flo
         }
         __syncthreads();
     }
+}
+
+void launch_reduce_partials(const TadpProgram &P, const TadpPointers &ptrs, unsigned blocks, cudaStream_t stream)
+{
+    if (P.zsplit > 128) tad_reduce_partials<32><<<blocks, 32 * 32, 0, stream>>>(P, ptrs.out, ptrs.part);
+    else tad_reduce_partials<8><<<blocks, 8 * 32, 0, stream>>>(P, ptrs.out, ptrs.part);
 }
 
 // Sixteen independent multiply-add chains per thread, operands in registers only: the rate at which this GPU
@@ -254,7 +261,7 @@ tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStrea
         if (e == cudaSuccess && L.zsplit > 1) {
             const unsigned n = (unsigned)k.prog.part_limit;
             const unsigned rblocks = std::min((n + 31u) / 32u, (unsigned)sm_count() * 8u);
-            tad_reduce_partials<<<rblocks, REDUCE_WARPS * 32, 0, stream>>>(k.prog, ptrs.out, ptrs.part);
+            launch_reduce_partials(k.prog, ptrs, rblocks, stream);
             e = cudaGetLastError();
         }
         if (e != cudaSuccess) { tad::set_error(std::string("line-sum launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
@@ -286,7 +293,7 @@ tad_status launch(const tad::Kernel &k, TadpPointers ptrs, bool debug, cudaStrea
     if (zsplit > 1) {
         const unsigned n = (unsigned)k.prog.part_limit;
         const unsigned rblocks = std::min((n + 31u) / 32u, (unsigned)sm_count() * 8u);
-        tad_reduce_partials<<<rblocks, REDUCE_WARPS * 32, 0, stream>>>(k.prog, ptrs.out, ptrs.part);
+        launch_reduce_partials(k.prog, ptrs, rblocks, stream);
         e = cudaGetLastError();
         if (e != cudaSuccess) { tad::set_error(std::string("reduce launch failed: ") + cudaGetErrorString(e)); return TAD_ERR_CUDA; }
     }
